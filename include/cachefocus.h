@@ -1,0 +1,217 @@
+/*
+ * cachefocus.h -- C ABI of the CacheFocus query-time path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the part of CacheFocus (arXiv 2502.11101) that runs between
+ * retrieval and decoding: cached per-document keys are moved to new positions by a rotary
+ * delta rotation (Sec. 2.3, Eq. 5), the query tokens attend over the concatenated
+ * re-positioned document caches (Eq. 1), every document's share of the attention mass is
+ * accumulated over layers, and at pruning layers only the best documents survive and are
+ * re-allocated next to the query (Sec. 2.4 Algorithm 2, Sec. 2.5).
+ *
+ * Conventions
+ *   - Every function returns CF_OK (0) or a CF_ERR_* code; cf_error_string() names it.
+ *   - "host" pointers are ordinary process memory, read or written only during the call.
+ *     "device" pointers are CUDA global memory owned by the caller.  The library allocates
+ *     and frees no device memory and never synchronises the device, except cf_plan_status()
+ *     which copies one word back.
+ *   - Device work is queued on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and is asynchronous.  Calls on one stream execute in order.
+ *   - Key/value store layout: one layer is `[total_tokens][n_kv_heads][head_dim]` with
+ *     `token_stride` elements between rows; the documents of all requests of a batch are
+ *     laid end to end; document i owns rows doc_offsets[i] .. doc_offsets[i+1]-1 and its
+ *     token t was cached at position doc_src_start[i] + t.  Keys are stored already
+ *     rotary-encoded at those positions.  Values are never modified.
+ *   - Query/output layout: `[n_requests][q_len][n_q_heads][head_dim]`, contiguous.  The
+ *     query states must already be rotary-encoded at positions query_start + j.
+ *   - Query head h reads key/value head h / (n_q_heads / n_kv_heads).
+ *   - Document ids inside a request are local (0 .. n_b-1); arrays indexed by document use
+ *     the global index req_doc_begin[b] + local id.
+ */
+#ifndef CACHEFOCUS_H_
+#define CACHEFOCUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CF_OK               0
+#define CF_ERR_INVALID_ARG  1   /* NULL pointer, negative size, inconsistent geometry            */
+#define CF_ERR_RANGE        2   /* the kept documents do not fit the positional range           */
+#define CF_ERR_UNSUPPORTED  3   /* head_dim / dtype / layout combination that is not built      */
+#define CF_ERR_WORKSPACE    4   /* plan or workspace buffer too small or misaligned             */
+#define CF_ERR_CUDA         5   /* a CUDA runtime or driver call failed                         */
+#define CF_ERR_TIMEOUT      6   /* a bounded device-side wait expired (reported via the plan)   */
+
+#define CF_BF16 0
+#define CF_F32  1
+
+#define CF_ROPE_HALF        0   /* slice p = coordinates (p, p + head_dim/2)                    */
+#define CF_ROPE_INTERLEAVED 1   /* slice p = coordinates (2p, 2p + 1)                           */
+
+#define CF_ALLOC_NONE  0        /* survivors keep their positions, gaps stay                    */
+#define CF_ALLOC_ALIGN 1        /* Dynamic Positional Allocation ("align", Sec. 2.5)            */
+#define CF_ALLOC_SORT  2        /* Attention-Guided Allocation ("sort", Sec. 2.5)               */
+
+#define CF_TILE_TOKENS 128      /* key tiles never straddle two documents                       */
+#define CF_MAX_DOCS_PER_REQUEST 1024
+#define CF_MAX_SPLITS 64
+
+/* Model-side geometry.  head_dim 64 or 128; pos_range = the model's positional range L of
+ * Eq. 6; rope_theta = base of the rotary frequencies theta^(-2p/head_dim). */
+typedef struct cf_geom {
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim;
+    int32_t dtype;        /* CF_BF16 | CF_F32: storage type of Q, K, V and the output */
+    int32_t rope_layout;  /* CF_ROPE_HALF | CF_ROPE_INTERLEAVED */
+    int32_t pos_range;
+    double  rope_theta;
+} cf_geom;
+
+/* One batch of independent requests over one packed store.  The three arrays are DEVICE
+ * memory and stay owned by the caller; they must remain valid while queued work uses them. */
+typedef struct cf_batch {
+    int32_t n_requests;
+    int32_t n_docs_total;      /* documents of all requests                                      */
+    int32_t q_len;             /* query tokens per request                                       */
+    int32_t prefix_len;        /* positions [0, prefix_len) are never given to documents         */
+    int32_t tail_reserve;      /* positions kept free after query_start (query + new tokens)     */
+    int32_t n_reuse;           /* number of parallel windows; 0 = Eq. 6                          */
+    int32_t tiles_hint;        /* upper bound of live key tiles per request (0 = derive from
+                                  total_tokens); only steers grid sizes, never correctness       */
+    int32_t reserved;
+    int64_t total_tokens;      /* rows in one layer of the store                                 */
+    int64_t token_stride;      /* elements between consecutive rows, >= n_kv_heads*head_dim      */
+    const int32_t* req_doc_begin;  /* device [n_requests+1]                                      */
+    const int32_t* doc_offsets;    /* device [n_docs_total+1]                                    */
+    const int32_t* doc_src_start;  /* device [n_docs_total]                                      */
+} cf_batch;
+
+/* Byte offsets of the fields inside a plan buffer (device memory written by cf_plan_init and
+ * cf_prune_topk, read by the other device calls).  All int32 unless noted. */
+typedef struct cf_plan_layout {
+    size_t total_bytes;
+    size_t status;          /* [4]   status[0] = first CF_ERR_* raised on the device, 0 if none  */
+    size_t kept;            /* [n_docs_total] local ids by rank, request b starts at
+                                     req_doc_begin[b]; rank 0 sits next to the query              */
+    size_t kept_count;      /* [n_requests]                                                      */
+    size_t dst_start;       /* [n_docs_total] destination position of token 0, -1 if pruned      */
+    size_t group;           /* [n_docs_total] window index, -1 if pruned                         */
+    size_t n_reuse;         /* [n_requests]                                                      */
+    size_t query_start;     /* [n_requests]                                                      */
+    size_t n_tiles;         /* [n_requests]                                                      */
+    size_t doc_tile_begin;  /* [n_docs_total] first tile of the document (index into tile_*)     */
+    size_t doc_tile_count;  /* [n_docs_total] 0 if pruned                                        */
+    size_t tile_doc;        /* [max_tiles] global document index                                 */
+    size_t tile_row0;       /* [max_tiles] first store row                                       */
+    size_t tile_len;        /* [max_tiles] 1..CF_TILE_TOKENS                                     */
+    size_t trig;            /* float [n_docs_total][head_dim/2][2] = cos, sin of delta*freq      */
+    int32_t max_tiles;
+    int32_t reserved;
+} cf_plan_layout;
+
+const char* cf_error_string(int code);
+
+/* ---------------------------------------------------------------- host-side integer steps */
+
+/* Adaptive Re-Positioning (Sec. 2.3.1, Eq. 6) and Adaptive Positional Allocation (Sec. 2.5)
+ * for ONE request, on the host.  All pointers are host memory.
+ *   doc_len[n_docs]   token count of every document of the request
+ *   order[n_kept]     distinct document ids; order[0] is placed closest to the query
+ *   n_reuse           >0 forces the number of parallel windows, 0 selects
+ *                     ceil(n_kept / floor(capacity / l_C)) with l_C = longest kept document and
+ *                     capacity = pos_range - prefix_len - tail_reserve
+ *   query_start       <0: the query closes the usable range (pos_range - tail_reserve)
+ * Rank r goes to window r mod n_reuse; inside a window documents take sequential positions,
+ * packed backwards from query_start.  Outputs: dst_start[n_docs], group[n_docs] (-1 for
+ * documents not in `order`), *n_reuse_out, *query_start_out (either may be NULL).
+ * Errors: CF_ERR_INVALID_ARG (bad ids, empty documents), CF_ERR_RANGE (does not fit). */
+int cf_allocate_positions(const cf_geom* geom, int32_t n_docs, const int32_t* doc_len,
+                          const int32_t* order, int32_t n_kept, int32_t prefix_len,
+                          int32_t tail_reserve, int32_t n_reuse, int32_t query_start,
+                          int32_t* dst_start, int32_t* group, int32_t* n_reuse_out,
+                          int32_t* query_start_out);
+
+/* Linear pruning schedule of App. C: pruning after every `every`-th layer (1-based),
+ * k_prune = (k - k_finish) / (n_layers / every) documents each time, any remainder removed at
+ * the last pruning layer.  Writes up to `capacity` (layer, keep) pairs into host arrays and the
+ * number of pruning layers into *count. */
+int cf_schedule_linear(int32_t n_layers, int32_t every, int32_t k, int32_t k_finish,
+                       int32_t capacity, int32_t* layers, int32_t* keeps, int32_t* count);
+
+/* ------------------------------------------------------------------------ device-side plan */
+
+/* Field offsets and size of the plan buffer for this geometry and batch (host computation). */
+int cf_plan_layout_of(const cf_geom* geom, const cf_batch* batch, cf_plan_layout* layout);
+
+/* Start a request batch (Algorithm 2, "Init"): sets the kept list of every request from
+ * `order` (device [n_docs_total], local ids by rank laid out like `kept`; NULL = identity,
+ * i.e. retrieval order) and `kept_count` (device [n_requests]; NULL = all documents), then
+ * allocates positions (same rules as cf_allocate_positions, query_start < 0 = end of range),
+ * and derives per-document rotation tables and the key-tile list.  `plan` is device memory of
+ * at least cf_plan_layout.total_bytes bytes, 256-byte aligned.  Device-side failures (range
+ * overflow) are recorded in the plan's status word. */
+int cf_plan_init(const cf_geom* geom, const cf_batch* batch, const int32_t* order,
+                 const int32_t* kept_count, int32_t query_start, void* plan, size_t plan_bytes,
+                 void* stream);
+
+/* Copies the plan's status word back (synchronises `stream`); returns it as the error code. */
+int cf_plan_status(const cf_geom* geom, const cf_batch* batch, const void* plan, void* stream);
+
+/* ------------------------------------------------------------------------------ hot path */
+
+/* Cache Re-Positioning (Eq. 5; Algorithm 2 Phase 2): for every kept document of the plan and
+ * every layer, rotates each two-dimensional slice of each key row by the angle of
+ * (dst_start - src_start) positions and writes it to k_out (same layout; k_out may equal k_in;
+ * rows of pruned documents are not written).  `n_layers` layers are processed,
+ * `layer_stride` elements apart.  Arithmetic: fp32, one rounding to the storage type. */
+int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                       int32_t n_layers, int64_t layer_stride, const void* k_in, void* k_out,
+                       void* stream);
+
+/* Scratch needed by cf_query_prefill_attn for this batch (bytes; 256-byte aligned buffer).
+ * Grows with batch->tiles_hint: ask with the largest hint that will be used. */
+size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch);
+
+/* One layer of query-token attention over the kept documents' caches (Eq. 1; Algorithm 2,
+ * "layer_l" restricted to its attention over the cached documents), fused with the
+ * re-positioning of the keys (Eq. 5): keys are read from the un-repositioned store `k_cache`
+ * and rotated on the way in.
+ *   q, out        device [n_requests][q_len][n_q_heads][head_dim], storage type
+ *   k_cache, v_cache  device, one layer of the store
+ *   softmax_scale 0 selects 1/sqrt(head_dim)
+ *   lse           device float [n_requests][n_q_heads][q_len], natural log of the softmax
+ *                 denominator (lets the caller merge further key blocks); may be NULL
+ *   doc_scores    device float [n_docs_total]: share of the attention mass on each document,
+ *                 averaged over heads and query rows (sums to 1 per request, 0 for pruned
+ *                 documents); may be NULL
+ *   score_accum   device float [n_docs_total], += doc_scores (Algorithm 2: S <- S + s^l);
+ *                 may be NULL
+ * Accumulation is fp32; reductions run in a fixed order (results are run-to-run identical). */
+int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                          const void* q, const void* k_cache, const void* v_cache,
+                          float softmax_scale, void* out, float* lse, float* doc_scores,
+                          float* score_accum, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
+/* Layer-Adaptive Cache Pruning step (Algorithm 2: argsort of S, prun) followed by the
+ * re-allocation of the survivors (Sec. 2.5), all on the device: per request keeps the `keep`
+ * documents with the largest score_accum among the kept ones (ties: lower id), orders them
+ * (ALIGN/NONE: previous order, SORT: by score, best first), re-allocates positions with the
+ * request's query_start unchanged (NONE: positions untouched) and rebuilds rotation tables and
+ * tile list in `plan`.  keep_per_request (device [n_requests]) overrides `keep` when not NULL. */
+int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
+                  const float* score_accum, int32_t keep, const int32_t* keep_per_request,
+                  int32_t strategy, void* stream);
+
+/* Selects the attention kernel: 0 = automatic (tensor-core kernel when the geometry allows),
+ * 1 = force the portable CUDA-core kernel.  Process-wide; meant for tests and debugging. */
+int cf_set_attn_path(int32_t path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CACHEFOCUS_H_ */

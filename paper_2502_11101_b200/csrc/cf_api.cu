@@ -1,0 +1,375 @@
+// C ABI entry points: argument checking, buffer layouts, the host-side integer steps.
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <vector>
+
+#include "cf_common.cuh"
+
+namespace cf {
+
+GeomView make_geom_view(const cf_geom* g) {
+    GeomView v;
+    v.n_q_heads = g->n_q_heads;
+    v.n_kv_heads = g->n_kv_heads;
+    v.head_dim = g->head_dim;
+    v.dtype = g->dtype;
+    v.rope_layout = g->rope_layout;
+    v.pos_range = g->pos_range;
+    v.rope_theta = g->rope_theta;
+    return v;
+}
+
+BatchView make_batch_view(const cf_batch* b) {
+    BatchView v;
+    v.n_requests = b->n_requests;
+    v.n_docs_total = b->n_docs_total;
+    v.q_len = b->q_len;
+    v.prefix_len = b->prefix_len;
+    v.tail_reserve = b->tail_reserve;
+    v.n_reuse = b->n_reuse;
+    v.total_tokens = b->total_tokens;
+    v.token_stride = b->token_stride;
+    v.req_doc_begin = b->req_doc_begin;
+    v.doc_offsets = b->doc_offsets;
+    v.doc_src_start = b->doc_src_start;
+    return v;
+}
+
+int validate(const cf_geom* g, const cf_batch* b) {
+    if (!g) return CF_ERR_INVALID_ARG;
+    if (g->n_q_heads <= 0 || g->n_kv_heads <= 0 || g->n_q_heads % g->n_kv_heads != 0)
+        return CF_ERR_INVALID_ARG;
+    if (g->pos_range <= 0 || !(g->rope_theta > 1.0)) return CF_ERR_INVALID_ARG;
+    if (g->head_dim != 64 && g->head_dim != 128) return CF_ERR_UNSUPPORTED;
+    if (g->dtype != CF_BF16 && g->dtype != CF_F32) return CF_ERR_UNSUPPORTED;
+    if (g->rope_layout != CF_ROPE_HALF && g->rope_layout != CF_ROPE_INTERLEAVED)
+        return CF_ERR_UNSUPPORTED;
+    if (!b) return CF_OK;
+    if (b->n_requests <= 0 || b->n_docs_total < 0 || b->q_len <= 0 || b->prefix_len < 0 ||
+        b->tail_reserve < 0 || b->n_reuse < 0 || b->tiles_hint < 0 || b->total_tokens < 0)
+        return CF_ERR_INVALID_ARG;
+    if (b->total_tokens > 0x7fffffffLL - kTile) return CF_ERR_INVALID_ARG;
+    if (b->token_stride < (int64_t)g->n_kv_heads * g->head_dim) return CF_ERR_INVALID_ARG;
+    // rows are moved in 16-byte vectors
+    const int esize = g->dtype == CF_BF16 ? 2 : 4;
+    if ((b->token_stride * esize) % 16 != 0) return CF_ERR_INVALID_ARG;
+    if (!b->req_doc_begin || !b->doc_offsets || !b->doc_src_start) return CF_ERR_INVALID_ARG;
+    if (g->pos_range - b->prefix_len - b->tail_reserve <= 0) return CF_ERR_RANGE;
+    return CF_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static void plan_layout(const cf_geom* g, const cf_batch* b, cf_plan_layout* L) {
+    const size_t nd = (size_t)b->n_docs_total, nb = (size_t)b->n_requests;
+    const size_t max_tiles = nd + (size_t)(b->total_tokens / kTile) + 1;
+    size_t off = 0;
+    auto take = [&](size_t count, size_t elem) {
+        size_t at = off;
+        off = align_up(off + count * elem, 256);
+        return at;
+    };
+    L->status = take(4, 4);
+    L->kept = take(nd, 4);
+    L->kept_count = take(nb, 4);
+    L->dst_start = take(nd, 4);
+    L->group = take(nd, 4);
+    L->n_reuse = take(nb, 4);
+    L->query_start = take(nb, 4);
+    L->n_tiles = take(nb, 4);
+    L->doc_tile_begin = take(nd, 4);
+    L->doc_tile_count = take(nd, 4);
+    L->tile_doc = take(max_tiles, 4);
+    L->tile_row0 = take(max_tiles, 4);
+    L->tile_len = take(max_tiles, 4);
+    L->trig = take(nd * (size_t)(g->head_dim / 2), 8);
+    L->total_bytes = off;
+    L->max_tiles = (int32_t)max_tiles;
+    L->reserved = 0;
+}
+
+PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan) {
+    cf_plan_layout L;
+    plan_layout(g, b, &L);
+    char* base = static_cast<char*>(plan);
+    PlanView v;
+    v.status = reinterpret_cast<int*>(base + L.status);
+    v.kept = reinterpret_cast<int*>(base + L.kept);
+    v.kept_count = reinterpret_cast<int*>(base + L.kept_count);
+    v.dst_start = reinterpret_cast<int*>(base + L.dst_start);
+    v.group = reinterpret_cast<int*>(base + L.group);
+    v.n_reuse = reinterpret_cast<int*>(base + L.n_reuse);
+    v.query_start = reinterpret_cast<int*>(base + L.query_start);
+    v.n_tiles = reinterpret_cast<int*>(base + L.n_tiles);
+    v.doc_tile_begin = reinterpret_cast<int*>(base + L.doc_tile_begin);
+    v.doc_tile_count = reinterpret_cast<int*>(base + L.doc_tile_count);
+    v.tile_doc = reinterpret_cast<int*>(base + L.tile_doc);
+    v.tile_row0 = reinterpret_cast<int*>(base + L.tile_row0);
+    v.tile_len = reinterpret_cast<int*>(base + L.tile_len);
+    v.trig = reinterpret_cast<float2*>(base + L.trig);
+    v.max_tiles = L.max_tiles;
+    return v;
+}
+
+int sm_count() {
+    static std::atomic<int> cached{0};
+    int n = cached.load();
+    if (n > 0) return n;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        return 148;
+    cached.store(n);
+    return n;
+}
+
+int tiles_per_request_bound(const cf_batch* b) {
+    if (b->tiles_hint > 0) return b->tiles_hint;
+    long long t = (long long)b->n_docs_total + b->total_tokens / kTile + 1;
+    return (int)std::min<long long>(t, 1 << 20);
+}
+
+// Splits of the key-tile list per (request, kv head, row group): enough CTAs for every SM,
+// never more splits than tiles.
+int choose_splits(const cf_geom* g, const cf_batch* b) {
+    const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
+    const int row_groups = (rows + 255) / 256;
+    const long long units = (long long)b->n_requests * g->n_kv_heads * row_groups;
+    long long s = (sm_count() + units - 1) / units;
+    s = std::min<long long>(s, tiles_per_request_bound(b));
+    s = std::min<long long>(s, CF_MAX_SPLITS);
+    return (int)std::max<long long>(s, 1);
+}
+
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,
+                             void* base_ptr) {
+    const size_t rows = (size_t)g->n_q_heads * b->q_len;
+    const size_t nb = (size_t)b->n_requests;
+    const size_t max_tiles = (size_t)b->n_docs_total + (size_t)(b->total_tokens / kTile) + 1;
+    char* base = static_cast<char*>(base_ptr);
+    size_t off = 0;
+    auto take = [&](size_t count) {
+        size_t at = off;
+        off = align_up(off + count * 4, 256);
+        return at;
+    };
+    size_t o = take(nb * n_splits * rows * g->head_dim);
+    size_t m = take(nb * n_splits * rows);
+    size_t l = take(nb * n_splits * rows);
+    size_t t = take(max_tiles * rows);
+    size_t r = take(nb * rows);
+    if (ws) {
+        ws->part_o = reinterpret_cast<float*>(base + o);
+        ws->part_m = reinterpret_cast<float*>(base + m);
+        ws->part_l = reinterpret_cast<float*>(base + l);
+        ws->tile_lse2 = reinterpret_cast<float*>(base + t);
+        ws->row_lse2 = reinterpret_cast<float*>(base + r);
+        ws->n_splits = n_splits;
+    }
+    return off;
+}
+
+static std::atomic<int> g_attn_path{0};
+
+}  // namespace cf
+
+using namespace cf;
+
+extern "C" {
+
+const char* cf_error_string(int code) {
+    switch (code) {
+        case CF_OK: return "ok";
+        case CF_ERR_INVALID_ARG: return "invalid argument";
+        case CF_ERR_RANGE: return "kept documents do not fit the positional range";
+        case CF_ERR_UNSUPPORTED: return "unsupported geometry";
+        case CF_ERR_WORKSPACE: return "plan or workspace buffer too small or misaligned";
+        case CF_ERR_CUDA: return "CUDA call failed";
+        case CF_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+int cf_allocate_positions(const cf_geom* geom, int32_t n_docs, const int32_t* doc_len,
+                          const int32_t* order, int32_t n_kept, int32_t prefix_len,
+                          int32_t tail_reserve, int32_t n_reuse, int32_t query_start,
+                          int32_t* dst_start, int32_t* group, int32_t* n_reuse_out,
+                          int32_t* query_start_out) {
+    if (!geom || n_docs < 0 || n_kept < 0 || n_kept > n_docs || prefix_len < 0 || tail_reserve < 0 ||
+        n_reuse < 0 || !dst_start || !group || (n_docs > 0 && !doc_len) || (n_kept > 0 && !order))
+        return CF_ERR_INVALID_ARG;
+    const int64_t range = geom->pos_range;
+    const int64_t capacity = range - prefix_len - tail_reserve;
+    for (int i = 0; i < n_docs; ++i) dst_start[i] = group[i] = -1;
+    const int64_t qs = query_start < 0 ? range - tail_reserve : query_start;
+    if (n_kept == 0) {
+        if (n_reuse_out) *n_reuse_out = std::max(1, n_reuse);
+        if (query_start_out) *query_start_out = (int32_t)qs;
+        return CF_OK;
+    }
+    std::vector<char> seen(n_docs, 0);
+    int64_t longest = 0;
+    for (int r = 0; r < n_kept; ++r) {
+        const int i = order[r];
+        if (i < 0 || i >= n_docs || seen[i] || doc_len[i] <= 0) return CF_ERR_INVALID_ARG;
+        seen[i] = 1;
+        longest = std::max<int64_t>(longest, doc_len[i]);
+    }
+    int64_t windows = n_reuse;
+    if (windows <= 0) {
+        const int64_t per_window = capacity > 0 ? capacity / longest : 0;   // L / l_C of Eq. 6
+        if (per_window <= 0) return CF_ERR_RANGE;
+        windows = (n_kept + per_window - 1) / per_window;
+    }
+    std::vector<int64_t> cursor((size_t)windows, qs);
+    for (int r = 0; r < n_kept; ++r) cursor[r % windows] -= doc_len[order[r]];
+    if (qs + tail_reserve > range || *std::min_element(cursor.begin(), cursor.end()) < prefix_len)
+        return CF_ERR_RANGE;
+    std::fill(cursor.begin(), cursor.end(), qs);
+    for (int r = 0; r < n_kept; ++r) {
+        const int i = order[r];
+        const int64_t w = r % windows;
+        cursor[w] -= doc_len[i];
+        dst_start[i] = (int32_t)cursor[w];
+        group[i] = (int32_t)w;
+    }
+    if (n_reuse_out) *n_reuse_out = (int32_t)windows;
+    if (query_start_out) *query_start_out = (int32_t)qs;
+    return CF_OK;
+}
+
+int cf_schedule_linear(int32_t n_layers, int32_t every, int32_t k, int32_t k_finish,
+                       int32_t capacity, int32_t* layers, int32_t* keeps, int32_t* count) {
+    if (n_layers <= 0 || every <= 0 || k < 0 || k_finish < 0 || k_finish > k || capacity < 0 || !count)
+        return CF_ERR_INVALID_ARG;
+    const int prunes = n_layers / every;
+    *count = prunes;
+    if (prunes == 0) return CF_OK;
+    if (capacity < prunes || !layers || !keeps) return CF_ERR_INVALID_ARG;
+    const int step = (k - k_finish) / prunes;
+    int kept = k;
+    for (int j = 1; j <= prunes; ++j) {
+        kept = (j == prunes) ? k_finish : kept - step;
+        layers[j - 1] = j * every;
+        keeps[j - 1] = kept;
+    }
+    return CF_OK;
+}
+
+int cf_plan_layout_of(const cf_geom* geom, const cf_batch* batch, cf_plan_layout* layout) {
+    if (!batch || !layout) return CF_ERR_INVALID_ARG;
+    int rc = validate(geom, batch);
+    if (rc != CF_OK) return rc;
+    plan_layout(geom, batch, layout);
+    return CF_OK;
+}
+
+static int check_plan(const cf_geom* geom, const cf_batch* batch, const void* plan) {
+    if (!batch || !plan) return CF_ERR_INVALID_ARG;
+    int rc = validate(geom, batch);
+    if (rc != CF_OK) return rc;
+    if (reinterpret_cast<uintptr_t>(plan) % 256 != 0) return CF_ERR_WORKSPACE;
+    return CF_OK;
+}
+
+int cf_plan_init(const cf_geom* geom, const cf_batch* batch, const int32_t* order,
+                 const int32_t* kept_count, int32_t query_start, void* plan, size_t plan_bytes,
+                 void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    cf_plan_layout L;
+    plan_layout(geom, batch, &L);
+    if (plan_bytes < L.total_bytes) return CF_ERR_WORKSPACE;
+    if (query_start >= 0 && (int64_t)query_start + batch->tail_reserve > geom->pos_range)
+        return CF_ERR_RANGE;
+    PlanView pv = make_plan_view(geom, batch, plan);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(pv.status, 0, 16, s) != cudaSuccess) return CF_ERR_CUDA;
+    return launch_plan(make_geom_view(geom), make_batch_view(batch), pv, 0, order, kept_count,
+                       query_start, nullptr, 0, nullptr, CF_ALLOC_ALIGN, s);
+}
+
+int cf_plan_status(const cf_geom* geom, const cf_batch* batch, const void* plan, void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    int word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, pv.status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return CF_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return CF_ERR_CUDA;
+    return word;
+}
+
+int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                       int32_t n_layers, int64_t layer_stride, const void* k_in, void* k_out,
+                       void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (!k_in || !k_out || n_layers <= 0) return CF_ERR_INVALID_ARG;
+    const int esize = geom->dtype == CF_BF16 ? 2 : 4;
+    if (reinterpret_cast<uintptr_t>(k_in) % 16 || reinterpret_cast<uintptr_t>(k_out) % 16 ||
+        (layer_stride * esize) % 16)
+        return CF_ERR_INVALID_ARG;
+    if (n_layers > 1 && layer_stride < batch->total_tokens * batch->token_stride)
+        return CF_ERR_INVALID_ARG;
+    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    return launch_reposition(geom, batch, pv, n_layers, layer_stride, k_in, k_out,
+                             static_cast<cudaStream_t>(stream));
+}
+
+size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch) {
+    if (!batch || validate(geom, batch) != CF_OK) return 0;
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch), nullptr, nullptr);
+}
+
+int cf_set_attn_path(int32_t path) {
+    if (path != 0 && path != 1) return CF_ERR_INVALID_ARG;
+    g_attn_path.store(path);
+    return CF_OK;
+}
+
+int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                          const void* q, const void* k_cache, const void* v_cache,
+                          float softmax_scale, void* out, float* lse, float* doc_scores,
+                          float* score_accum, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (!q || !k_cache || !v_cache || !out || !workspace) return CF_ERR_INVALID_ARG;
+    if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return CF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return CF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(q) % 16 || reinterpret_cast<uintptr_t>(out) % 16 ||
+        reinterpret_cast<uintptr_t>(k_cache) % 16 || reinterpret_cast<uintptr_t>(v_cache) % 16)
+        return CF_ERR_INVALID_ARG;
+    const int n_splits = choose_splits(geom, batch);
+    AttnWorkspace ws;
+    const size_t need = attn_workspace_layout(geom, batch, n_splits, &ws, workspace);
+    if (workspace_bytes < need) return CF_ERR_WORKSPACE;
+    const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
+    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch))
+        rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
+    else
+        rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
+    if (rc != CF_OK) return rc;
+    return launch_combine(geom, batch, pv, ws, out, lse, doc_scores, score_accum, s);
+}
+
+int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
+                  const float* score_accum, int32_t keep, const int32_t* keep_per_request,
+                  int32_t strategy, void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (!score_accum || (keep < 0 && !keep_per_request)) return CF_ERR_INVALID_ARG;
+    if (strategy != CF_ALLOC_NONE && strategy != CF_ALLOC_ALIGN && strategy != CF_ALLOC_SORT)
+        return CF_ERR_INVALID_ARG;
+    PlanView pv = make_plan_view(geom, batch, plan);
+    return launch_plan(make_geom_view(geom), make_batch_view(batch), pv, 1, nullptr, nullptr, -1,
+                       score_accum, keep, keep_per_request, strategy,
+                       static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,293 @@
+// Portable CUDA-core version of the fused re-position + query-prefill attention (Eq. 5 fused
+// into Eq. 1), and the kernels that merge split partials and reduce document scores.  This
+// kernel serves the geometries the tensor-core kernel does not cover (fp32 storage, head_dim
+// 64) and is the second implementation the tensor-core kernel is checked against.
+#include <algorithm>
+
+#include "cf_common.cuh"
+
+namespace cf {
+
+constexpr int kSimtThreads = 256;
+constexpr int kSimtRows = 64;     // query rows per CTA
+constexpr int kSimtSub = 32;      // key rows per inner step
+
+template <int D>
+constexpr size_t simt_smem_bytes() {
+    return sizeof(float) * (size_t)(kSimtRows * (D + 1) + kSimtSub * (D + 1) + kSimtSub * D +
+                                    kSimtRows * (kSimtSub + 1));
+}
+
+template <typename T, int D, int LAYOUT>
+__global__ void __launch_bounds__(kSimtThreads)
+attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads,
+                 float scale_log2, const T* __restrict__ q, const T* __restrict__ k_cache,
+                 const T* __restrict__ v_cache) {
+    extern __shared__ float smem[];
+    float (*Qs)[D + 1] = reinterpret_cast<float (*)[D + 1]>(smem);
+    float (*Ks)[D + 1] = reinterpret_cast<float (*)[D + 1]>(smem + kSimtRows * (D + 1));
+    float (*Vs)[D] = reinterpret_cast<float (*)[D]>(smem + (kSimtRows + kSimtSub) * (D + 1));
+    float (*Ps)[kSimtSub + 1] =
+        reinterpret_cast<float (*)[kSimtSub + 1]>(smem + (kSimtRows + kSimtSub) * (D + 1) + kSimtSub * D);
+
+    const int tid = threadIdx.x;
+    const int group = n_q_heads / n_kv_heads;
+    const int lq = bv.q_len;
+    const int rows = group * lq;                                   // query rows sharing one kv head
+    const int row_chunks = (rows + kSimtRows - 1) / kSimtRows;
+    const int b = blockIdx.z;
+    const int kvh = blockIdx.y / row_chunks;
+    const int r0 = (blockIdx.y - kvh * row_chunks) * kSimtRows;
+    const int n_rows = min(kSimtRows, rows - r0);
+    const int split = blockIdx.x;
+    const int rows_total = n_q_heads * lq;
+
+    for (int idx = tid; idx < kSimtRows * D; idx += kSimtThreads) {
+        const int rr = idx / D, d = idx - rr * D;
+        float val = 0.f;
+        if (rr < n_rows) {
+            const int row = r0 + rr;
+            const int g = row / lq, j = row - g * lq;
+            const int h = kvh * group + g;
+            val = to_float(q[(((size_t)b * lq + j) * n_q_heads + h) * D + d]);
+        }
+        Qs[rr][d] = val;
+    }
+
+    const int doc0 = bv.req_doc_begin[b];
+    const int base = tile_base(doc0, bv.doc_offsets[doc0]);
+    const int n_tiles = pv.n_tiles[b];
+    const int t_begin = (int)((long long)n_tiles * split / ws.n_splits);
+    const int t_end = (int)((long long)n_tiles * (split + 1) / ws.n_splits);
+
+    const int r = tid >> 2, q4 = tid & 3;
+    float m = -INFINITY, l = 0.f;
+    float acc[D / 4];
+#pragma unroll
+    for (int k = 0; k < D / 4; ++k) acc[k] = 0.f;
+    const size_t row_global = (size_t)kvh * rows + r0 + r;
+
+    for (int ti = t_begin; ti < t_end; ++ti) {
+        const int doc = pv.tile_doc[base + ti];
+        const long long row0 = pv.tile_row0[base + ti];
+        const int len = pv.tile_len[base + ti];
+        const float2* trig = pv.trig + (size_t)doc * (D / 2);
+        float l_tile = 0.f;
+        for (int sub = 0; sub < len; sub += kSimtSub) {
+            const int n = min(kSimtSub, len - sub);
+            __syncthreads();
+            // keys: rotate each slice by the document's delta (Eq. 5), round to the storage type
+            for (int idx = tid; idx < kSimtSub * (D / 2); idx += kSimtThreads) {
+                const int t = idx / (D / 2), p = idx - t * (D / 2);
+                const int ia = LAYOUT == CF_ROPE_HALF ? p : 2 * p;
+                const int ib = LAYOUT == CF_ROPE_HALF ? p + D / 2 : 2 * p + 1;
+                float ya = 0.f, yb = 0.f;
+                if (t < n) {
+                    const T* src = k_cache + (row0 + sub + t) * bv.token_stride + (size_t)kvh * D;
+                    const float2 cs = trig[p];
+                    rotate_pair(to_float(src[ia]), to_float(src[ib]), cs.x, cs.y, ya, yb);
+                    ya = to_float(from_float<T>(ya));
+                    yb = to_float(from_float<T>(yb));
+                }
+                Ks[t][ia] = ya;
+                Ks[t][ib] = yb;
+            }
+            for (int idx = tid; idx < kSimtSub * D; idx += kSimtThreads) {
+                const int t = idx / D, d = idx - t * D;
+                Vs[t][d] = t < n ? to_float(v_cache[(row0 + sub + t) * bv.token_stride + (size_t)kvh * D + d]) : 0.f;
+            }
+            __syncthreads();
+            float sc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sc[i] = 0.f;
+            for (int d = 0; d < D; ++d) {
+                const float qv = Qs[r][d];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sc[i] = fmaf(qv, Ks[q4 * 8 + i][d], sc[i]);
+            }
+            float sub_max = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                sc[i] = (q4 * 8 + i < n) ? sc[i] * scale_log2 : -INFINITY;
+                sub_max = fmaxf(sub_max, sc[i]);
+            }
+            sub_max = fmaxf(sub_max, __shfl_xor_sync(0xffffffffu, sub_max, 1));
+            sub_max = fmaxf(sub_max, __shfl_xor_sync(0xffffffffu, sub_max, 2));
+            const float m_new = fmaxf(m, sub_max);
+            const float alpha = exp2f(m - m_new);
+            float sub_sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float pr = exp2f(sc[i] - m_new);
+                Ps[r][q4 * 8 + i] = pr;
+                sub_sum += pr;
+            }
+            sub_sum += __shfl_xor_sync(0xffffffffu, sub_sum, 1);
+            sub_sum += __shfl_xor_sync(0xffffffffu, sub_sum, 2);
+            l = fmaf(l, alpha, sub_sum);
+            l_tile = fmaf(l_tile, alpha, sub_sum);
+            m = m_new;
+#pragma unroll
+            for (int k = 0; k < D / 4; ++k) acc[k] *= alpha;
+            __syncwarp();
+            for (int t = 0; t < kSimtSub; ++t) {
+                const float pr = Ps[r][t];
+#pragma unroll
+                for (int k = 0; k < D / 4; ++k) acc[k] = fmaf(pr, Vs[t][4 * k + q4], acc[k]);
+            }
+        }
+        if (q4 == 0 && r < n_rows)
+            ws.tile_lse2[(size_t)(base + ti) * rows_total + row_global] = m + log2f(l_tile);
+    }
+    if (r < n_rows) {
+        const size_t slot = ((size_t)b * ws.n_splits + split) * rows_total + row_global;
+        if (q4 == 0) {
+            ws.part_m[slot] = m;
+            ws.part_l[slot] = l;
+        }
+#pragma unroll
+        for (int k = 0; k < D / 4; ++k) ws.part_o[slot * D + 4 * k + q4] = acc[k];
+    }
+}
+
+// Merge the splits of one query row (one warp per row): out = sum_s w_s O_s / sum_s w_s l_s with
+// w_s = 2^(m_s - max m), and the row's log-sum-exp.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+combine_kernel(AttnWorkspace ws, int n_requests, int n_q_heads, int lq, T* __restrict__ out,
+               float* __restrict__ lse) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int rows_total = n_q_heads * lq;
+    if (warp >= n_requests * rows_total) return;
+    const int b = warp / rows_total, rg = warp - b * rows_total;
+    const int h = rg / lq, j = rg - h * lq;
+    float m_max = -INFINITY;
+    for (int s = 0; s < ws.n_splits; ++s)
+        m_max = fmaxf(m_max, ws.part_m[((size_t)b * ws.n_splits + s) * rows_total + rg]);
+    float acc[D / 32];
+#pragma unroll
+    for (int k = 0; k < D / 32; ++k) acc[k] = 0.f;
+    float l_sum = 0.f;
+    if (m_max > -INFINITY) {
+        for (int s = 0; s < ws.n_splits; ++s) {
+            const size_t slot = ((size_t)b * ws.n_splits + s) * rows_total + rg;
+            const float ms = ws.part_m[slot];
+            if (ms == -INFINITY) continue;
+            const float w = exp2f(ms - m_max);
+            l_sum = fmaf(ws.part_l[slot], w, l_sum);
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(ws.part_o[slot * D + lane + 32 * k], w, acc[k]);
+        }
+    }
+    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+    T* dst = out + (((size_t)b * lq + j) * n_q_heads + h) * D;
+#pragma unroll
+    for (int k = 0; k < D / 32; ++k) dst[lane + 32 * k] = from_float<T>(acc[k] * inv);
+    if (lane == 0) {
+        const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
+        ws.row_lse2[(size_t)b * rows_total + rg] = lse2;
+        if (lse) lse[(size_t)b * rows_total + rg] = lse2 * kLn2;
+    }
+}
+
+// Document scores (footnote of Sec. 2.4; Algorithm 2: S <- S + s^l): one block per document sums
+// 2^(tile_lse - row_lse) over the document's tiles and all query rows, in a fixed order.
+__global__ void __launch_bounds__(256)
+score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float* __restrict__ doc_scores,
+             float* __restrict__ score_accum) {
+    __shared__ float s_red[256];
+    const int doc = blockIdx.x;
+    const int count = pv.doc_tile_count[doc];
+    if (count == 0) {
+        if (threadIdx.x == 0 && doc_scores) doc_scores[doc] = 0.f;
+        return;
+    }
+    int lo = 0, hi = bv.n_requests;                 // request that owns the document
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (bv.req_doc_begin[mid] <= doc) lo = mid; else hi = mid;
+    }
+    const float* row_lse2 = ws.row_lse2 + (size_t)lo * rows_total;
+    const float* tile_lse2 = ws.tile_lse2 + (size_t)pv.doc_tile_begin[doc] * rows_total;
+    float sum = 0.f;
+    for (int idx = threadIdx.x; idx < count * rows_total; idx += 256) {
+        const int rg = idx % rows_total;
+        sum += exp2f(tile_lse2[idx] - row_lse2[rg]);
+    }
+    s_red[threadIdx.x] = sum;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) s_red[threadIdx.x] += s_red[threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const float score = s_red[0] / (float)rows_total;
+        if (doc_scores) doc_scores[doc] = score;
+        if (score_accum) score_accum[doc] += score;
+    }
+}
+
+template <typename T, int D>
+static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
+                             const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
+                             cudaStream_t stream) {
+    const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
+    const int row_chunks = (rows + kSimtRows - 1) / kSimtRows;
+    if ((long long)g->n_kv_heads * row_chunks > 65535 || b->n_requests > 65535) return CF_ERR_INVALID_ARG;
+    dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_chunks), (unsigned)b->n_requests);
+    BatchView bv = make_batch_view(b);
+    const size_t smem = simt_smem_bytes<D>();
+    auto run = [&](auto kernel) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return CF_ERR_CUDA;
+        kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, g->n_q_heads, g->n_kv_heads, scale_log2,
+                                                     static_cast<const T*>(q), static_cast<const T*>(k),
+                                                     static_cast<const T*>(v));
+        return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+    };
+    if (g->rope_layout == CF_ROPE_HALF) return run(attn_simt_kernel<T, D, CF_ROPE_HALF>);
+    return run(attn_simt_kernel<T, D, CF_ROPE_INTERLEAVED>);
+}
+
+int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
+                     const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
+                     cudaStream_t stream) {
+    if (g->dtype == CF_BF16) {
+        if (g->head_dim == 128) return launch_simt_typed<__nv_bfloat16, 128>(g, b, pv, q, k, v, scale_log2, ws, stream);
+        return launch_simt_typed<__nv_bfloat16, 64>(g, b, pv, q, k, v, scale_log2, ws, stream);
+    }
+    if (g->head_dim == 128) return launch_simt_typed<float, 128>(g, b, pv, q, k, v, scale_log2, ws, stream);
+    return launch_simt_typed<float, 64>(g, b, pv, q, k, v, scale_log2, ws, stream);
+}
+
+template <typename T, int D>
+static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const AttnWorkspace& ws, void* out,
+                                float* lse, cudaStream_t stream) {
+    const long long warps = (long long)b->n_requests * g->n_q_heads * b->q_len;
+    const long long blocks = (warps + 7) / 8;
+    combine_kernel<T, D><<<(unsigned)blocks, 256, 0, stream>>>(ws, b->n_requests, g->n_q_heads, b->q_len,
+                                                            static_cast<T*>(out), lse);
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
+
+int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
+                   void* out, float* lse, float* doc_scores, float* score_accum, cudaStream_t stream) {
+    int rc;
+    if (g->dtype == CF_BF16)
+        rc = g->head_dim == 128 ? launch_combine_typed<__nv_bfloat16, 128>(g, b, ws, out, lse, stream)
+                                : launch_combine_typed<__nv_bfloat16, 64>(g, b, ws, out, lse, stream);
+    else
+        rc = g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, ws, out, lse, stream)
+                                : launch_combine_typed<float, 64>(g, b, ws, out, lse, stream);
+    if (rc != CF_OK) return rc;
+    if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
+        score_kernel<<<(unsigned)b->n_docs_total, 256, 0, stream>>>(make_batch_view(b), pv, ws,
+                                                                   g->n_q_heads * b->q_len, doc_scores,
+                                                                   score_accum);
+        if (cudaGetLastError() != cudaSuccess) return CF_ERR_CUDA;
+    }
+    return CF_OK;
+}
+
+}  // namespace cf

@@ -1,0 +1,108 @@
+// Shared declarations of the CUDA side: views of the caller's buffers, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cachefocus.h"
+
+namespace cf {
+
+constexpr int kTile = CF_TILE_TOKENS;
+constexpr int kMaxDocs = CF_MAX_DOCS_PER_REQUEST;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct GeomView {
+    int n_q_heads, n_kv_heads, head_dim, dtype, rope_layout, pos_range;
+    double rope_theta;
+};
+
+struct BatchView {
+    int n_requests, n_docs_total, q_len, prefix_len, tail_reserve, n_reuse;
+    long long total_tokens, token_stride;
+    const int* req_doc_begin;
+    const int* doc_offsets;
+    const int* doc_src_start;
+};
+
+// Typed pointers into a plan buffer (see cf_plan_layout).
+struct PlanView {
+    int* status;
+    int* kept;
+    int* kept_count;
+    int* dst_start;
+    int* group;
+    int* n_reuse;
+    int* query_start;
+    int* n_tiles;
+    int* doc_tile_begin;
+    int* doc_tile_count;
+    int* tile_doc;
+    int* tile_row0;
+    int* tile_len;
+    float2* trig;
+    int max_tiles;
+};
+
+// First tile slot of request b: an upper bound of the tiles all earlier requests can own
+// (a document of len tokens owns ceil(len/kTile) <= 1 + len/kTile tiles).
+__host__ __device__ inline int tile_base(int doc_begin, int row_begin) {
+    return doc_begin + row_begin / kTile;
+}
+
+GeomView make_geom_view(const cf_geom* g);
+BatchView make_batch_view(const cf_batch* b);
+PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan);
+int validate(const cf_geom* g, const cf_batch* b);
+int sm_count();
+int choose_splits(const cf_geom* g, const cf_batch* b);
+int tiles_per_request_bound(const cf_batch* b);
+
+// Partial results of the attention kernels, one slice per split, merged by the combine kernel.
+// All logits are in base-2 units: t = (q.k) * softmax_scale * log2(e).
+struct AttnWorkspace {
+    float* part_o;     // [B][n_splits][Hq*Lq][D]   sum_t 2^(t - m) v_t, not normalised
+    float* part_m;     // [B][n_splits][Hq*Lq]      running maximum m (-inf if the split is empty)
+    float* part_l;     // [B][n_splits][Hq*Lq]      sum_t 2^(t - m)
+    float* tile_lse2;  // [max_tiles][Hq*Lq]        log2 of sum over the tile's tokens of 2^t
+    float* row_lse2;   // [B][Hq*Lq]                log2 of the full softmax denominator
+    int n_splits;
+};
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,
+                             void* base);
+
+// ---- launchers (each returns a CF_* code) -------------------------------------------------
+int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
+                const int* order, const int* kept_count, int query_start, const float* score_accum,
+                int keep, const int* keep_per_request, int strategy, cudaStream_t stream);
+int launch_reposition(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers,
+                      long long layer_stride, const void* k_in, void* k_out, cudaStream_t stream);
+int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
+                     const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
+                     cudaStream_t stream);
+int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
+                   const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
+                   cudaStream_t stream);
+bool attn_tc_supported(const cf_geom* g, const cf_batch* b);
+int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
+                   void* out, float* lse, float* doc_scores, float* score_accum,
+                   cudaStream_t stream);
+
+// ---- device helpers -----------------------------------------------------------------------
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_float(float x);
+template <> __device__ __forceinline__ float from_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) {
+    return __float2bfloat16_rn(x);
+}
+
+// Eq. 2 on one slice (a, b) with (c, s) = cos, sin of the delta angle; fp32, fused multiply-adds.
+__device__ __forceinline__ void rotate_pair(float a, float b, float c, float s, float& ya, float& yb) {
+    ya = fmaf(a, c, -(b * s));
+    yb = fmaf(a, s, b * c);
+}
+
+}  // namespace cf

@@ -1,0 +1,216 @@
+// Device-side bookkeeping of a request batch: the kept list and its order (Algorithm 2:
+// Init, argsort of S, prun), the positional allocation of the kept documents (Sec. 2.3.1 Eq. 6,
+// Sec. 2.5), and what the hot kernels consume: per-document rotation tables (Eq. 2 angles of
+// the delta of Eq. 5) and the list of key tiles.  One thread block per request; everything
+// runs in stream order so a layer stack needs no host round trip between layers.
+#include "cf_common.cuh"
+
+namespace cf {
+
+constexpr int kPlanThreads = 256;
+
+__device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+// mode 0: initialise from (order, kept_count); mode 1: prune by score, then rebuild.
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restrict__ order,
+            const int* __restrict__ kept_count_in, int query_start_arg,
+            const float* __restrict__ score_accum, int keep, const int* __restrict__ keep_per_request,
+            int strategy) {
+    __shared__ int s_ids[kMaxDocs];       // kept local ids by rank
+    __shared__ int s_tmp[kMaxDocs];       // new order / per-rank tile counts / window cursors
+    __shared__ float s_score[kMaxDocs];
+    __shared__ unsigned char s_flag[kMaxDocs];
+    __shared__ double s_inv_freq[64];
+    __shared__ int s_longest, s_min_cursor;
+
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int doc0 = bv.req_doc_begin[b];
+    const int n_docs = bv.req_doc_begin[b + 1] - doc0;
+    if (n_docs > kMaxDocs || n_docs < 0) {
+        if (tid == 0) {
+            raise_status(pv.status, CF_ERR_INVALID_ARG);
+            pv.kept_count[b] = 0;
+            pv.n_tiles[b] = 0;
+        }
+        return;
+    }
+    const int half = gv.head_dim / 2;
+    for (int p = tid; p < half; p += kPlanThreads)
+        s_inv_freq[p] = pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
+    if (tid == 0) {
+        s_longest = 0;
+        s_min_cursor = 0x7fffffff;
+    }
+
+    // ---- the kept list, in rank order -------------------------------------------------------
+    int n_kept;
+    if (mode == 0) {
+        n_kept = kept_count_in ? kept_count_in[b] : n_docs;
+        n_kept = max(0, min(n_kept, n_docs));
+        for (int r = tid; r < n_kept; r += kPlanThreads) {
+            int id = order ? order[doc0 + r] : r;
+            if (id < 0 || id >= n_docs) {
+                raise_status(pv.status, CF_ERR_INVALID_ARG);
+                id = 0;
+            }
+            s_ids[r] = id;
+        }
+        __syncthreads();
+    } else {
+        const int n_old = max(0, min(pv.kept_count[b], n_docs));
+        int keep_b = keep_per_request ? keep_per_request[b] : keep;
+        keep_b = max(0, min(keep_b, n_old));
+        for (int r = tid; r < n_old; r += kPlanThreads) {
+            s_ids[r] = pv.kept[doc0 + r];
+            s_score[r] = score_accum[doc0 + s_ids[r]];
+        }
+        __syncthreads();
+        // rank by counting: how many kept documents beat this one (ties: lower id wins)
+        for (int r = tid; r < n_old; r += kPlanThreads) {
+            const float s = s_score[r];
+            const int id = s_ids[r];
+            int better = 0;
+            for (int o = 0; o < n_old; ++o) {
+                const float so = s_score[o];
+                better += (so > s) || (so == s && s_ids[o] < id);
+            }
+            s_flag[r] = better < keep_b;
+            if (strategy == CF_ALLOC_SORT && better < keep_b) s_tmp[better] = id;
+        }
+        __syncthreads();
+        if (strategy != CF_ALLOC_SORT) {
+            for (int r = tid; r < n_old; r += kPlanThreads) {
+                if (!s_flag[r]) continue;
+                int before = 0;
+                for (int o = 0; o < r; ++o) before += s_flag[o];
+                s_tmp[before] = s_ids[r];
+            }
+        }
+        __syncthreads();
+        n_kept = keep_b;
+        // (the clamp only matters for malformed input -- duplicate ids, NaN scores -- where two
+        //  documents can claim one slot and leave another unwritten)
+        for (int r = tid; r < n_kept; r += kPlanThreads) s_ids[r] = max(0, min(s_tmp[r], n_docs - 1));
+        __syncthreads();
+    }
+
+    // ---- documents that are not kept ----------------------------------------------------------
+    const bool reallocate = (mode == 0) || (strategy != CF_ALLOC_NONE);
+    for (int i = tid; i < n_docs; i += kPlanThreads) s_flag[i] = 0;
+    __syncthreads();
+    for (int r = tid; r < n_kept; r += kPlanThreads) s_flag[s_ids[r]] = 1;
+    __syncthreads();
+    for (int i = tid; i < n_docs; i += kPlanThreads) {
+        pv.doc_tile_count[doc0 + i] = 0;
+        pv.doc_tile_begin[doc0 + i] = 0;
+        if (!s_flag[i]) {
+            pv.dst_start[doc0 + i] = -1;
+            pv.group[doc0 + i] = -1;
+        }
+    }
+
+    // ---- positional allocation ----------------------------------------------------------------
+    int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
+                                : pv.query_start[b];
+    int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
+    if (reallocate && n_kept > 0) {
+        int longest = 0;
+        for (int r = tid; r < n_kept; r += kPlanThreads) {
+            const int i = doc0 + s_ids[r];
+            longest = max(longest, bv.doc_offsets[i + 1] - bv.doc_offsets[i]);
+        }
+        atomicMax(&s_longest, longest);
+        __syncthreads();
+        longest = s_longest;
+        const int capacity = gv.pos_range - bv.prefix_len - bv.tail_reserve;
+        windows = bv.n_reuse;
+        if (windows <= 0) {
+            const int per_window = longest > 0 ? capacity / longest : 0;     // L / l_C of Eq. 6
+            if (per_window <= 0) {
+                if (tid == 0) raise_status(pv.status, CF_ERR_RANGE);
+                windows = n_kept;
+            } else {
+                windows = (n_kept + per_window - 1) / per_window;
+            }
+        }
+        // one thread per window walks its ranks r = w, w + windows, ... backwards from the query
+        for (int w = tid; w < windows && w < n_kept; w += kPlanThreads) {
+            int cursor = query_start;
+            for (int r = w; r < n_kept; r += windows) {
+                const int i = doc0 + s_ids[r];
+                cursor -= bv.doc_offsets[i + 1] - bv.doc_offsets[i];
+                pv.dst_start[i] = cursor;
+                pv.group[i] = w;
+            }
+            atomicMin(&s_min_cursor, cursor);
+        }
+        __syncthreads();
+        if (tid == 0 && (s_min_cursor < bv.prefix_len || query_start + bv.tail_reserve > gv.pos_range))
+            raise_status(pv.status, CF_ERR_RANGE);
+    }
+
+    // ---- key tiles: document-aligned runs of at most kTile rows -------------------------------
+    for (int r = tid; r < n_kept; r += kPlanThreads) {
+        const int i = doc0 + s_ids[r];
+        s_tmp[r] = (bv.doc_offsets[i + 1] - bv.doc_offsets[i] + kTile - 1) / kTile;
+    }
+    __syncthreads();
+    const int base = tile_base(doc0, bv.doc_offsets[doc0]);
+    if (tid == 0) {
+        int run = 0;
+        for (int r = 0; r < n_kept; ++r) {
+            const int c = s_tmp[r];
+            s_tmp[r] = run;
+            run += c;
+        }
+        if (base + run > pv.max_tiles) {      // cannot happen with a plan sized by cf_plan_layout_of
+            raise_status(pv.status, CF_ERR_WORKSPACE);
+            s_longest = -1;
+        }
+        pv.n_tiles[b] = s_longest < 0 ? 0 : run;
+        pv.kept_count[b] = s_longest < 0 ? 0 : n_kept;
+        pv.n_reuse[b] = windows;
+        pv.query_start[b] = query_start;
+    }
+    __syncthreads();
+    if (s_longest < 0) return;
+    for (int r = tid; r < n_kept; r += kPlanThreads) {
+        const int i = doc0 + s_ids[r];
+        const int row0 = bv.doc_offsets[i];
+        const int len = bv.doc_offsets[i + 1] - row0;
+        const int first = base + s_tmp[r];
+        const int count = (len + kTile - 1) / kTile;
+        pv.kept[doc0 + r] = s_ids[r];
+        pv.doc_tile_begin[i] = first;
+        pv.doc_tile_count[i] = count;
+        for (int k = 0; k < count; ++k) {
+            pv.tile_doc[first + k] = i;
+            pv.tile_row0[first + k] = row0 + k * kTile;
+            pv.tile_len[first + k] = min(kTile, len - k * kTile);
+        }
+    }
+
+    // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D), angle in fp64 --------------
+    // (dst_start was written by other threads of this block: the barriers above order it)
+    for (int idx = tid; idx < n_kept * half; idx += kPlanThreads) {
+        const int r = idx / half, p = idx - r * half;
+        const int i = doc0 + s_ids[r];
+        const double delta = (double)(pv.dst_start[i] - bv.doc_src_start[i]);
+        double sn, cs;
+        sincos(delta * s_inv_freq[p], &sn, &cs);
+        pv.trig[(size_t)i * half + p] = make_float2((float)cs, (float)sn);
+    }
+}
+
+int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
+                const int* order, const int* kept_count, int query_start, const float* score_accum,
+                int keep, const int* keep_per_request, int strategy, cudaStream_t stream) {
+    plan_kernel<<<bv.n_requests, kPlanThreads, 0, stream>>>(gv, bv, pv, mode, order, kept_count,
+                                                           query_start, score_accum, keep,
+                                                           keep_per_request, strategy);
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
+
+}  // namespace cf
