@@ -1,0 +1,217 @@
+"""Thin ctypes binding of libcachefocus.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch tensors used purely as device (or host) buffers; every step of the path runs
+in the library's kernels."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+CF_OK, CF_ERR_INVALID_ARG, CF_ERR_RANGE, CF_ERR_UNSUPPORTED, CF_ERR_WORKSPACE, CF_ERR_CUDA, CF_ERR_TIMEOUT = range(7)
+CF_BF16, CF_F32 = 0, 1
+CF_ROPE_HALF, CF_ROPE_INTERLEAVED = 0, 1
+CF_ALLOC_NONE, CF_ALLOC_ALIGN, CF_ALLOC_SORT = 0, 1, 2
+CF_TILE_TOKENS = 128
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefocus.so")
+
+EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
+           "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
+           "cf_query_prefill_attn", "cf_prune_topk", "cf_set_attn_path"]
+
+
+class cf_geom(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("rope_layout", ctypes.c_int32), ("pos_range", ctypes.c_int32),
+                ("rope_theta", ctypes.c_double)]
+
+
+class cf_batch(ctypes.Structure):
+    _fields_ = [("n_requests", ctypes.c_int32), ("n_docs_total", ctypes.c_int32), ("q_len", ctypes.c_int32),
+                ("prefix_len", ctypes.c_int32), ("tail_reserve", ctypes.c_int32), ("n_reuse", ctypes.c_int32),
+                ("tiles_hint", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("total_tokens", ctypes.c_int64), ("token_stride", ctypes.c_int64),
+                ("req_doc_begin", ctypes.c_void_p), ("doc_offsets", ctypes.c_void_p),
+                ("doc_src_start", ctypes.c_void_p)]
+
+
+class cf_plan_layout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_size_t) for n in
+                ("total_bytes", "status", "kept", "kept_count", "dst_start", "group", "n_reuse", "query_start",
+                 "n_tiles", "doc_tile_begin", "doc_tile_count", "tile_doc", "tile_row0", "tile_len", "trig")] + \
+               [("max_tiles", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class CacheFocusError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {cf_error_string(code)} (code {code})")
+
+
+_LIB = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libcachefocus.so (built by paper_2502_11101_b200.build); no fallback exists."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_11101_b200.build` "
+                           "(the CUDA library is the only implementation, there is no CPU path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    gp, bp = ctypes.POINTER(cf_geom), ctypes.POINTER(cf_batch)
+    lib.cf_error_string.restype = ctypes.c_char_p
+    lib.cf_error_string.argtypes = [ctypes.c_int]
+    lib.cf_allocate_positions.argtypes = [gp, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.cf_schedule_linear.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp]
+    lib.cf_plan_layout_of.argtypes = [gp, bp, ctypes.POINTER(cf_plan_layout)]
+    lib.cf_plan_init.argtypes = [gp, bp, vp, vp, i32, vp, ctypes.c_size_t, vp]
+    lib.cf_plan_status.argtypes = [gp, bp, vp, vp]
+    lib.cf_reposition_keys.argtypes = [gp, bp, vp, i32, i64, vp, vp, vp]
+    lib.cf_attn_workspace_bytes.restype = ctypes.c_size_t
+    lib.cf_attn_workspace_bytes.argtypes = [gp, bp]
+    lib.cf_query_prefill_attn.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
+                                          ctypes.c_size_t, vp]
+    lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
+    lib.cf_set_attn_path.argtypes = [i32]
+    for name in EXPORTS:
+        if name not in ("cf_error_string", "cf_attn_workspace_bytes"):
+            getattr(lib, name).restype = ctypes.c_int
+    _LIB = lib
+    return lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != CF_OK:
+        raise CacheFocusError(code, where)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return int(t)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def make_geom(n_q_heads: int, n_kv_heads: int, head_dim: int, dtype, pos_range: int, rope_theta: float,
+              rope_layout: int = CF_ROPE_HALF) -> cf_geom:
+    if isinstance(dtype, torch.dtype):
+        dtype = {torch.bfloat16: CF_BF16, torch.float32: CF_F32}[dtype]
+    return cf_geom(n_q_heads, n_kv_heads, head_dim, dtype, rope_layout, pos_range, float(rope_theta))
+
+
+def make_batch(n_requests: int, q_len: int, total_tokens: int, token_stride: int,
+               req_doc_begin: torch.Tensor, doc_offsets: torch.Tensor, doc_src_start: torch.Tensor,
+               prefix_len: int = 0, tail_reserve: int = 0, n_reuse: int = 0, tiles_hint: int = 0) -> cf_batch:
+    """`req_doc_begin`, `doc_offsets`, `doc_src_start` are int32 device tensors the caller keeps alive."""
+    for t in (req_doc_begin, doc_offsets, doc_src_start):
+        assert t.dtype == torch.int32 and t.is_contiguous()
+    return cf_batch(n_requests, doc_src_start.numel(), q_len, prefix_len, tail_reserve, n_reuse, tiles_hint, 0,
+                    total_tokens, token_stride, req_doc_begin.data_ptr(), doc_offsets.data_ptr(),
+                    doc_src_start.data_ptr())
+
+
+def cf_error_string(code: int) -> str:
+    return load_library().cf_error_string(code).decode()
+
+
+def cf_allocate_positions(geom: cf_geom, doc_len: Sequence[int], order: Sequence[int], prefix_len: int = 0,
+                          tail_reserve: int = 0, n_reuse: int = 0, query_start: int = -1
+                          ) -> Tuple[np.ndarray, np.ndarray, int, int]:
+    """Host-side allocation for one request; returns (dst_start, group, n_reuse, query_start)."""
+    doc_len, order = _i32(doc_len), _i32(order)
+    dst, grp = np.empty(len(doc_len), np.int32), np.empty(len(doc_len), np.int32)
+    used, qs = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = load_library().cf_allocate_positions(ctypes.byref(geom), len(doc_len), doc_len.ctypes.data, order.ctypes.data,
+                                              len(order), prefix_len, tail_reserve, n_reuse, query_start,
+                                              dst.ctypes.data, grp.ctypes.data, ctypes.addressof(used),
+                                              ctypes.addressof(qs))
+    _check(rc, "cf_allocate_positions")
+    return dst, grp, used.value, qs.value
+
+
+def cf_schedule_linear(n_layers: int, every: int, k: int, k_finish: int) -> List[Tuple[int, int]]:
+    cap = max(1, n_layers)
+    layers, keeps = np.zeros(cap, np.int32), np.zeros(cap, np.int32)
+    count = ctypes.c_int32(0)
+    rc = load_library().cf_schedule_linear(n_layers, every, k, k_finish, cap, layers.ctypes.data, keeps.ctypes.data,
+                                           ctypes.addressof(count))
+    _check(rc, "cf_schedule_linear")
+    return [(int(layers[i]), int(keeps[i])) for i in range(count.value)]
+
+
+def cf_plan_layout_of(geom: cf_geom, batch: cf_batch) -> cf_plan_layout:
+    layout = cf_plan_layout()
+    _check(load_library().cf_plan_layout_of(ctypes.byref(geom), ctypes.byref(batch), ctypes.byref(layout)),
+           "cf_plan_layout_of")
+    return layout
+
+
+def cf_plan_init(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, order: Optional[torch.Tensor] = None,
+                 kept_count: Optional[torch.Tensor] = None, query_start: int = -1, stream=None) -> None:
+    rc = load_library().cf_plan_init(ctypes.byref(geom), ctypes.byref(batch), _ptr(order), _ptr(kept_count),
+                                     query_start, plan.data_ptr(), plan.numel() * plan.element_size(), _stream(stream))
+    _check(rc, "cf_plan_init")
+
+
+def cf_plan_status(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, stream=None) -> int:
+    return load_library().cf_plan_status(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), _stream(stream))
+
+
+def cf_reposition_keys(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, k_in: torch.Tensor, k_out: torch.Tensor,
+                       n_layers: int = 1, layer_stride: int = 0, stream=None) -> None:
+    rc = load_library().cf_reposition_keys(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), n_layers,
+                                           layer_stride, k_in.data_ptr(), k_out.data_ptr(), _stream(stream))
+    _check(rc, "cf_reposition_keys")
+
+
+def cf_attn_workspace_bytes(geom: cf_geom, batch: cf_batch) -> int:
+    return int(load_library().cf_attn_workspace_bytes(ctypes.byref(geom), ctypes.byref(batch)))
+
+
+def cf_query_prefill_attn(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor, k_cache: torch.Tensor,
+                          v_cache: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor,
+                          lse: Optional[torch.Tensor] = None, doc_scores: Optional[torch.Tensor] = None,
+                          score_accum: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, stream=None) -> None:
+    rc = load_library().cf_query_prefill_attn(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), q.data_ptr(),
+                                              k_cache.data_ptr(), v_cache.data_ptr(), softmax_scale, out.data_ptr(),
+                                              _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
+                                              workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn")
+
+
+def cf_prune_topk(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, score_accum: torch.Tensor, keep: int,
+                  strategy: int, keep_per_request: Optional[torch.Tensor] = None, stream=None) -> None:
+    rc = load_library().cf_prune_topk(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), score_accum.data_ptr(),
+                                      keep, _ptr(keep_per_request), strategy, _stream(stream))
+    _check(rc, "cf_prune_topk")
+
+
+def cf_set_attn_path(path: int) -> None:
+    _check(load_library().cf_set_attn_path(path), "cf_set_attn_path")
+
+
+def plan_field(plan: torch.Tensor, layout: cf_plan_layout, name: str, count: int, dtype=torch.int32) -> torch.Tensor:
+    """View of one field of a plan buffer (a uint8 device tensor)."""
+    off = getattr(layout, name)
+    size = count * torch.empty((), dtype=dtype).element_size()
+    return plan[off:off + size].view(dtype)

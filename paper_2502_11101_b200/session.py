@@ -1,0 +1,108 @@
+"""Buffer ownership and call sequencing around the C ABI (no arithmetic happens here).
+
+A `Session` owns the device copies of a batch's integer description, the plan buffer, the
+attention workspace and the score vectors, and issues the library calls of Algorithm 2 in
+order on the current CUDA stream."""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class Session:
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: torch.dtype, pos_range: int,
+                 rope_theta: float, q_len: int, doc_len: np.ndarray, req_doc_begin: np.ndarray,
+                 doc_src_start: np.ndarray, tail_reserve: int, prefix_len: int = 0, n_reuse: int = 0,
+                 rope_layout: int = B.CF_ROPE_HALF, token_stride: Optional[int] = None,
+                 device: str = "cuda:0"):
+        self.device = torch.device(device)
+        self.doc_len = np.asarray(doc_len, dtype=np.int32)
+        self.req_doc_begin_h = np.asarray(req_doc_begin, dtype=np.int32)
+        doc_offsets = np.zeros(len(self.doc_len) + 1, dtype=np.int32)
+        doc_offsets[1:] = np.cumsum(self.doc_len)
+        self.doc_offsets_h = doc_offsets
+        self.n_requests = len(self.req_doc_begin_h) - 1
+        self.n_docs_total = len(self.doc_len)
+        self.total_tokens = int(doc_offsets[-1])
+        self.q_len = q_len
+        self.geom = B.make_geom(n_q_heads, n_kv_heads, head_dim, dtype, pos_range, rope_theta, rope_layout)
+        self._req_doc_begin = torch.from_numpy(self.req_doc_begin_h).to(self.device)
+        self._doc_offsets = torch.from_numpy(doc_offsets).to(self.device)
+        self._doc_src_start = torch.from_numpy(np.asarray(doc_src_start, dtype=np.int32)).to(self.device)
+        stride = n_kv_heads * head_dim if token_stride is None else token_stride
+        self.batch = B.make_batch(self.n_requests, q_len, self.total_tokens, stride, self._req_doc_begin,
+                                  self._doc_offsets, self._doc_src_start, prefix_len, tail_reserve, n_reuse, 0)
+        self.layout = B.cf_plan_layout_of(self.geom, self.batch)
+        self.plan = torch.zeros(self.layout.total_bytes, dtype=torch.uint8, device=self.device)
+        self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()) if self.n_requests else 0)
+        self.workspace = torch.empty(max(256, B.cf_attn_workspace_bytes(self.geom, self.batch)), dtype=torch.uint8,
+                                     device=self.device)
+        self.doc_scores = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
+        self.score_accum = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
+
+    def set_live_docs(self, kept_per_request: int) -> None:
+        """Tell the library how many documents a request can still hold (sizes kernel grids only):
+        the hint is the tile count of the `kept_per_request` longest documents of any request."""
+        worst = 1
+        for b in range(self.n_requests):
+            lens = self.doc_len[self.req_doc_begin_h[b]:self.req_doc_begin_h[b + 1]]
+            tiles = np.sort((lens + B.CF_TILE_TOKENS - 1) // B.CF_TILE_TOKENS)[::-1]
+            worst = max(worst, int(tiles[:kept_per_request].sum()))
+        self.batch.tiles_hint = worst
+
+    def init(self, order: Optional[torch.Tensor] = None, kept_count: Optional[torch.Tensor] = None,
+             query_start: int = -1) -> None:
+        self.score_accum.zero_()
+        B.cf_plan_init(self.geom, self.batch, self.plan, order, kept_count, query_start)
+
+    def attend(self, q: torch.Tensor, k_layer: torch.Tensor, v_layer: torch.Tensor, out: torch.Tensor,
+               lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0) -> None:
+        B.cf_query_prefill_attn(self.geom, self.batch, self.plan, q, k_layer, v_layer, out, self.workspace, lse,
+                                self.doc_scores, self.score_accum, softmax_scale)
+
+    def prune(self, keep: int, strategy: int) -> None:
+        B.cf_prune_topk(self.geom, self.batch, self.plan, self.score_accum, keep, strategy)
+        self.set_live_docs(keep)
+
+    def reposition(self, k_in: torch.Tensor, k_out: torch.Tensor, n_layers: int = 1, layer_stride: int = 0) -> None:
+        B.cf_reposition_keys(self.geom, self.batch, self.plan, k_in, k_out, n_layers, layer_stride)
+
+    def status(self) -> int:
+        return B.cf_plan_status(self.geom, self.batch, self.plan)
+
+    def field(self, name: str, count: int, dtype=torch.int32) -> torch.Tensor:
+        return B.plan_field(self.plan, self.layout, name, count, dtype)
+
+    def read_plan(self) -> Dict[str, object]:
+        """Copy the integer state of the plan back to the host."""
+        nd, nb = self.n_docs_total, self.n_requests
+        kept = self.field("kept", nd).cpu().numpy()
+        count = self.field("kept_count", nb).cpu().numpy()
+        order = [list(map(int, kept[self.req_doc_begin_h[b]:self.req_doc_begin_h[b] + count[b]])) for b in range(nb)]
+        return {"order": order, "dst_start": self.field("dst_start", nd).cpu().numpy(),
+                "group": self.field("group", nd).cpu().numpy(), "n_reuse": self.field("n_reuse", nb).cpu().numpy(),
+                "query_start": self.field("query_start", nb).cpu().numpy(),
+                "n_tiles": self.field("n_tiles", nb).cpu().numpy()}
+
+    def run_stack(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, schedule: Sequence[Tuple[int, int]],
+                  strategy: int, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                  k_final: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None) -> None:
+        """Algorithm 2, Phases 1 and 2, as library calls: q, out [L, B, Lq, Hq, D]; k, v [L, T, Hkv, D];
+        lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores."""
+        sched = dict(schedule)
+        n_layers = q.shape[0]
+        self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))
+        self.init()
+        for layer in range(1, n_layers + 1):
+            i = layer - 1
+            self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
+            if layer_scores is not None:
+                layer_scores[i].copy_(self.doc_scores)
+            if layer in sched:
+                self.prune(sched[layer], strategy)
+        if k_final is not None:
+            self.reposition(k, k_final, n_layers, k.stride(0))

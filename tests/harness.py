@@ -1,0 +1,150 @@
+"""Runs the CUDA library and the CPU oracle on the same seeded workload and compares them."""
+from __future__ import annotations
+
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2502_11101_b200 import workloads as W
+
+OUT_ATOL, OUT_RTOL = 1e-2, 2e-2          # attention outputs: |g - o| <= atol + rtol |o|
+SCORE_RTOL = 2e-2                        # scores: |g - o| <= 1e-2 / n_kept + rtol |o|
+
+
+def bf16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 numbers at the binade of |x| (8 significand bits)."""
+    ax = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(ax)) - 7)
+
+
+def f32_ulp(x: np.ndarray) -> np.ndarray:
+    ax = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(ax)) - 23)
+
+
+def oracle_stack(meta: W.WorkloadMeta, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, strategy: int,
+                 schedule=None, final_reposition: bool = True, n_reuse: int = 0) -> List[Dict]:
+    cfg = meta.cfg
+    qd, kd, vd = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
+    res = []
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        res.append(oracle.run_stack(qd[:, b], kd, vd, meta.doc_len[lo:hi], meta.doc_offsets,
+                                    meta.doc_src_start[lo:hi], cfg.rope_theta, cfg.pos_range,
+                                    cfg.schedule if schedule is None else schedule, strategy,
+                                    tail_reserve=cfg.q_len, n_reuse=n_reuse, doc_base=lo,
+                                    final_reposition=final_reposition))
+    return res
+
+
+def cut_margins(meta: W.WorkloadMeta, ref: List[Dict], strategy: int, schedule=None) -> float:
+    """Smallest relative score gap that decides an integer result: at every cut of the schedule,
+    and for "sort" between neighbouring survivors."""
+    cfg = meta.cfg
+    worst = np.inf
+    for b in range(cfg.batch):
+        for layer, keep in (cfg.schedule if schedule is None else schedule):
+            rec = ref[b]["layers"][layer - 1]
+            vals = sorted((rec["score_accum"][i] for i in rec["order_in"]), reverse=True)
+            if keep < len(vals):
+                worst = min(worst, (vals[keep - 1] - vals[keep]) / vals[keep - 1])
+            if strategy == oracle.ALLOC_SORT:
+                for a, c in zip(vals[:keep], vals[1:keep]):
+                    worst = min(worst, (a - c) / a)
+    return float(worst)
+
+
+def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, device="cuda:0", n_reuse: int = 0,
+              with_final: bool = True):
+    from paper_2502_11101_b200.session import Session
+    cfg = meta.cfg
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len,
+                   n_reuse=n_reuse, device=device)
+    qg, kg, vg = q.to(device), k.to(device), v.to(device)
+    n_layers = q.shape[0]
+    out = torch.full_like(qg, float("nan"))
+    lse = torch.full((n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), float("nan"), device=device)
+    scores = torch.full((n_layers, meta.n_docs_total), float("nan"), device=device)
+    k_final = kg.clone() if with_final else None
+    sched = cfg.schedule if schedule is None else schedule
+    sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores)
+    torch.cuda.synchronize()
+    status = sess.status()
+    return {"out": out.float().cpu().numpy(), "lse": lse.cpu().numpy(), "scores": scores.cpu().numpy(),
+            "accum": sess.score_accum.cpu().numpy(), "plan": sess.read_plan(), "status": status,
+            "k_final": None if k_final is None else k_final.float().cpu().numpy(), "session": sess}
+
+
+def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Tensor) -> Dict[str, float]:
+    """Element-by-element comparison; raises AssertionError with the offending quantity."""
+    cfg = meta.cfg
+    n_layers = len(ref[0]["layers"])
+    assert got["status"] == 0, f"device status {got['status']}"
+    report = {"out_max_abs": 0.0, "score_max_rel": 0.0, "lse_max_abs": 0.0, "key_max_ulp": 0.0}
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        r = ref[b]
+        # integer results: bit-exact
+        assert got["plan"]["order"][b] == r["order"], f"request {b}: kept set/order differs"
+        assert np.array_equal(got["plan"]["dst_start"][lo:hi], r["dst_start"]), f"request {b}: dst_start differs"
+        assert np.array_equal(got["plan"]["group"][lo:hi], r["group"]), f"request {b}: window index differs"
+        assert int(got["plan"]["query_start"][b]) == r["query_start"]
+        assert int(got["plan"]["n_reuse"][b]) == r["n_reuse"]
+        for l in range(n_layers):
+            rec = r["layers"][l]
+            o_ref = rec["out"]
+            o_got = got["out"][l, b]
+            err = np.abs(o_got - o_ref)
+            assert np.all(err <= OUT_ATOL + OUT_RTOL * np.abs(o_ref)), \
+                f"request {b} layer {l + 1}: output error {err.max():.3e}"
+            report["out_max_abs"] = max(report["out_max_abs"], float(err.max()))
+            lse_err = np.abs(got["lse"][l, b] - rec["lse"])
+            assert np.all(lse_err <= 1e-2), f"request {b} layer {l + 1}: lse error {lse_err.max():.3e}"
+            report["lse_max_abs"] = max(report["lse_max_abs"], float(lse_err.max()))
+            s_ref = rec["doc_scores"]
+            s_got = got["scores"][l, lo:hi]
+            n_kept = len(rec["order_in"])
+            s_err = np.abs(s_got - s_ref)
+            assert np.all(s_err <= 1e-2 / n_kept + SCORE_RTOL * np.abs(s_ref)), \
+                f"request {b} layer {l + 1}: score error {s_err.max():.3e}"
+            kept = np.array(rec["order_in"])
+            report["score_max_rel"] = max(report["score_max_rel"], float((s_err[kept] / s_ref[kept]).max()))
+            pruned = np.setdiff1d(np.arange(hi - lo), kept)
+            assert np.all(s_got[pruned] == 0.0), "pruned documents must score exactly 0"
+            assert abs(float(s_got.sum()) - 1.0) < 1e-3, "document scores of a request must sum to 1"
+        acc_err = np.abs(got["accum"][lo:hi] - r["score_accum"])
+        assert np.all(acc_err <= 1e-2 + SCORE_RTOL * np.abs(r["score_accum"]))
+    if got["k_final"] is not None:
+        k_in = k_store.float().cpu().numpy()
+        ulp = bf16_ulp if cfg.dtype == "bf16" else (lambda x: 4.0 * f32_ulp(x))
+        for b in range(cfg.batch):
+            lo = int(meta.req_doc_begin[b])
+            survivors = set(ref[b]["order"])
+            for l in range(n_layers):
+                kf_ref = ref[b]["k_final"][l]
+                for i in range(int(meta.req_doc_begin[b + 1]) - lo):
+                    a, c = int(meta.doc_offsets[lo + i]), int(meta.doc_offsets[lo + i + 1])
+                    if i in survivors:
+                        err = np.abs(got["k_final"][l, a:c] - kf_ref[a:c]) / ulp(kf_ref[a:c])
+                        assert err.max() <= 1.0, f"rotated key off by {err.max():.3f} ulp (layer {l + 1}, doc {i})"
+                        report["key_max_ulp"] = max(report["key_max_ulp"], float(err.max()))
+                    else:
+                        assert np.array_equal(got["k_final"][l, a:c], k_in[l, a:c]), "pruned rows must stay untouched"
+    return report
+
+
+def run_and_compare(cfg: W.WorkloadConfig, seed: int, strategy: int, device="cuda:0", n_reuse: int = 0,
+                    min_margin: float = 2e-3, doc_len_override=None) -> Dict[str, float]:
+    meta = W.make_meta(cfg, seed, doc_len_override)
+    q = W.make_q(meta)
+    k, v = W.make_kv(meta)
+    ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse)
+    margin = cut_margins(meta, ref, strategy)
+    assert margin >= min_margin, f"workload rejected: decisive score gap {margin:.2e} below {min_margin:.0e}"
+    got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse)
+    report = compare(meta, ref, got, k)
+    report["margin"] = margin
+    return report

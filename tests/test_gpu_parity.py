@@ -1,0 +1,176 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle on seeded workloads.
+
+Tolerances: integer results (positions, windows, kept sets and their order) bit-exact; rotated
+keys within 1 bf16 ulp (4 fp32 ulp for fp32 storage) of the fp64 value; attention outputs within
+1e-2 + 2e-2*|ref|; document scores within 1e-2/n_kept + 2e-2*|ref|."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2502_11101_b200 import workloads as W
+from tests import harness
+
+pytestmark = pytest.mark.gpu
+
+STRATEGIES = [oracle.ALLOC_NONE, oracle.ALLOC_ALIGN, oracle.ALLOC_SORT]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    assert torch.cuda.is_available()
+    from paper_2502_11101_b200 import build
+    build.build()
+    import paper_2502_11101_b200 as cf
+    cf.load_library()
+
+
+def _pick_seed(cfg, strategy, min_margin=2e-3, tries=6):
+    """First seed whose oracle run has no decisive score gap inside the tolerance."""
+    for seed in range(tries):
+        meta = W.make_meta(cfg, seed)
+        ref = harness.oracle_stack(meta, W.make_q(meta), *W.make_kv(meta), strategy, final_reposition=False)
+        if harness.cut_margins(meta, ref, strategy) >= min_margin:
+            return seed
+    raise AssertionError("no seed with a safe margin")
+
+
+@pytest.mark.parametrize("strategy", STRATEGIES)
+def test_config1_tiny_fp32(strategy):
+    cfg = W.CONFIGS[1]
+    rep = harness.run_and_compare(cfg, _pick_seed(cfg, strategy), strategy)
+    assert rep["out_max_abs"] < 1e-4 and rep["score_max_rel"] < 1e-4      # fp32 path is much tighter
+
+
+@pytest.mark.parametrize("strategy", [oracle.ALLOC_ALIGN, oracle.ALLOC_SORT])
+def test_config2_llama_layer(strategy):
+    cfg = W.CONFIGS[2]
+    harness.run_and_compare(cfg, _pick_seed(cfg, strategy), strategy)
+
+
+@pytest.mark.parametrize("strategy", STRATEGIES)
+def test_config3_qwen_stack(strategy):
+    cfg = W.CONFIGS[3]
+    harness.run_and_compare(cfg, _pick_seed(cfg, strategy, min_margin=1e-3), strategy, min_margin=1e-3)
+
+
+def test_config4_reduced_batch_of_requests():
+    cfg = W.scaled_config(W.CONFIGS[4], n_layers=5, batch=2, schedule=((1, 50), (3, 25), (4, 12)))
+    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3)
+
+
+def test_config5_reduced_parallel_windows():
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=3, batch=2, schedule=((1, 60), (2, 30)))
+    meta = W.make_meta(cfg, 0)
+    dst, grp, n_reuse, qs = oracle.allocate_positions(meta.doc_len[:120], range(120), 4096, 0, 64)
+    assert n_reuse == 6                                   # six parallel windows inside the 4096 range
+    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_SORT, 1e-3), oracle.ALLOC_SORT, min_margin=1e-3)
+
+
+@pytest.mark.parametrize("dtype,head_dim", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
+def test_ragged_document_lengths(dtype, head_dim):
+    lens = [1, 63, 64, 65, 127, 128, 129, 200, 300, 17, 256, 31]
+    cfg = W.WorkloadConfig("ragged", 2, 8, 2, head_dim, dtype, 1e4, 4096, len(lens), 1, 300, 5, 1, 2,
+                           ((1, 7),))
+    harness.run_and_compare(cfg, 1, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=1e-3)
+
+
+def test_forced_window_counts():
+    cfg = W.scaled_config(W.CONFIGS[2], n_docs=12, n_planted=2, schedule=((1, 6),))
+    for n_reuse in (1, 3, 12):                            # sequential, k/4, fully parallel (Sec. 3.3)
+        harness.run_and_compare(cfg, 0, oracle.ALLOC_ALIGN, n_reuse=n_reuse, min_margin=1e-3)
+
+
+def test_keep_larger_than_live_set_and_no_pruning():
+    cfg = W.scaled_config(W.CONFIGS[3], n_layers=3, n_docs=9, n_planted=2, schedule=((1, 20), (2, 9)))
+    harness.run_and_compare(cfg, 0, oracle.ALLOC_SORT, min_margin=1e-3)
+
+
+def test_results_are_bitwise_reproducible():
+    cfg = W.scaled_config(W.CONFIGS[3], n_layers=2, n_docs=20, schedule=((1, 10),))
+    meta = W.make_meta(cfg, 0)
+    q = W.make_q(meta)
+    k, v = W.make_kv(meta)
+    a = harness.gpu_stack(meta, q, k, v, oracle.ALLOC_ALIGN)
+    b = harness.gpu_stack(meta, q, k, v, oracle.ALLOC_ALIGN)
+    for key in ("out", "lse", "scores", "accum", "k_final"):
+        assert np.array_equal(a[key], b[key]), key
+
+
+def test_interleaved_slice_layout():
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[2], n_docs=6, n_planted=1, n_q_heads=4, n_kv_heads=2)
+    meta = W.make_meta(cfg, 0)
+    q = W.make_q(meta)
+    k, v = W.make_kv(meta)
+    sess = Session(4, 2, 128, torch.bfloat16, 4096, 1e4, cfg.q_len, meta.doc_len, meta.req_doc_begin,
+                   meta.doc_src_start, tail_reserve=cfg.q_len, rope_layout=cf.CF_ROPE_INTERLEAVED)
+    qg, kg, vg = q.cuda(), k.cuda(), v.cuda()
+    out = torch.empty_like(qg[0])
+    sess.init()
+    sess.attend(qg[0], kg[0], vg[0], out)
+    k_rot = torch.empty_like(kg[0])
+    sess.reposition(kg[0], k_rot)
+    plan = sess.read_plan()
+    order = plan["order"][0]
+    kr = oracle.reposition_keys(k[0].double().numpy(), meta.doc_offsets, meta.doc_src_start, plan["dst_start"],
+                                order, 1e4, oracle.ROPE_INTERLEAVED)
+    o_ref, _, _, s_ref = oracle.query_prefill_attn(q[0, 0].double().numpy(), kr, v[0].double().numpy(),
+                                                   meta.doc_offsets, order, cfg.n_docs)
+    err = np.abs(k_rot.float().cpu().numpy() - kr) / harness.bf16_ulp(kr)
+    assert err.max() <= 1.0
+    assert np.all(np.abs(out[0].float().cpu().numpy() - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
+    assert np.allclose(sess.doc_scores.cpu().numpy(), s_ref, rtol=2e-2, atol=1e-3)
+
+
+def test_fused_equals_reposition_then_attend():
+    """Rotating on the way in (fused) and re-positioning the store first, then attending with a zero
+    delta, are the same computation: outputs agree bit for bit."""
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[3], n_layers=1, n_docs=12, n_planted=2, schedule=())
+    meta = W.make_meta(cfg, 2)
+    q, (k, v) = W.make_q(meta).cuda(), [t.cuda() for t in W.make_kv(meta)]
+
+    def session(src_start):
+        return Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                       cfg.q_len, meta.doc_len, meta.req_doc_begin, src_start, tail_reserve=cfg.q_len)
+    fused = session(meta.doc_src_start)
+    fused.init()
+    out_a = torch.empty_like(q[0])
+    fused.attend(q[0], k[0], v[0], out_a)
+    k_rot = torch.empty_like(k[0])
+    fused.reposition(k[0], k_rot)
+    moved = session(fused.read_plan()["dst_start"])       # the store now sits at its destination
+    moved.init()
+    out_b = torch.empty_like(q[0])
+    moved.attend(q[0], k_rot, v[0], out_b)
+    assert torch.equal(out_a, out_b)
+    assert torch.equal(fused.doc_scores, moved.doc_scores)
+
+
+def test_argument_errors_are_reported_not_faulted():
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[2], n_docs=4, n_planted=1)
+    meta = W.make_meta(cfg, 0)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+    q, (k, v) = W.make_q(meta).cuda(), [t.cuda() for t in W.make_kv(meta)]
+    out = torch.empty_like(q[0])
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(cf.CacheFocusError) as e:
+        cf.cf_query_prefill_attn(sess.geom, sess.batch, sess.plan, q[0], k[0], v[0], out, small)
+    assert e.value.code == cf.CF_ERR_WORKSPACE
+    with pytest.raises(cf.CacheFocusError) as e:
+        cf.cf_plan_init(sess.geom, sess.batch, small)
+    assert e.value.code == cf.CF_ERR_WORKSPACE
+    bad = cf.make_geom(5, 2, 128, cf.CF_BF16, 4096, 1e4)
+    with pytest.raises(cf.CacheFocusError) as e:
+        cf.cf_plan_layout_of(bad, sess.batch)
+    assert e.value.code == cf.CF_ERR_INVALID_ARG
+    # a range too small for the documents is reported through the plan's status word
+    tight = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, 100 + cfg.q_len, cfg.rope_theta,
+                    cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+    tight.init()
+    assert tight.status() == cf.CF_ERR_RANGE
