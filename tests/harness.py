@@ -119,7 +119,7 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
         assert np.all(acc_err <= 1e-2 + SCORE_RTOL * np.abs(r["score_accum"]))
     if got["k_final"] is not None:
         k_in = k_store.float().cpu().numpy()
-        ulp = bf16_ulp if cfg.dtype == "bf16" else (lambda x: 4.0 * f32_ulp(x))
+        half = cfg.head_dim // 2
         for b in range(cfg.batch):
             lo = int(meta.req_doc_begin[b])
             survivors = set(ref[b]["order"])
@@ -128,8 +128,14 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
                 for i in range(int(meta.req_doc_begin[b + 1]) - lo):
                     a, c = int(meta.doc_offsets[lo + i]), int(meta.doc_offsets[lo + i + 1])
                     if i in survivors:
-                        err = np.abs(got["k_final"][l, a:c] - kf_ref[a:c]) / ulp(kf_ref[a:c])
-                        assert err.max() <= 1.0, f"rotated key off by {err.max():.3f} ulp (layer {l + 1}, doc {i})"
+                        want = kf_ref[a:c]
+                        # one rounding to the storage type at the result, plus fp32 arithmetic at the
+                        # magnitude of the slice (a slice keeps its norm under rotation)
+                        norm = np.sqrt(want[..., :half] ** 2 + want[..., half:] ** 2)
+                        arith = 4.0 * f32_ulp(np.concatenate([norm, norm], axis=-1))
+                        tol = arith if cfg.dtype == "f32" else bf16_ulp(want) + arith
+                        err = np.abs(got["k_final"][l, a:c] - want) / tol
+                        assert err.max() <= 1.0, f"rotated key off by {err.max():.3f} tol (layer {l + 1}, doc {i})"
                         report["key_max_ulp"] = max(report["key_max_ulp"], float(err.max()))
                     else:
                         assert np.array_equal(got["k_final"][l, a:c], k_in[l, a:c]), "pruned rows must stay untouched"

@@ -64,7 +64,7 @@ def test_config5_reduced_parallel_windows():
     meta = W.make_meta(cfg, 0)
     dst, grp, n_reuse, qs = oracle.allocate_positions(meta.doc_len[:120], range(120), 4096, 0, 64)
     assert n_reuse == 6                                   # six parallel windows inside the 4096 range
-    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_SORT, 1e-3), oracle.ALLOC_SORT, min_margin=1e-3)
+    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3)
 
 
 @pytest.mark.parametrize("dtype,head_dim", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
