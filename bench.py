@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the CacheFocus query-time path on B200.
+
+One "step" is one pass of the whole hot path for one batch of synthetic requests: positional
+allocation, then per layer the fused re-position + query-prefill attention with document scores
+and score accumulation, pruning + re-allocation at the scheduled layers, and the final
+re-positioning of the surviving caches in every layer (Algorithm 2, Phases 1 and 2).
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload 3]
+
+Prints one JSON line (rank 0).  `value` = cached KV tokens (one token position of one layer of a
+kept document) processed per second with inputs resident in HBM; `e2e` = the same with the
+query and the cache store starting in pinned host memory every step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2502_11101_b200 import workloads as W  # noqa: E402
+
+METRIC = "cached KV tokens/s through reposition+query-prefill attn"
+UNIT = "tokens/s"
+STRATEGY_ALIGN = 1
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "tflops": float(p["bf16_tflops"]),
+                "tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples = []
+        self.proc = None
+        self.thread = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) >= 7:
+                try:
+                    self.samples.append((time.time(), float(parts[0]), float(parts[1]), parts[3:7]))
+                except ValueError:
+                    pass
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        inside = [s for s in self.samples if t0 <= s[0] <= t1 + 0.15] or self.samples[-3:]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for s in inside for i in range(4) if s[3][i].lower().startswith("active")})
+        return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": inside[0][2],
+                "reasons": reasons, "samples": len(inside)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def token_layers(cfg, meta, kept_lists):
+    """Cached tokens visited per layer given the kept sets in force at each layer."""
+    per_layer = []
+    for layer in range(1, cfg.n_layers + 1):
+        total = 0
+        for b in range(cfg.batch):
+            base = int(meta.req_doc_begin[b])
+            total += int(sum(int(meta.doc_len[base + i]) for i in kept_lists[layer - 1][b]))
+        per_layer.append(total)
+    return per_layer
+
+
+class GpuWorkload:
+    """A ring of resident input sets (distinct seeds) so that consecutive steps never find their
+    inputs in L2, plus the session and output buffers of the library."""
+
+    def __init__(self, cfg, seed, device, ring):
+        from paper_2502_11101_b200.session import Session
+        self.cfg, self.device = cfg, device
+        self.meta = W.make_meta(cfg, seed)
+        m = self.meta
+        self.sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range,
+                            cfg.rope_theta, cfg.q_len, m.doc_len, m.req_doc_begin, m.doc_src_start,
+                            tail_reserve=cfg.q_len, device=device)
+        self.slots = []
+        for r in range(ring):
+            # same documents (lengths, relevance), fresh tensor contents per slot
+            mr = W.make_meta(cfg, seed + 1000 * r, doc_len_override=m.doc_len) if r else m
+            mr.key_scale[:] = m.key_scale
+            q = W.make_q(mr, device)
+            k, v = W.make_kv(mr, device)
+            self.slots.append((q, k, v))
+        q0 = self.slots[0][0]
+        self.out = torch.empty_like(q0)
+        self.lse = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), device=device)
+        self.k_final = torch.empty_like(self.slots[0][1])
+
+    def step(self, slot):
+        q, k, v = self.slots[slot % len(self.slots)]
+        self.sess.run_stack(q, k, v, self.cfg.schedule, STRATEGY_ALIGN, self.out, self.lse, self.k_final)
+
+    def kept_per_layer(self, slot=0):
+        """One instrumented step: the kept sets seen by every layer."""
+        q, k, v = self.slots[slot]
+        cfg, sess = self.cfg, self.sess
+        sched = dict(cfg.schedule)
+        sess.set_live_docs(cfg.n_docs)
+        sess.init()
+        kept = []
+        current = sess.read_plan()["order"]
+        for layer in range(1, cfg.n_layers + 1):
+            kept.append(current)
+            sess.attend(q[layer - 1], k[layer - 1], v[layer - 1], self.out[layer - 1], self.lse[layer - 1])
+            if layer in sched:
+                sess.prune(sched[layer], STRATEGY_ALIGN)
+                current = sess.read_plan()["order"]
+        return kept, current
+
+    def launches_per_step(self):
+        cfg = self.cfg
+        # plan init + per layer (attention, merge, scores) + prune/plan kernels + final re-positioning
+        return 1 + 3 * cfg.n_layers + len(cfg.schedule) + 1
+
+
+def time_steps(fn, steps, warmup, world):
+    import torch.distributed as dist
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    start.record()
+    for i in range(steps):
+        fn(warmup + i)
+    stop.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    if world > 1:
+        dist.barrier()
+    return start.elapsed_time(stop), t0, t1
+
+
+def oracle_sample(cfg, seed):
+    """The oracle, as it stands, on one request of the workload (all layers, pruning schedule)."""
+    import oracle
+    one = W.scaled_config(cfg, batch=1)
+    meta = W.make_meta(one, seed)
+    q = W.make_q(meta).double().numpy()
+    k, v = W.make_kv(meta)
+    k, v = k.double().numpy(), v.double().numpy()
+    t0 = time.perf_counter()
+    res = oracle.run_stack(q[:, 0], k, v, meta.doc_len, meta.doc_offsets, meta.doc_src_start, one.rope_theta,
+                           one.pos_range, one.schedule, STRATEGY_ALIGN, tail_reserve=one.q_len)
+    dt = time.perf_counter() - t0
+    tokens = sum(int(sum(int(meta.doc_len[i]) for i in rec["order_in"])) for rec in res["layers"])
+    return dt, tokens
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg, rank):
+    if rank != 0:
+        return
+    times, tokens = [], []
+    for i in range(args.warmup):
+        oracle_sample(cfg, 100 + i)
+    for i in range(args.steps):
+        dt, tk = oracle_sample(cfg, i)
+        times.append(dt)
+        tokens.append(tk)
+    value = sum(tokens) / sum(times)
+    sample = f"one request of workload {args.workload} per step (all {cfg.n_layers} layers, pruning schedule), fp64"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"configs[{args.workload - 1}] {cfg.name}", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, help="1-based index into the named configurations")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--ring", type=int, default=3, help="distinct resident input sets cycled between steps")
+    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.CONFIGS[args.workload]
+    rank, world, local = dist_env()
+
+    if args.impl == "reference":
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, cfg, rank)
+        return
+
+    args.steps = 300 if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else max(3, args.warmup)
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200 import build as cf_build
+    if rank == 0:
+        cf_build.build()
+    if world > 1:
+        dist.barrier()
+    cf.load_library()
+    if args.force_simt:
+        cf.cf_set_attn_path(1)
+    peaks = load_peaks()
+
+    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring)
+    kept, survivors = wl.kept_per_layer()
+    per_layer_tokens = token_layers(cfg, wl.meta, kept)
+    tokens_per_step = sum(per_layer_tokens)
+    final_tokens = sum(int(wl.meta.doc_len[int(wl.meta.req_doc_begin[b]) + i]) for b in range(cfg.batch)
+                       for i in survivors[b]) * cfg.n_layers
+    assert wl.sess.status() == 0
+
+    # ---- CUDA graphs: one per ring slot (pointers differ) -------------------------------------
+    graphs = None
+    if not args.no_graph:
+        try:
+            wl.step(0)
+            torch.cuda.synchronize()
+            graphs = []
+            side = torch.cuda.Stream()
+            for r in range(args.ring):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    wl.step(r)
+                graphs.append(g)
+        except Exception as exc:  # capture not possible: time eager launches and say so
+            graphs = None
+            sys.stderr.write(f"[bench] graph capture failed, timing eager launches: {exc}\n")
+            torch.cuda.synchronize()
+
+    def run(i):
+        if graphs is not None:
+            graphs[i % args.ring].replay()
+        else:
+            wl.step(i)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, t0, t1 = time_steps(run, args.steps, args.warmup, world)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    assert wl.sess.status() == 0
+
+    stats = torch.tensor([ms, float(tokens_per_step)], dtype=torch.float64, device=device)
+    if world > 1:
+        mx = stats.clone()
+        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = stats.clone()
+        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms_max, tokens_all = float(mx[0]), float(sm[1])
+    else:
+        ms_max, tokens_all = ms, float(tokens_per_step)
+    value = tokens_all * args.steps / (ms_max * 1e-3)
+
+    # ---- the dominant kernel alone: event pairs around every attention-kernel launch ----------
+    prof_steps = max(1, min(args.steps, 20))
+    for i in range(3):
+        wl.step(i)
+    torch.cuda.synchronize()
+    cf.cf_profile_begin(prof_steps * cfg.n_layers)
+    for i in range(prof_steps):
+        wl.step(3 + i)
+    durations = cf.cf_profile_end(prof_steps * cfg.n_layers).astype(np.float64)
+    kv_bytes_per_token = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4) * cfg.n_kv_heads
+    flops_per_token = 4 * cfg.group_size * cfg.q_len * cfg.head_dim * cfg.n_kv_heads
+    launch_bytes = np.tile(np.array(per_layer_tokens, dtype=np.float64) * kv_bytes_per_token, prof_steps)
+    launch_flops = np.tile(np.array(per_layer_tokens, dtype=np.float64) * flops_per_token, prof_steps)
+    n = min(len(durations), len(launch_bytes))
+    dur_s = durations[:n].sum() * 1e-3
+    gbs = launch_bytes[:n].sum() / dur_s / 1e9
+    tfs = launch_flops[:n].sum() / dur_s / 1e12
+    t_hbm = launch_bytes[:n].sum() / (peaks["hbm_gbs"] * 1e9)
+    t_tc = launch_flops[:n].sum() / (peaks["tflops"] * 1e12)
+    if t_tc > t_hbm:
+        roofline = {"bound": "tensor", "achieved": tfs, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                    "frac": tfs / peaks["tflops"]}
+    else:
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": gbs / peaks["hbm_gbs"]}
+    roofline.update({"traffic": None, "kernel": "fused re-position + query-prefill attention",
+                     "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
+                     "launches_timed": int(n), "hbm_gbs": gbs, "tflops": tfs,
+                     "frac_of_applicable_roofline": max(t_hbm, t_tc) / dur_s})
+
+    # ---- end to end: query and cache store start in pinned host memory every step --------------
+    q0, k0, v0 = wl.slots[0]
+    host = [t.cpu().pin_memory() for t in (q0, k0, v0)]
+    out_h = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
+    acc_h = torch.empty(wl.sess.score_accum.shape, dtype=torch.float32).pin_memory()
+    kept_h = torch.empty(wl.sess.n_docs_total, dtype=torch.int32).pin_memory()
+
+    def e2e_step(_):
+        for src, dst in zip(host, (q0, k0, v0)):
+            dst.copy_(src, non_blocking=True)
+        wl.step(0)
+        out_h.copy_(wl.out, non_blocking=True)
+        acc_h.copy_(wl.sess.score_accum, non_blocking=True)
+        kept_h.copy_(wl.sess.field("kept", wl.sess.n_docs_total), non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 20))
+    e2e_ms, _, _ = time_steps(e2e_step, e2e_steps, 3, world)
+    e2e_stats = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(e2e_stats, op=dist.ReduceOp.MAX)
+    h2d = sum(t.numel() * t.element_size() for t in host)
+    d2h = sum(t.numel() * t.element_size() for t in (out_h, acc_h, kept_h))
+    e2e = {"value": tokens_all * e2e_steps / (float(e2e_stats[0]) * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.skip_cpu_baseline:
+        t_total, tok_total, reps = 0.0, 0, 0
+        while t_total < 10.0 and reps < 8:
+            dt, tk = oracle_sample(cfg, 50 + reps)
+            t_total += dt
+            tok_total += tk
+            reps += 1
+        cpu = {"value": tok_total / t_total, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"{reps} x one request of workload {args.workload} (all {cfg.n_layers} layers, "
+                         f"pruning schedule), {t_total:.1f} s of fp64 numpy"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": f"configs[{args.workload - 1}] {cfg.name}", "n_layers": cfg.n_layers,
+                       "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+                       "docs_per_request": cfg.n_docs, "requests": cfg.batch, "q_len": cfg.q_len,
+                       "schedule": [list(s) for s in cfg.schedule], "strategy": "align",
+                       "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
+                       "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
+                             f"{sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6:.0f} MB) cycled between steps",
+                       "launch": "cuda graph per ring slot" if graphs is not None else "eager",
+                       "attention_kernel": "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05",
+                       "parallelism": f"replicas x{world}"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": wl.launches_per_step() * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def _tc_used(cf, wl):
+    return wl.cfg.dtype == "bf16" and wl.cfg.head_dim == 128 and getattr(cf, "TC_KERNEL_BUILT", False)
+
+
+if __name__ == "__main__":
+    main()

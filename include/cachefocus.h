@@ -211,6 +211,16 @@ int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
  * 1 = force the portable CUDA-core kernel.  Process-wide; meant for tests and debugging. */
 int cf_set_attn_path(int32_t path);
 
+/* Timing aid for benchmarks (not part of the method).  cf_profile_begin(n) makes every later
+ * cf_query_prefill_attn call bracket its main attention kernel (the fused re-position +
+ * QK^T + softmax + PV kernel, without the small merge kernels) with a pair of CUDA events on
+ * the launching stream, for at most n calls.  cf_profile_end() waits for those events, writes
+ * the kernel durations in milliseconds to the host array `ms` (capacity entries), the number
+ * of recorded launches to *count, and switches recording off.  Do not use inside stream
+ * capture.  The events are created by cf_profile_begin and destroyed by cf_profile_end. */
+int cf_profile_begin(int32_t max_records);
+int cf_profile_end(float* ms, int32_t capacity, int32_t* count);
+
 #ifdef __cplusplus
 }
 #endif

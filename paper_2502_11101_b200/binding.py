@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
-           "cf_query_prefill_attn", "cf_prune_topk", "cf_set_attn_path"]
+           "cf_query_prefill_attn", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -80,6 +80,8 @@ def load_library() -> ctypes.CDLL:
                                           ctypes.c_size_t, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
     lib.cf_set_attn_path.argtypes = [i32]
+    lib.cf_profile_begin.argtypes = [i32]
+    lib.cf_profile_end.argtypes = [vp, i32, vp]
     for name in EXPORTS:
         if name not in ("cf_error_string", "cf_attn_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
@@ -208,6 +210,18 @@ def cf_prune_topk(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, score_accu
 
 def cf_set_attn_path(path: int) -> None:
     _check(load_library().cf_set_attn_path(path), "cf_set_attn_path")
+
+
+def cf_profile_begin(max_records: int) -> None:
+    _check(load_library().cf_profile_begin(max_records), "cf_profile_begin")
+
+
+def cf_profile_end(capacity: int) -> np.ndarray:
+    """Durations (ms) of the attention kernel launches recorded since cf_profile_begin."""
+    ms = np.zeros(max(1, capacity), np.float32)
+    count = ctypes.c_int32(0)
+    _check(load_library().cf_profile_end(ms.ctypes.data, capacity, ctypes.addressof(count)), "cf_profile_end")
+    return ms[:min(capacity, count.value)]
 
 
 def plan_field(plan: torch.Tensor, layout: cf_plan_layout, name: str, count: int, dtype=torch.int32) -> torch.Tensor:

@@ -172,6 +172,11 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
 
 static std::atomic<int> g_attn_path{0};
 
+// Event pairs around the main attention kernel (cf_profile_begin / cf_profile_end).
+static std::vector<cudaEvent_t> g_prof_events;
+static int g_prof_capacity = 0;
+static int g_prof_used = 0;
+
 }  // namespace cf
 
 using namespace cf;
@@ -324,6 +329,34 @@ size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch) {
     return attn_workspace_layout(geom, batch, choose_splits(geom, batch), nullptr, nullptr);
 }
 
+int cf_profile_begin(int32_t max_records) {
+    if (max_records <= 0 || max_records > (1 << 20) || g_prof_capacity != 0) return CF_ERR_INVALID_ARG;
+    g_prof_events.resize(2 * (size_t)max_records);
+    for (auto& e : g_prof_events)
+        if (cudaEventCreate(&e) != cudaSuccess) return CF_ERR_CUDA;
+    g_prof_used = 0;
+    g_prof_capacity = max_records;
+    return CF_OK;
+}
+
+int cf_profile_end(float* ms, int32_t capacity, int32_t* count) {
+    if (!count || capacity < 0 || (capacity > 0 && !ms)) return CF_ERR_INVALID_ARG;
+    int rc = CF_OK;
+    const int n = g_prof_used;
+    for (int i = 0; i < n; ++i) {
+        float t = 0.f;
+        if (cudaEventSynchronize(g_prof_events[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&t, g_prof_events[2 * i], g_prof_events[2 * i + 1]) != cudaSuccess)
+            rc = CF_ERR_CUDA;
+        if (i < capacity) ms[i] = t;
+    }
+    for (auto& e : g_prof_events) cudaEventDestroy(e);
+    g_prof_events.clear();
+    g_prof_capacity = g_prof_used = 0;
+    *count = n;
+    return rc;
+}
+
 int cf_set_attn_path(int32_t path) {
     if (path != 0 && path != 1) return CF_ERR_INVALID_ARG;
     g_attn_path.store(path);
@@ -350,10 +383,13 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool timed = g_prof_used < g_prof_capacity;
+    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
     if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch))
         rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
     else
         rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
+    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);
     if (rc != CF_OK) return rc;
     return launch_combine(geom, batch, pv, ws, out, lse, doc_scores, score_accum, s);
 }

@@ -238,16 +238,20 @@ static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView
     dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_chunks), (unsigned)b->n_requests);
     BatchView bv = make_batch_view(b);
     const size_t smem = simt_smem_bytes<D>();
-    auto run = [&](auto kernel) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return CF_ERR_CUDA;
+    static bool configured[2] = {false, false};      // per (T, D) instantiation and slice layout
+    auto run = [&](auto kernel, int which) {
+        if (!configured[which]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return CF_ERR_CUDA;
+            configured[which] = true;
+        }
         kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, g->n_q_heads, g->n_kv_heads, scale_log2,
                                                      static_cast<const T*>(q), static_cast<const T*>(k),
                                                      static_cast<const T*>(v));
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
-    if (g->rope_layout == CF_ROPE_HALF) return run(attn_simt_kernel<T, D, CF_ROPE_HALF>);
-    return run(attn_simt_kernel<T, D, CF_ROPE_INTERLEAVED>);
+    if (g->rope_layout == CF_ROPE_HALF) return run(attn_simt_kernel<T, D, CF_ROPE_HALF>, 0);
+    return run(attn_simt_kernel<T, D, CF_ROPE_INTERLEAVED>, 1);
 }
 
 int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
