@@ -58,6 +58,7 @@ extern "C" {
 #define CF_TILE_TOKENS 128      /* key tiles never straddle two documents                       */
 #define CF_MAX_DOCS_PER_REQUEST 1024
 #define CF_MAX_SPLITS 64
+#define CF_STATIC_WORKSPACE_BYTES (32u << 20)   /* scratch carried by cf_query_prefill_attn_static */
 
 /* Model-side geometry.  head_dim 64 or 128; pos_range = the model's positional range L of
  * Eq. 6; rope_theta = base of the rotary frequencies theta^(-2p/head_dim). */
@@ -196,6 +197,30 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
                           float softmax_scale, void* out, float* lse, float* doc_scores,
                           float* score_accum, void* workspace, size_t workspace_bytes,
                           void* stream);
+
+/* The same computation as cf_query_prefill_attn for callers that cannot allocate device memory
+ * (the paper has no counterpart; this is a property of the library, not of the method).
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that owns the allocator and hands out only input and output buffers, a serving
+ * loop that has frozen its memory pool, a caller already inside a region where allocation would
+ * synchronise the device.  Such a caller has nowhere to put the attention workspace, so here the
+ * workspace is a fixed array of CF_STATIC_WORKSPACE_BYTES (32 MiB) that is part of the library
+ * image: every GPU that loads the library holds those bytes until the process exits.
+ *   - Arguments are those of cf_query_prefill_attn without workspace / workspace_bytes.
+ *   - Returns CF_ERR_WORKSPACE, launching nothing, when cf_attn_workspace_bytes(geom, batch) for
+ *     this batch exceeds CF_STATIC_WORKSPACE_BYTES.  Use a smaller batch or the ordinary call.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress); make that first call outside any stream capture.  No call allocates
+ *     or frees device memory.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     Nothing in it has to start at zero: each call overwrites every word it later reads.  Two
+ *     calls that run on the GPU at the same time (different streams, or different host threads)
+ *     would overwrite each other's partial results: issue them on one stream, or otherwise make
+ *     sure they do not overlap. */
+int cf_query_prefill_attn_static(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                                 const void* q, const void* k_cache, const void* v_cache,
+                                 float softmax_scale, void* out, float* lse, float* doc_scores,
+                                 float* score_accum, void* stream);
 
 /* Layer-Adaptive Cache Pruning step (Algorithm 2: argsort of S, prun) followed by the
  * re-allocation of the survivors (Sec. 2.5), all on the device: per request keeps the `keep`

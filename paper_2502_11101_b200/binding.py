@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
-           "cf_query_prefill_attn", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_query_prefill_attn", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -78,6 +78,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes.argtypes = [gp, bp]
     lib.cf_query_prefill_attn.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
+    lib.cf_query_prefill_attn_static.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
@@ -199,6 +200,21 @@ def cf_query_prefill_attn(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q:
                                               _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
                                               workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn")
+
+
+def cf_query_prefill_attn_static(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,
+                                 k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+                                 lse: Optional[torch.Tensor] = None, doc_scores: Optional[torch.Tensor] = None,
+                                 score_accum: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                                 stream=None) -> None:
+    """cf_query_prefill_attn without a workspace argument: the scratch is a fixed 32 MiB array inside
+    the library, for callers that may not allocate device memory.  Raises CacheFocusError with
+    CF_ERR_WORKSPACE when the batch needs more scratch than that."""
+    rc = load_library().cf_query_prefill_attn_static(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(),
+                                                     q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), softmax_scale,
+                                                     out.data_ptr(), _ptr(lse), _ptr(doc_scores), _ptr(score_accum),
+                                                     _stream(stream))
+    _check(rc, "cf_query_prefill_attn_static")
 
 
 def cf_prune_topk(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, score_accum: torch.Tensor, keep: int,

@@ -171,6 +171,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
 }
 
 static std::atomic<int> g_attn_path{0};
+int attn_path() { return g_attn_path.load(); }
 
 // Event pairs around the main attention kernel (cf_profile_begin / cf_profile_end).
 static std::vector<cudaEvent_t> g_prof_events;
