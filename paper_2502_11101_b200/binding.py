@@ -16,6 +16,7 @@ CF_BF16, CF_F32 = 0, 1
 CF_ROPE_HALF, CF_ROPE_INTERLEAVED = 0, 1
 CF_ALLOC_NONE, CF_ALLOC_ALIGN, CF_ALLOC_SORT = 0, 1, 2
 CF_TILE_TOKENS = 128
+TC_KERNEL_BUILT = True      # bf16 / head_dim 128 batches take the tcgen05 attention kernel
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefocus.so")
 

@@ -1,13 +1,562 @@
-// Placeholder translation unit for the tensor-core attention kernel.
+// Fused re-position + query-prefill attention on the Blackwell tensor cores (bf16, head_dim 128).
+//
+// Eq. 5 fused into Eq. 1: key tiles are streamed from the un-repositioned store by TMA into
+// 128B-swizzled shared memory, every key is rotated by its document's delta in registers and
+// written back in place, QK^T and PV run as tcgen05.mma with fp32 accumulators in tensor memory,
+// the softmax runs one query row per thread out of tensor memory.  The cache is read once.
+//
+// One CTA owns a (request, kv head, group of <=256 query rows, split of the key-tile list) and
+// keeps the running softmax state of its rows; partial results go to the workspace and are merged
+// by the combine kernel.  Warp roles (448 threads):
+//   warps 0-3   softmax of row tile 0 (thread = query row = TMEM lane)
+//   warps 4-7   softmax of row tile 1
+//   warps 8-11  key rotation in shared memory
+//   warp 12     TMA producer (one lane)
+//   warp 13     TMEM allocation and MMA issue (one lane)
+// Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
+// plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
 #include "cf_common.cuh"
 
 namespace cf {
 
-bool attn_tc_supported(const cf_geom*, const cf_batch*) { return false; }
+namespace {
 
-int launch_attn_tc(const cf_geom*, const cf_batch*, const PlanView&, const void*, const void*,
-                   const void*, float, const AttnWorkspace&, cudaStream_t) {
-    return CF_ERR_UNSUPPORTED;
+constexpr int kThreads = 448;
+constexpr int kD = 128;
+constexpr int kHalfBytes = kTile * 128;            // one 64-column half of a 128-row tile, 128 B per row
+constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile, a Q tile or a P tile
+constexpr int kBoxRows = 32;                       // rows per TMA box
+constexpr int kBoxBytes = kBoxRows * 128;
+constexpr int kSmemBytes = 7 * kTileBytes + 1024 + 256;   // 2 Q + 2 P + 3 ring (or 1 Q + 1 P + 5 ring)
+constexpr int kMaxStages = 5;
+constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
+constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference maximum moves only
+                                                   // when a tile exceeds it by more than 2^8
+
+struct Barriers {
+    unsigned long long kv_full[kMaxStages];
+    unsigned long long kv_empty[kMaxStages];
+    unsigned long long k_ready[kMaxStages];
+    unsigned long long s_full[2];
+    unsigned long long s_free[2];
+    unsigned long long p_ready[2];
+    unsigned long long o_done[2];
+    unsigned int tmem_base;
+    volatile int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major; B K-major or MN-major.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane; returns after the data has arrived.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};\n"
+        "tcgen05.wait::st.sync.aligned;"
+        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
+          "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+// Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128B-swizzled half tile.
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+    return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
+}
+
+template <int LAYOUT>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+               BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads, float scale_log2,
+               const __nv_bfloat16* __restrict__ q) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t smem_base = smem_u32(smem);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int group = n_q_heads / n_kv_heads;
+    const int lq = bv.q_len;
+    const int rows = group * lq;
+    const int row_groups = (rows + 255) / 256;
+    const int b = blockIdx.z;
+    const int kvh = blockIdx.y / row_groups;
+    const int rg = blockIdx.y - kvh * row_groups;
+    const int rows_here = min(256, rows - rg * 256);
+    const int n_mt = (rows_here + 127) / 128;                       // row tiles owned by this CTA: 1 or 2
+    const int n_stages = n_mt == 2 ? 3 : 5;
+    const int split = blockIdx.x;
+    const int rows_total = n_q_heads * lq;
+
+    // shared memory map: [Q tiles][P tiles][ring][barriers]
+    const uint32_t q_base = smem_base;
+    const uint32_t p_base = q_base + n_mt * kTileBytes;
+    const uint32_t ring_base = p_base + n_mt * kTileBytes;
+    Barriers* bars = reinterpret_cast<Barriers*>(smem + 7 * kTileBytes);
+    volatile int* abort_flag = &bars->abort_flag;
+
+    const int doc0 = bv.req_doc_begin[b];
+    const int tbase = tile_base(doc0, bv.doc_offsets[doc0]);
+    const int n_tiles = pv.n_tiles[b];
+    const int t_begin = (int)((long long)n_tiles * split / ws.n_splits);
+    const int t_end = (int)((long long)n_tiles * (split + 1) / ws.n_splits);
+    const int n_it = t_end - t_begin;
+    const size_t slot0 = ((size_t)b * ws.n_splits + split) * rows_total + (size_t)kvh * rows + rg * 256;
+
+    if (n_it <= 0) {                                                // empty split: neutral partials
+        for (int r = tid; r < rows_here; r += kThreads) {
+            ws.part_m[slot0 + r] = -INFINITY;
+            ws.part_l[slot0 + r] = 0.f;
+        }
+        for (int i = tid; i < rows_here * (kD / 4); i += kThreads)
+            reinterpret_cast<float4*>(ws.part_o + slot0 * kD)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars->kv_full[s]), 1);
+            mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+            mbar_init(smem_u32(&bars->k_ready[s]), 128);
+        }
+        for (int m = 0; m < 2; ++m) {
+            mbar_init(smem_u32(&bars->s_full[m]), 1);
+            mbar_init(smem_u32(&bars->s_free[m]), 128);
+            mbar_init(smem_u32(&bars->p_ready[m]), 128);
+            mbar_init(smem_u32(&bars->o_done[m]), 1);
+        }
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 13) {                                               // all 512 TMEM columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones)
+    for (int idx = tid; idx < n_mt * 128 * 16; idx += kThreads) {
+        const int chunk = idx & 15, r = idx >> 4;                   // r: row within the CTA's row group
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (r < rows_here) {
+            const int row = rg * 256 + r;
+            const int g = row / lq, j = row - g * lq;
+            const int h = kvh * group + g;
+            val = *reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8);
+        }
+        const int mt = r >> 7, rr = r & 127;
+        unsigned char* dst = smem + (size_t)mt * kTileBytes + (chunk >> 3) * kHalfBytes + swz(rr, chunk & 7);
+        *reinterpret_cast<uint4*>(dst) = val;
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    if (warp == 12) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            for (int u = 0; u < 2 * n_it; ++u) {
+                const int st = u % n_stages;
+                if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
+                const int ti = tbase + t_begin + (u >> 1);
+                const int row0 = pv.tile_row0[ti];
+                const int boxes = (pv.tile_len[ti] + kBoxRows - 1) / kBoxRows;
+                const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
+                const uint32_t bar = smem_u32(&bars->kv_full[st]);
+                const uint32_t dst = ring_base + st * kTileBytes;
+                mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
+                for (int bx = 0; bx < boxes; ++bx) {
+                    tma_load_3d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, bar);
+                    tma_load_3d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, bar);
+                }
+            }
+        }
+    } else if (warp == 13) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            bool ok = true;
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int ti = tbase + t_begin + it;
+                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
+                const int uk = 2 * it, uv = 2 * it + 1;
+                const int stk = uk % n_stages, stv = uv % n_stages;
+                const uint32_t k_buf = ring_base + stk * kTileBytes, v_buf = ring_base + stv * kTileBytes;
+                ok = mbar_wait(smem_u32(&bars->k_ready[stk]), (uk / n_stages) & 1, abort_flag);
+                if (!ok) break;
+                const uint32_t idesc_s = instr_desc(n_keys, false);
+                for (int m = 0; m < n_mt && ok; ++m) {
+                    if (it > 0) ok = mbar_wait(smem_u32(&bars->s_free[m]), (it - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_buf = q_base + m * kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {                // S = Q K'^T, 16 dims per instruction
+                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        umma(tmem + m * 128, smem_desc(a_buf + off, 16, 1024), smem_desc(k_buf + off, 16, 1024),
+                             idesc_s, kk > 0);
+                    }
+                    umma_commit(smem_u32(&bars->s_full[m]));
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&bars->kv_empty[stk]));
+                ok = mbar_wait(smem_u32(&bars->kv_full[stv]), (uv / n_stages) & 1, abort_flag);
+                if (!ok) break;
+                const uint32_t idesc_o = instr_desc(kD, true);
+                for (int m = 0; m < n_mt && ok; ++m) {
+                    ok = mbar_wait(smem_u32(&bars->p_ready[m]), it & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t p_buf = p_base + m * kTileBytes;
+                    for (int kk = 0; kk < n_keys / 16; ++kk) {      // O += P V, 16 keys per instruction
+                        const uint32_t a_off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        umma(tmem + 256 + m * 128, smem_desc(p_buf + a_off, 16, 1024),
+                             smem_desc(v_buf + kk * 2048, kHalfBytes, 1024), idesc_o, (it > 0 || kk > 0));
+                    }
+                    umma_commit(smem_u32(&bars->o_done[m]));
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&bars->kv_empty[stv]));
+            }
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------------ key rotation (Eq. 5)
+        const int t = tid - 256;                                    // 0..127
+        const int chunk = t & 7, rsub = t >> 3;
+        for (int it = 0; it < n_it; ++it) {
+            const int ti = tbase + t_begin + it;
+            const int len = pv.tile_len[ti];
+            const float2* trig = pv.trig + (size_t)pv.tile_doc[ti] * (kD / 2);
+            const int u = 2 * it, st = u % n_stages;
+            float2 cs[8];
+            if (LAYOUT == CF_ROPE_HALF) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) cs[e] = __ldg(trig + chunk * 8 + e);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    cs[e] = __ldg(trig + chunk * 4 + e);            // first half: dims chunk*8 .. +7
+                    cs[4 + e] = __ldg(trig + 32 + chunk * 4 + e);   // second half: dims 64 + chunk*8 ..
+                }
+            }
+            if (!mbar_wait(smem_u32(&bars->kv_full[st]), (u / n_stages) & 1, abort_flag)) break;
+            unsigned char* buf = smem + (ring_base - smem_base) + (size_t)st * kTileBytes;
+#pragma unroll 2
+            for (int r = rsub; r < len; r += 16) {
+                uint4* pa = reinterpret_cast<uint4*>(buf + swz(r, chunk));
+                uint4* pb = reinterpret_cast<uint4*>(buf + kHalfBytes + swz(r, chunk));
+                uint4 va = *pa, vb = *pb;
+                uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wb[4] = {vb.x, vb.y, vb.z, vb.w};
+                if (LAYOUT == CF_ROPE_HALF) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float a0 = __uint_as_float(wa[i] << 16), a1 = __uint_as_float(wa[i] & 0xffff0000u);
+                        float b0 = __uint_as_float(wb[i] << 16), b1 = __uint_as_float(wb[i] & 0xffff0000u);
+                        float ya0, yb0, ya1, yb1;
+                        rotate_pair(a0, b0, cs[2 * i].x, cs[2 * i].y, ya0, yb0);
+                        rotate_pair(a1, b1, cs[2 * i + 1].x, cs[2 * i + 1].y, ya1, yb1);
+                        wa[i] = pack_bf16(ya0, ya1);
+                        wb[i] = pack_bf16(yb0, yb1);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float a0 = __uint_as_float(wa[i] << 16), a1 = __uint_as_float(wa[i] & 0xffff0000u);
+                        float b0 = __uint_as_float(wb[i] << 16), b1 = __uint_as_float(wb[i] & 0xffff0000u);
+                        float ya0, ya1, yb0, yb1;
+                        rotate_pair(a0, a1, cs[i].x, cs[i].y, ya0, ya1);
+                        rotate_pair(b0, b1, cs[4 + i].x, cs[4 + i].y, yb0, yb1);
+                        wa[i] = pack_bf16(ya0, ya1);
+                        wb[i] = pack_bf16(yb0, yb1);
+                    }
+                }
+                *pa = make_uint4(wa[0], wa[1], wa[2], wa[3]);
+                *pb = make_uint4(wb[0], wb[1], wb[2], wb[3]);
+            }
+            fence_proxy_async();
+            mbar_arrive(smem_u32(&bars->k_ready[st]));
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax, one row per thread
+        const int m = warp >> 2;                                    // row tile
+        if (m < n_mt) {
+            const int r = tid & 127;                                // row within the tile = TMEM lane
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+            const uint32_t s_addr = tmem + lane_addr + m * 128;
+            const uint32_t o_addr = tmem + lane_addr + 256 + m * 128;
+            const bool row_valid = m * 128 + r < rows_here;
+            unsigned char* p_buf = smem + (p_base - smem_base) + (size_t)m * kTileBytes;
+            float m_ref = -INFINITY, l_run = 0.f;
+            bool ok = true;
+            for (int it = 0; it < n_it; ++it) {
+                const int ti = tbase + t_begin + it;
+                const int len = pv.tile_len[ti];
+                const int n_chunks = (len + 31) >> 5;
+                ok = mbar_wait(smem_u32(&bars->s_full[m]), it & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                // pass 1: row maximum over the valid keys
+                float mx = -INFINITY;
+                for (int c = 0; c < n_chunks; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c * 32, v);
+                    const int valid = len - c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < valid ? __uint_as_float(v[i]) : -INFINITY);
+                }
+                mx *= scale_log2;
+                float alpha = 1.f;
+                const bool move = mx > m_ref + kRescaleThreshold;   // first tile: m_ref = -inf, always moves
+                if (move) {
+                    alpha = fast_exp2(m_ref - mx);                  // 0 on the first tile
+                    m_ref = mx;
+                }
+                if (it > 0) {
+                    // PV of the previous tile must be complete before P is overwritten or O rescaled
+                    ok = mbar_wait(smem_u32(&bars->o_done[m]), (it - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, move)) {
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t v[32];
+                            tmem_ld32(o_addr + c * 32, v);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                            tmem_st32(o_addr + c * 32, v);
+                        }
+                        l_run *= alpha;
+                    }
+                }
+                // pass 2: p = 2^(s*scale - m_ref), row sum, P tile in bf16 (K-major, 128B swizzle)
+                float tile_sum = 0.f;
+                const float neg_ref = -m_ref;
+                for (int c = 0; c < n_chunks; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c * 32, v);
+                    const int valid = len - c * 32;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = i < valid ? fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref)) : 0.f;
+                        const float p1 = i + 1 < valid ? fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref)) : 0.f;
+                        tile_sum += p0 + p1;
+                        packed[i >> 1] = pack_bf16(p0, p1);
+                    }
+                    unsigned char* half = p_buf + (c >> 1) * kHalfBytes;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(half + swz(r, (c & 1) * 4 + j)) =
+                            make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars->s_free[m]));
+                fence_proxy_async();
+                mbar_arrive(smem_u32(&bars->p_ready[m]));
+                l_run += tile_sum;
+                if (row_valid)
+                    ws.tile_lse2[(size_t)ti * rows_total + (size_t)kvh * rows + rg * 256 + m * 128 + r] =
+                        m_ref + log2f(tile_sum);
+            }
+            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[m]), (n_it - 1) & 1, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                const size_t slot = slot0 + m * 128 + r;
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(o_addr + c * 32, v);
+                    if (row_valid) {
+                        float4* dst = reinterpret_cast<float4*>(ws.part_o + slot * kD + c * 32);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    }
+                }
+                if (row_valid) {
+                    ws.part_m[slot] = m_ref;
+                    ws.part_l[slot] = l_run;
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (bars->abort_flag) {
+        // a wait expired: let loads already in flight land before the shared memory is given back
+        if (warp == 12 && lane == 0) {
+            for (int u = 0; u < 2 * n_it; ++u) {
+                const uint32_t bar = smem_u32(&bars->kv_full[u % n_stages]);
+                const long long t0 = clock64();
+                while (!mbar_try_wait(bar, (u / n_stages) & 1) && clock64() - t0 < kWaitLimitCycles / 16) {}
+            }
+        }
+        if (tid == 0) atomicCAS(pv.status, 0, CF_ERR_TIMEOUT);
+        __syncthreads();
+    }
+    if (warp == 13) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult status;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &status) == cudaSuccess &&
+            status == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+// One layer of the store as a 3-D tensor (head_dim, kv heads, rows); boxes of 64 x 1 x 32.
+int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return CF_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, (cuuint64_t)b->total_tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)b->token_stride * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kBoxRows};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
+}
+
+}  // namespace
+
+bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
+    return g->dtype == CF_BF16 && g->head_dim == 128 && b->total_tokens > 0;
+}
+
+int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q, const void* k,
+                   const void* v, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
+    const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
+    const int row_groups = (rows + 255) / 256;
+    if ((long long)g->n_kv_heads * row_groups > 65535 || b->n_requests > 65535) return CF_ERR_INVALID_ARG;
+    CUtensorMap map_k, map_v;
+    int rc = make_store_map(&map_k, k, g, b);
+    if (rc != CF_OK) return rc;
+    rc = make_store_map(&map_v, v, g, b);
+    if (rc != CF_OK) return rc;
+    dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_groups), (unsigned)b->n_requests);
+    BatchView bv = make_batch_view(b);
+    static bool configured[2] = {false, false};
+    auto run = [&](auto kernel, int which) {
+        if (!configured[which]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+                return CF_ERR_CUDA;
+            configured[which] = true;
+        }
+        kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_k, map_v, bv, pv, ws, g->n_q_heads, g->n_kv_heads,
+                                                       scale_log2, static_cast<const __nv_bfloat16*>(q));
+        return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+    };
+    if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);
+    return run(attn_tc_kernel<CF_ROPE_INTERLEAVED>, 1);
 }
 
 }  // namespace cf

@@ -97,6 +97,41 @@ def test_results_are_bitwise_reproducible():
         assert np.array_equal(a[key], b[key]), key
 
 
+@pytest.mark.parametrize("heads,q_len,lens", [
+    ((4, 4), 16, [128]),                                   # one full tile, one row tile
+    ((4, 4), 16, [40, 128, 7]),                            # ragged tiles
+    ((12, 2), 48, [130, 160, 192, 128, 150]),              # two row tiles (288 rows), two-tile documents
+    ((28, 4), 64, [128, 192, 161, 140, 177, 133]),         # 448 rows: two row groups per kv head
+])
+def test_tensor_core_kernel_matches_cuda_core_kernel(heads, q_len, lens):
+    """Same inputs through both attention kernels of the library."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    cfg = W.WorkloadConfig("tc-vs-simt", 1, heads[0], heads[1], 128, "bf16", 1e6, 32768, len(lens), 1, 400, q_len,
+                           1, 1, ())
+    meta = W.make_meta(cfg, 3, doc_len_override=lens)
+    q, (k, v) = W.make_q(meta).cuda(), [t.cuda() for t in W.make_kv(meta)]
+    results = []
+    try:
+        for path in (1, 0):
+            cf.cf_set_attn_path(path)
+            sess = Session(cfg.n_q_heads, cfg.n_kv_heads, 128, torch.bfloat16, cfg.pos_range, cfg.rope_theta, q_len,
+                           meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=q_len)
+            sess.init()
+            out = torch.full_like(q[0], float("nan"))
+            lse = torch.full((1, cfg.n_q_heads, q_len), float("nan"), device="cuda")
+            sess.attend(q[0], k[0], v[0], out, lse)
+            torch.cuda.synchronize()
+            assert sess.status() == 0
+            results.append((out.float().cpu(), lse.cpu(), sess.doc_scores.cpu()))
+    finally:
+        cf.cf_set_attn_path(0)
+    (o_a, l_a, s_a), (o_b, l_b, s_b) = results
+    assert torch.all((o_a - o_b).abs() <= 1e-2 + 2e-2 * o_a.abs()), float((o_a - o_b).abs().max())
+    assert torch.all((l_a - l_b).abs() <= 1e-3), float((l_a - l_b).abs().max())
+    assert torch.all((s_a - s_b).abs() <= 1e-3 * s_a.abs() + 1e-6)
+
+
 def test_interleaved_slice_layout():
     import paper_2502_11101_b200 as cf
     from paper_2502_11101_b200.session import Session
