@@ -276,7 +276,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 const int uk = 2 * it, uv = 2 * it + 1;
                 const int stk = uk % n_stages, stv = uv % n_stages;
                 const uint32_t k_buf = ring_base + stk * kTileBytes, v_buf = ring_base + stv * kTileBytes;
-                ok = mbar_wait(smem_u32(&bars->k_ready[stk]), (uk / n_stages) & 1, abort_flag);
+                // a stage holds keys once every n_stages tiles (n_stages is odd, keys are the even uses)
+                ok = mbar_wait(smem_u32(&bars->k_ready[stk]), (it / n_stages) & 1, abort_flag);
                 if (!ok) break;
                 const uint32_t idesc_s = instr_desc(n_keys, false);
                 for (int m = 0; m < n_mt && ok; ++m) {
