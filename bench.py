@@ -242,8 +242,12 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
+    if args.layers:
+        cfg = W.scaled_config(cfg, n_layers=args.layers,
+                              schedule=tuple(s for s in cfg.schedule if s[0] <= args.layers))
     rank, world, local = dist_env()
 
     if args.impl == "reference":

@@ -104,6 +104,7 @@ typedef struct cf_plan_layout {
     size_t n_reuse;         /* [n_requests]                                                      */
     size_t query_start;     /* [n_requests]                                                      */
     size_t n_tiles;         /* [n_requests]                                                      */
+    size_t tile_begin;      /* [n_requests] first tile slot of the request (index into tile_*)   */
     size_t doc_tile_begin;  /* [n_docs_total] first tile of the document (index into tile_*)     */
     size_t doc_tile_count;  /* [n_docs_total] 0 if pruned                                        */
     size_t tile_doc;        /* [max_tiles] global document index                                 */

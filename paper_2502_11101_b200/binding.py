@@ -43,7 +43,7 @@ class cf_batch(ctypes.Structure):
 class cf_plan_layout(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("total_bytes", "status", "kept", "kept_count", "dst_start", "group", "n_reuse", "query_start",
-                 "n_tiles", "doc_tile_begin", "doc_tile_count", "tile_doc", "tile_row0", "tile_len", "trig")] + \
+                 "n_tiles", "tile_begin", "doc_tile_begin", "doc_tile_count", "tile_doc", "tile_row0", "tile_len", "trig")] + \
                [("max_tiles", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 

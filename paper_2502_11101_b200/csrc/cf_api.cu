@@ -78,6 +78,7 @@ static void plan_layout(const cf_geom* g, const cf_batch* b, cf_plan_layout* L) 
     L->n_reuse = take(nb, 4);
     L->query_start = take(nb, 4);
     L->n_tiles = take(nb, 4);
+    L->tile_begin = take(nb, 4);
     L->doc_tile_begin = take(nd, 4);
     L->doc_tile_count = take(nd, 4);
     L->tile_doc = take(max_tiles, 4);
@@ -102,6 +103,7 @@ PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan) {
     v.n_reuse = reinterpret_cast<int*>(base + L.n_reuse);
     v.query_start = reinterpret_cast<int*>(base + L.query_start);
     v.n_tiles = reinterpret_cast<int*>(base + L.n_tiles);
+    v.tile_begin = reinterpret_cast<int*>(base + L.tile_begin);
     v.doc_tile_begin = reinterpret_cast<int*>(base + L.doc_tile_begin);
     v.doc_tile_count = reinterpret_cast<int*>(base + L.doc_tile_count);
     v.tile_doc = reinterpret_cast<int*>(base + L.tile_doc);
@@ -130,16 +132,17 @@ int tiles_per_request_bound(const cf_batch* b) {
     return (int)std::min<long long>(t, 1 << 20);
 }
 
-// Splits of the key-tile list per (request, kv head, row group): enough CTAs for every SM,
-// never more splits than tiles.
+// Parts the key-tile list of a request is cut into.  The tensor-core kernel runs one CTA per
+// (request, kv head, group of 256 query rows, pair of parts): enough CTAs for every SM, never more
+// CTAs than tiles.  The count is always even.
 int choose_splits(const cf_geom* g, const cf_batch* b) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_groups = (rows + 255) / 256;
     const long long units = (long long)b->n_requests * g->n_kv_heads * row_groups;
     long long s = (sm_count() + units - 1) / units;
     s = std::min<long long>(s, tiles_per_request_bound(b));
-    s = std::min<long long>(s, CF_MAX_SPLITS);
-    return (int)std::max<long long>(s, 1);
+    s = std::min<long long>(s, CF_MAX_SPLITS / 2);
+    return 2 * (int)std::max<long long>(s, 1);
 }
 
 size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,

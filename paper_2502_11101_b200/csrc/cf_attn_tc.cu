@@ -5,14 +5,18 @@
 // written back in place, QK^T and PV run as tcgen05.mma with fp32 accumulators in tensor memory,
 // the softmax runs one query row per thread out of tensor memory.  The cache is read once.
 //
-// One CTA owns a (request, kv head, group of <=256 query rows, split of the key-tile list) and
-// keeps the running softmax state of its rows; partial results go to the workspace and are merged
-// by the combine kernel.  Warp roles (448 threads):
-//   warps 0-3   softmax of row tile 0 (thread = query row = TMEM lane)
-//   warps 4-7   softmax of row tile 1
+// One CTA owns a (request, kv head, group of <=256 query rows, range of key tiles).  Two softmax
+// warpgroups work side by side, each with its own S and O accumulators in tensor memory:
+//   - with more than 128 query rows in the group, warpgroup w owns row tile w and both see every
+//     key tile of the CTA's range;
+//   - with at most 128 rows, both own the same rows and take alternate key tiles, i.e. the CTA
+//     produces two independent parts of the split-KV decomposition.
+// Partial results (reference maximum, sum, unnormalised O) go to the workspace and are merged by
+// the combine kernel.  Warp roles (512 threads):
+//   warps 0-3   softmax warpgroup 0 (thread = query row = TMEM lane)
+//   warps 4-7   softmax warpgroup 1
 //   warps 8-11  key rotation in shared memory
-//   warp 12     TMA producer (one lane)
-//   warp 13     TMEM allocation and MMA issue (one lane)
+//   warp 12     TMA producer (one lane)      warp 13  TMEM allocation and MMA issue (one lane)
 // Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
 // plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
 #include <cuda.h>
@@ -26,14 +30,15 @@ namespace cf {
 
 namespace {
 
-constexpr int kThreads = 448;
+constexpr int kThreads = 512;
 constexpr int kD = 128;
 constexpr int kHalfBytes = kTile * 128;            // one 64-column half of a 128-row tile, 128 B per row
 constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile, a Q tile or a P tile
 constexpr int kBoxRows = 32;                       // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * 128;
-constexpr int kSmemBytes = 7 * kTileBytes + 1024 + 256;   // 2 Q + 2 P + 3 ring (or 1 Q + 1 P + 5 ring)
-constexpr int kMaxStages = 5;
+constexpr int kSmemTiles = 7;                      // 2 Q + 2 P + 3 ring, or 1 Q + 2 P + 4 ring
+constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 256;
+constexpr int kMaxStages = 4;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
 constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference maximum moves only
                                                    // when a tile exceeds it by more than 2^8
@@ -145,6 +150,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
           "r"(taddr)
         : "memory");
 }
+// 64 consecutive fp32 columns of this thread's TMEM lane; returns after the data has arrived.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&v)[64]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -157,6 +171,45 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128B-swizzled half tile.
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
+}
+
+// p = 2^(s*scale - ref) for 64 key columns held in v (keys at or beyond `valid` give 0), written
+// as one half of a bf16 P tile row (K-major, 128B swizzle); `n_cols` (a multiple of 16) columns
+// are written.  Returns the row sum.  MASKED=false assumes valid >= 64.
+template <bool MASKED>
+__device__ __forceinline__ float exp_and_store(const uint32_t (&v)[64], int valid, int n_cols, float scale_log2,
+                                               float neg_ref, unsigned char* p_half, int r) {
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {                                    // 16-byte chunk = 8 keys
+        if (MASKED && c * 8 >= n_cols) break;
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = c * 8 + 2 * j;
+            float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref));
+            float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref));
+            if (MASKED) {
+                p0 = i < valid ? p0 : 0.f;
+                p1 = i + 1 < valid ? p1 : 0.f;
+            }
+            sum0 += p0;
+            sum1 += p1;
+            w[j] = pack_bf16(p0, p1);
+        }
+        *reinterpret_cast<uint4*>(p_half + swz(r, c)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    return sum0 + sum1;
+}
+template <bool MASKED>
+__device__ __forceinline__ float row_max(const uint32_t (&v)[64], int valid) {
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 64; i += 2) {
+        m0 = fmaxf(m0, (!MASKED || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
+        m1 = fmaxf(m1, (!MASKED || i + 1 < valid) ? __uint_as_float(v[i + 1]) : -INFINITY);
+    }
+    return fmaxf(m0, m1);
 }
 
 template <int LAYOUT>
@@ -178,47 +231,49 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int kvh = blockIdx.y / row_groups;
     const int rg = blockIdx.y - kvh * row_groups;
     const int rows_here = min(256, rows - rg * 256);
-    const int n_mt = (rows_here + 127) / 128;                       // row tiles owned by this CTA: 1 or 2
-    const int n_stages = n_mt == 2 ? 3 : 5;
-    const int split = blockIdx.x;
+    const bool alternate = rows_here <= 128;                        // both warpgroups on the same rows
+    const int n_qt = alternate ? 1 : 2;                             // query tiles in shared memory
+    const int n_stages = alternate ? 4 : 3;
+    const int n_parts = ws.n_splits;                                // parts per request, even
+    const int pair = blockIdx.x;                                    // this CTA fills parts 2*pair, 2*pair+1
     const int rows_total = n_q_heads * lq;
 
-    // shared memory map: [Q tiles][P tiles][ring][barriers]
+    // shared memory map: [Q tiles][2 P tiles][ring][barriers]
     const uint32_t q_base = smem_base;
-    const uint32_t p_base = q_base + n_mt * kTileBytes;
-    const uint32_t ring_base = p_base + n_mt * kTileBytes;
-    Barriers* bars = reinterpret_cast<Barriers*>(smem + 7 * kTileBytes);
+    const uint32_t p_base = q_base + n_qt * kTileBytes;
+    const uint32_t ring_base = p_base + 2 * kTileBytes;
+    Barriers* bars = reinterpret_cast<Barriers*>(smem + kSmemTiles * kTileBytes);
     volatile int* abort_flag = &bars->abort_flag;
 
-    const int doc0 = bv.req_doc_begin[b];
-    const int tbase = tile_base(doc0, bv.doc_offsets[doc0]);
+    const int tbase = pv.tile_begin[b];
     const int n_tiles = pv.n_tiles[b];
-    const int t_begin = (int)((long long)n_tiles * split / ws.n_splits);
-    const int t_end = (int)((long long)n_tiles * (split + 1) / ws.n_splits);
-    const int n_it = t_end - t_begin;
-    const size_t slot0 = ((size_t)b * ws.n_splits + split) * rows_total + (size_t)kvh * rows + rg * 256;
+    const int n_pairs = n_parts >> 1;
+    const int t_begin = (int)((long long)n_tiles * pair / n_pairs);
+    const int t_end = (int)((long long)n_tiles * (pair + 1) / n_pairs);
+    const int n_it = t_end - t_begin;                               // key tiles of this CTA
+    // first workspace row of this CTA in part 2*pair
+    const size_t slot0 = ((size_t)b * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * 256;
 
-    if (n_it <= 0) {                                                // empty split: neutral partials
-        for (int r = tid; r < rows_here; r += kThreads) {
-            ws.part_m[slot0 + r] = -INFINITY;
-            ws.part_l[slot0 + r] = 0.f;
-        }
-        for (int i = tid; i < rows_here * (kD / 4); i += kThreads)
-            reinterpret_cast<float4*>(ws.part_o + slot0 * kD)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        return;
+    // rows that will carry no data in one of the two parts: mark them neutral (m = -inf)
+    for (int r = tid; r < rows_here; r += kThreads) {
+        if (n_it <= 0) ws.part_m[slot0 + r] = -INFINITY;
+        if (n_it <= 0 || !alternate || n_it < 2) ws.part_m[slot0 + rows_total + r] = -INFINITY;
     }
+    if (n_it <= 0) return;
 
     if (tid == 0) {
+        const int rows_t0 = min(rows_here, 128), rows_t1 = alternate ? rows_t0 : rows_here - 128;
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s]), 1);
             mbar_init(smem_u32(&bars->kv_empty[s]), 1);
             mbar_init(smem_u32(&bars->k_ready[s]), 128);
         }
-        for (int m = 0; m < 2; ++m) {
-            mbar_init(smem_u32(&bars->s_full[m]), 1);
-            mbar_init(smem_u32(&bars->s_free[m]), 128);
-            mbar_init(smem_u32(&bars->p_ready[m]), 128);
-            mbar_init(smem_u32(&bars->o_done[m]), 1);
+        for (int w = 0; w < 2; ++w) {
+            const int active = 32 * (((w ? rows_t1 : rows_t0) + 31) / 32);   // threads of warps that own rows
+            mbar_init(smem_u32(&bars->s_full[w]), 1);
+            mbar_init(smem_u32(&bars->s_free[w]), active);
+            mbar_init(smem_u32(&bars->p_ready[w]), active);
+            mbar_init(smem_u32(&bars->o_done[w]), 1);
         }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -227,8 +282,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    __syncthreads();                                                // barriers are initialised
+
+    // the producer starts streaming before the query tile is staged
+    int produced = 0;
+    auto produce = [&](int u) {                                     // u-th ring use: K(u/2) if even, V(u/2) if odd
+        const int st = u % n_stages;
+        const int ti = tbase + t_begin + (u >> 1);
+        const int row0 = pv.tile_row0[ti];
+        const int boxes = (pv.tile_len[ti] + kBoxRows - 1) / kBoxRows;
+        const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
+        const uint32_t bar = smem_u32(&bars->kv_full[st]);
+        const uint32_t dst = ring_base + st * kTileBytes;
+        mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
+        for (int bx = 0; bx < boxes; ++bx) {
+            tma_load_3d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, bar);
+            tma_load_3d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, bar);
+        }
+    };
+    if (warp == 12 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+        for (; produced < min(n_stages, 2 * n_it); ++produced) produce(produced);
+    }
+
     // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones)
-    for (int idx = tid; idx < n_mt * 128 * 16; idx += kThreads) {
+    for (int idx = tid; idx < n_qt * 128 * 16; idx += kThreads) {
         const int chunk = idx & 15, r = idx >> 4;                   // r: row within the CTA's row group
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
         if (r < rows_here) {
@@ -247,71 +326,83 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
-    if (warp == 12) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            for (int u = 0; u < 2 * n_it; ++u) {
+    // Work of warpgroup w: item j uses key tile kt(w, j) and query tile qt(w).
+    //   side by side (two row tiles): kt = j,          n_items = n_it
+    //   alternating  (one row tile):  kt = 2 j + w,    n_items = ceil((n_it - w) / 2)
+    if (warp >= 12) {
+        if (warp == 12 && lane == 0) {
+            // -------------------------------------------------------------- TMA producer
+            for (int u = produced; u < 2 * n_it; ++u) {
                 const int st = u % n_stages;
-                if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
-                const int ti = tbase + t_begin + (u >> 1);
-                const int row0 = pv.tile_row0[ti];
-                const int boxes = (pv.tile_len[ti] + kBoxRows - 1) / kBoxRows;
-                const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
-                const uint32_t bar = smem_u32(&bars->kv_full[st]);
-                const uint32_t dst = ring_base + st * kTileBytes;
-                mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
-                for (int bx = 0; bx < boxes; ++bx) {
-                    tma_load_3d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, bar);
-                    tma_load_3d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, bar);
-                }
+                if (!mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
+                produce(u);
             }
-        }
-    } else if (warp == 13) {
-        // ------------------------------------------------------------------ MMA issue
-        if (lane == 0) {
+        } else if (warp == 13 && lane == 0) {
+            // -------------------------------------------------------------- MMA issue
+            const uint32_t idesc_o = instr_desc(kD, true);
             bool ok = true;
-            for (int it = 0; it < n_it && ok; ++it) {
+            // S of (warpgroup w, key tile it): D = S_w, A = Q tile, B = rotated keys
+            auto issue_s = [&](int w, int it) -> bool {
                 const int ti = tbase + t_begin + it;
                 const int n_keys = (pv.tile_len[ti] + 15) & ~15;
-                const int uk = 2 * it, uv = 2 * it + 1;
-                const int stk = uk % n_stages, stv = uv % n_stages;
-                const uint32_t k_buf = ring_base + stk * kTileBytes, v_buf = ring_base + stv * kTileBytes;
-                // a stage holds keys once every n_stages tiles (n_stages is odd, keys are the even uses)
-                ok = mbar_wait(smem_u32(&bars->k_ready[stk]), (it / n_stages) & 1, abort_flag);
-                if (!ok) break;
+                const int stk = (2 * it) % n_stages;
+                const int kuse = (n_stages & 1) ? it / n_stages : (2 * it) / n_stages;
+                if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
+                const int j = alternate ? (it >> 1) : it;
+                if (j > 0 && !mbar_wait(smem_u32(&bars->s_free[w]), (j - 1) & 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint64_t a0 = smem_desc(q_base + (alternate ? 0 : w) * kTileBytes, 16, 1024);
+                const uint64_t b0 = smem_desc(ring_base + stk * kTileBytes, 16, 1024);
                 const uint32_t idesc_s = instr_desc(n_keys, false);
-                for (int m = 0; m < n_mt && ok; ++m) {
-                    if (it > 0) ok = mbar_wait(smem_u32(&bars->s_free[m]), (it - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t a_buf = q_base + m * kTileBytes;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {                // S = Q K'^T, 16 dims per instruction
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        umma(tmem + m * 128, smem_desc(a_buf + off, 16, 1024), smem_desc(k_buf + off, 16, 1024),
-                             idesc_s, kk > 0);
-                    }
-                    umma_commit(smem_u32(&bars->s_full[m]));
+                for (int kk = 0; kk < 8; ++kk) {                    // 16 dims per instruction
+                    const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+                    umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
-                if (!ok) break;
-                umma_commit(smem_u32(&bars->kv_empty[stk]));
-                ok = mbar_wait(smem_u32(&bars->kv_full[stv]), (uv / n_stages) & 1, abort_flag);
-                if (!ok) break;
-                const uint32_t idesc_o = instr_desc(kD, true);
-                for (int m = 0; m < n_mt && ok; ++m) {
-                    ok = mbar_wait(smem_u32(&bars->p_ready[m]), it & 1, abort_flag);
+                umma_commit(smem_u32(&bars->s_full[w]));
+                return true;
+            };
+            // O_w += P_w V for key tile it
+            auto issue_pv = [&](int w, int it) -> bool {
+                const int ti = tbase + t_begin + it;
+                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
+                const int uv = 2 * it + 1, stv = uv % n_stages;
+                const int j = alternate ? (it >> 1) : it;
+                if (!mbar_wait(smem_u32(&bars->kv_full[stv]), (uv / n_stages) & 1, abort_flag)) return false;
+                if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint64_t a0 = smem_desc(p_base + w * kTileBytes, 16, 1024);
+                const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
+                for (int kk = 0; kk < n_keys / 16; ++kk) {          // 16 keys per instruction
+                    const uint64_t a_off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+                    umma(tmem + 256 + w * 128, a0 + a_off, b0 + (uint64_t)(kk * 128), idesc_o, (j > 0 || kk > 0));
+                }
+                umma_commit(smem_u32(&bars->o_done[w]));
+                return true;
+            };
+            if (!alternate) {
+                for (int it = 0; it < n_it && ok; ++it) {
+                    ok = issue_s(0, it) && issue_s(1, it);
                     if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t p_buf = p_base + m * kTileBytes;
-                    for (int kk = 0; kk < n_keys / 16; ++kk) {      // O += P V, 16 keys per instruction
-                        const uint32_t a_off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        umma(tmem + 256 + m * 128, smem_desc(p_buf + a_off, 16, 1024),
-                             smem_desc(v_buf + kk * 2048, kHalfBytes, 1024), idesc_o, (it > 0 || kk > 0));
-                    }
-                    umma_commit(smem_u32(&bars->o_done[m]));
+                    umma_commit(smem_u32(&bars->kv_empty[(2 * it) % n_stages]));
+                    ok = issue_pv(0, it) && issue_pv(1, it);
+                    if (!ok) break;
+                    umma_commit(smem_u32(&bars->kv_empty[(2 * it + 1) % n_stages]));
                 }
-                if (!ok) break;
-                umma_commit(smem_u32(&bars->kv_empty[stv]));
+            } else {
+                // S(it) is issued one tile ahead of PV(it-1): the two warpgroups overlap
+                for (int it = 0; it <= n_it && ok; ++it) {
+                    if (it < n_it) {
+                        ok = issue_s(it & 1, it);
+                        if (!ok) break;
+                        umma_commit(smem_u32(&bars->kv_empty[(2 * it) % n_stages]));
+                    }
+                    if (it > 0) {
+                        ok = issue_pv((it - 1) & 1, it - 1);
+                        if (!ok) break;
+                        umma_commit(smem_u32(&bars->kv_empty[(2 * it - 1) % n_stages]));
+                    }
+                }
             }
         }
     } else if (warp >= 8) {
@@ -373,98 +464,93 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------------ softmax, one row per thread
-        const int m = warp >> 2;                                    // row tile
-        if (m < n_mt) {
-            const int r = tid & 127;                                // row within the tile = TMEM lane
+        const int w = warp >> 2;                                    // warpgroup
+        const int r = tid & 127;                                    // row within the tile = TMEM lane
+        const int row_in_group = (alternate ? 0 : w * 128) + r;
+        const int n_items = alternate ? (n_it - w + 1) / 2 : n_it;
+        // a warp none of whose rows exist does not take part (the barrier counts exclude it)
+        const bool warp_active = (alternate ? 0 : w * 128) + (warp & 3) * 32 < rows_here;
+        if (warp_active && n_items > 0) {
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t s_addr = tmem + lane_addr + m * 128;
-            const uint32_t o_addr = tmem + lane_addr + 256 + m * 128;
-            const bool row_valid = m * 128 + r < rows_here;
-            unsigned char* p_buf = smem + (p_base - smem_base) + (size_t)m * kTileBytes;
+            const uint32_t s_addr = tmem + lane_addr + w * 128;
+            const uint32_t o_addr = tmem + lane_addr + 256 + w * 128;
+            const bool row_valid = row_in_group < rows_here;
+            unsigned char* p_buf = smem + (p_base - smem_base) + (size_t)w * kTileBytes;
+            const size_t tile_row = (size_t)kvh * rows + rg * 256 + row_in_group;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
-            for (int it = 0; it < n_it; ++it) {
+            for (int j = 0; j < n_items; ++j) {
+                const int it = alternate ? 2 * j + w : j;
                 const int ti = tbase + t_begin + it;
                 const int len = pv.tile_len[ti];
-                const int n_chunks = (len + 31) >> 5;
-                ok = mbar_wait(smem_u32(&bars->s_full[m]), it & 1, abort_flag);
+                ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                // pass 1: row maximum over the valid keys
-                float mx = -INFINITY;
-                for (int c = 0; c < n_chunks; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(s_addr + c * 32, v);
-                    const int valid = len - c * 32;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < valid ? __uint_as_float(v[i]) : -INFINITY);
+                const int n_keys = (len + 15) & ~15;
+                const bool two_halves = len > 64;
+                // row maximum: first half, then second half (whose values stay in registers)
+                uint32_t v[64];
+                tmem_ld64(s_addr, v);
+                float mx = len >= 64 ? row_max<false>(v, 64) : row_max<true>(v, len);
+                if (two_halves) {
+                    tmem_ld64(s_addr + 64, v);
+                    mx = fmaxf(mx, len == kTile ? row_max<false>(v, 64) : row_max<true>(v, len - 64));
                 }
                 mx *= scale_log2;
+                const bool move = mx > m_ref + kRescaleThreshold;   // first item: m_ref = -inf, always moves
                 float alpha = 1.f;
-                const bool move = mx > m_ref + kRescaleThreshold;   // first tile: m_ref = -inf, always moves
                 if (move) {
-                    alpha = fast_exp2(m_ref - mx);                  // 0 on the first tile
+                    alpha = fast_exp2(m_ref - mx);                  // 0 on the first item
                     m_ref = mx;
                 }
-                if (it > 0) {
-                    // PV of the previous tile must be complete before P is overwritten or O rescaled
-                    ok = mbar_wait(smem_u32(&bars->o_done[m]), (it - 1) & 1, abort_flag);
+                if (j > 0) {
+                    // PV of the previous item must be complete before P is overwritten or O rescaled
+                    ok = mbar_wait(smem_u32(&bars->o_done[w]), (j - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    if (__any_sync(0xffffffffu, move)) {
+                    if (__any_sync(0xffffffffu, move)) {            // rare after the first tiles
+                        // (the S values in registers are dropped and read again below)
                         for (int c = 0; c < 4; ++c) {
-                            uint32_t v[32];
-                            tmem_ld32(o_addr + c * 32, v);
+                            uint32_t o[32];
+                            tmem_ld32(o_addr + c * 32, o);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                            tmem_st32(o_addr + c * 32, v);
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(o_addr + c * 32, o);
                         }
                         l_run *= alpha;
+                        if (two_halves) tmem_ld64(s_addr + 64, v);
                     }
                 }
-                // pass 2: p = 2^(s*scale - m_ref), row sum, P tile in bf16 (K-major, 128B swizzle)
                 float tile_sum = 0.f;
-                const float neg_ref = -m_ref;
-                for (int c = 0; c < n_chunks; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(s_addr + c * 32, v);
-                    const int valid = len - c * 32;
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = i < valid ? fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref)) : 0.f;
-                        const float p1 = i + 1 < valid ? fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref)) : 0.f;
-                        tile_sum += p0 + p1;
-                        packed[i >> 1] = pack_bf16(p0, p1);
-                    }
-                    unsigned char* half = p_buf + (c >> 1) * kHalfBytes;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        *reinterpret_cast<uint4*>(half + swz(r, (c & 1) * 4 + j)) =
-                            make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                if (two_halves) {
+                    tile_sum = len == kTile ? exp_and_store<false>(v, 64, 64, scale_log2, -m_ref, p_buf + kHalfBytes, r)
+                                            : exp_and_store<true>(v, len - 64, n_keys - 64, scale_log2, -m_ref,
+                                                                  p_buf + kHalfBytes, r);
+                    tmem_ld64(s_addr, v);
                 }
+                // S is no longer needed in tensor memory: the next QK^T for this warpgroup may start
                 tc_fence_before();
-                mbar_arrive(smem_u32(&bars->s_free[m]));
+                mbar_arrive(smem_u32(&bars->s_free[w]));
+                tile_sum += len >= 64 ? exp_and_store<false>(v, 64, 64, scale_log2, -m_ref, p_buf, r)
+                                      : exp_and_store<true>(v, len, n_keys, scale_log2, -m_ref, p_buf, r);
                 fence_proxy_async();
-                mbar_arrive(smem_u32(&bars->p_ready[m]));
+                mbar_arrive(smem_u32(&bars->p_ready[w]));
                 l_run += tile_sum;
-                if (row_valid)
-                    ws.tile_lse2[(size_t)ti * rows_total + (size_t)kvh * rows + rg * 256 + m * 128 + r] =
-                        m_ref + log2f(tile_sum);
+                if (row_valid) ws.tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
             }
-            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[m]), (n_it - 1) & 1, abort_flag);
+            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (n_items - 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after();
-                const size_t slot = slot0 + m * 128 + r;
+                const size_t slot = slot0 + (alternate ? (size_t)w * rows_total : 0) + row_in_group;
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(o_addr + c * 32, v);
+                    uint32_t o[32];
+                    tmem_ld32(o_addr + c * 32, o);
                     if (row_valid) {
                         float4* dst = reinterpret_cast<float4*>(ws.part_o + slot * kD + c * 32);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_float4(__uint_as_float(o[4 * i]), __uint_as_float(o[4 * i + 1]),
+                                                 __uint_as_float(o[4 * i + 2]), __uint_as_float(o[4 * i + 3]));
                     }
                 }
                 if (row_valid) {
@@ -537,13 +623,14 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                    const void* v, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_groups = (rows + 255) / 256;
-    if ((long long)g->n_kv_heads * row_groups > 65535 || b->n_requests > 65535) return CF_ERR_INVALID_ARG;
+    if ((long long)g->n_kv_heads * row_groups > 65535 || b->n_requests > 65535 || (ws.n_splits & 1))
+        return CF_ERR_INVALID_ARG;
     CUtensorMap map_k, map_v;
     int rc = make_store_map(&map_k, k, g, b);
     if (rc != CF_OK) return rc;
     rc = make_store_map(&map_v, v, g, b);
     if (rc != CF_OK) return rc;
-    dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_groups), (unsigned)b->n_requests);
+    dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups), (unsigned)b->n_requests);
     BatchView bv = make_batch_view(b);
     static bool configured[2] = {false, false};
     auto run = [&](auto kernel, int which) {

@@ -33,6 +33,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
             raise_status(pv.status, CF_ERR_INVALID_ARG);
             pv.kept_count[b] = 0;
             pv.n_tiles[b] = 0;
+            pv.tile_begin[b] = 0;
         }
         return;
     }
@@ -171,6 +172,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
         }
         pv.n_tiles[b] = s_longest < 0 ? 0 : run;
         pv.kept_count[b] = s_longest < 0 ? 0 : n_kept;
+        pv.tile_begin[b] = base;
         pv.n_reuse[b] = windows;
         pv.query_start[b] = query_start;
     }

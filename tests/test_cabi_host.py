@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_sizes_match_the_header(lib):
     assert ctypes.sizeof(cf.cf_geom) == 32
     assert ctypes.sizeof(cf.cf_batch) == 72
-    assert ctypes.sizeof(cf.cf_plan_layout) == 15 * 8 + 8
+    assert ctypes.sizeof(cf.cf_plan_layout) == 16 * 8 + 8
     assert cf.cf_error_string(cf.CF_ERR_RANGE).startswith("kept documents")
 
 
