@@ -3,7 +3,8 @@
 // Eq. 5 fused into Eq. 1: key tiles are streamed from the un-repositioned store by TMA into
 // 128B-swizzled shared memory, every key is rotated by its document's delta in registers and
 // written back in place, QK^T and PV run as tcgen05.mma with fp32 accumulators in tensor memory,
-// the softmax runs one query row per thread out of tensor memory.  The cache is read once.
+// the softmax runs one query row per thread out of tensor memory and hands P back through tensor
+// memory (bf16, aliased onto the upper half of S).  The cache is read once.
 //
 // One CTA owns a (request, kv head, group of <=256 query rows, range of key tiles).  Two softmax
 // warpgroups work side by side, each with its own S and O accumulators in tensor memory:
@@ -13,10 +14,12 @@
 //     produces two independent parts of the split-KV decomposition.
 // Partial results (reference maximum, sum, unnormalised O) go to the workspace and are merged by
 // the combine kernel.  Warp roles (512 threads):
-//   warps 0-3   softmax warpgroup 0 (thread = query row = TMEM lane)
-//   warps 4-7   softmax warpgroup 1
-//   warps 8-11  key rotation in shared memory
-//   warp 12     TMA producer (one lane)      warp 13  TMEM allocation and MMA issue (one lane)
+//   warps 0-3    softmax warpgroup 0 (thread = query row = TMEM lane)
+//   warps 4-7    softmax warpgroup 1
+//   warps 8-11, 14, 15  key rotation in shared memory
+//   warp 12      TMA producer (one lane)     warp 13  TMEM allocation and MMA issue (one lane)
+// The MMA warp interleaves the two warpgroups (PV of one, then the next QK^T of the same one), so
+// one warpgroup's exponentials overlap the other's tensor-core work.
 // Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
 // plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
 #include <cuda.h>
@@ -36,9 +39,10 @@ constexpr int kHalfBytes = kTile * 128;            // one 64-column half of a 12
 constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile, a Q tile or a P tile
 constexpr int kBoxRows = 32;                       // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * 128;
-constexpr int kSmemTiles = 7;                      // 2 Q + 2 P + 3 ring, or 1 Q + 2 P + 4 ring
+constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
 constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 256;
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 6;
+constexpr int kRotateThreads = 192;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
 constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference maximum moves only
                                                    // when a tile exceeds it by more than 2^8
@@ -48,7 +52,6 @@ struct Barriers {
     unsigned long long kv_empty[kMaxStages];
     unsigned long long k_ready[kMaxStages];
     unsigned long long s_full[2];
-    unsigned long long s_free[2];
     unsigned long long p_ready[2];
     unsigned long long o_done[2];
     unsigned int tmem_base;
@@ -119,6 +122,14 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same with the A operand (bf16, two elements per 32-bit column) in tensor memory.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -173,33 +184,37 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
 }
 
-// p = 2^(s*scale - ref) for 64 key columns held in v (keys at or beyond `valid` give 0), written
-// as one half of a bf16 P tile row (K-major, 128B swizzle); `n_cols` (a multiple of 16) columns
-// are written.  Returns the row sum.  MASKED=false assumes valid >= 64.
+// p = 2^(s*scale - ref) for 64 key columns held in v (keys at or beyond `valid` give 0), packed
+// to bf16 pairs in place: v[0..31] become 32 tensor-memory columns of the P operand.  Returns the
+// row sum.  MASKED=false assumes valid >= 64.
 template <bool MASKED>
-__device__ __forceinline__ float exp_and_store(const uint32_t (&v)[64], int valid, int n_cols, float scale_log2,
-                                               float neg_ref, unsigned char* p_half, int r) {
+__device__ __forceinline__ float exp_and_pack(uint32_t (&v)[64], int valid, float scale_log2, float neg_ref) {
     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {                                    // 16-byte chunk = 8 keys
-        if (MASKED && c * 8 >= n_cols) break;
-        uint32_t w[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int i = c * 8 + 2 * j;
-            float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref));
-            float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref));
-            if (MASKED) {
-                p0 = i < valid ? p0 : 0.f;
-                p1 = i + 1 < valid ? p1 : 0.f;
-            }
-            sum0 += p0;
-            sum1 += p1;
-            w[j] = pack_bf16(p0, p1);
+    for (int i = 0; i < 64; i += 2) {
+        float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref));
+        float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref));
+        if (MASKED) {
+            p0 = i < valid ? p0 : 0.f;
+            p1 = i + 1 < valid ? p1 : 0.f;
         }
-        *reinterpret_cast<uint4*>(p_half + swz(r, c)) = make_uint4(w[0], w[1], w[2], w[3]);
+        sum0 += p0;
+        sum1 += p1;
+        v[i >> 1] = pack_bf16(p0, p1);
     }
     return sum0 + sum1;
+}
+__device__ __forceinline__ void tmem_st32_from64(uint32_t taddr, const uint32_t (&v)[64]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
+          "r"(taddr)
+        : "memory");
 }
 template <bool MASKED>
 __device__ __forceinline__ float row_max(const uint32_t (&v)[64], int valid) {
@@ -233,15 +248,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int rows_here = min(256, rows - rg * 256);
     const bool alternate = rows_here <= 128;                        // both warpgroups on the same rows
     const int n_qt = alternate ? 1 : 2;                             // query tiles in shared memory
-    const int n_stages = alternate ? 4 : 3;
+    const int n_stages = kSmemTiles - n_qt;                         // 6 or 5
     const int n_parts = ws.n_splits;                                // parts per request, even
     const int pair = blockIdx.x;                                    // this CTA fills parts 2*pair, 2*pair+1
     const int rows_total = n_q_heads * lq;
 
-    // shared memory map: [Q tiles][2 P tiles][ring][barriers]
+    // shared memory map: [Q tiles][ring][barriers]
     const uint32_t q_base = smem_base;
-    const uint32_t p_base = q_base + n_qt * kTileBytes;
-    const uint32_t ring_base = p_base + 2 * kTileBytes;
+    const uint32_t ring_base = q_base + n_qt * kTileBytes;
     Barriers* bars = reinterpret_cast<Barriers*>(smem + kSmemTiles * kTileBytes);
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -266,12 +280,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s]), 1);
             mbar_init(smem_u32(&bars->kv_empty[s]), 1);
-            mbar_init(smem_u32(&bars->k_ready[s]), 128);
+            mbar_init(smem_u32(&bars->k_ready[s]), kRotateThreads);
         }
         for (int w = 0; w < 2; ++w) {
             const int active = 32 * (((w ? rows_t1 : rows_t0) + 31) / 32);   // threads of warps that own rows
             mbar_init(smem_u32(&bars->s_full[w]), 1);
-            mbar_init(smem_u32(&bars->s_free[w]), active);
             mbar_init(smem_u32(&bars->p_ready[w]), active);
             mbar_init(smem_u32(&bars->o_done[w]), 1);
         }
@@ -306,19 +319,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         for (; produced < min(n_stages, 2 * n_it); ++produced) produce(produced);
     }
 
-    // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones)
-    for (int idx = tid; idx < n_qt * 128 * 16; idx += kThreads) {
-        const int chunk = idx & 15, r = idx >> 4;                   // r: row within the CTA's row group
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (r < rows_here) {
-            const int row = rg * 256 + r;
-            const int g = row / lq, j = row - g * lq;
-            const int h = kvh * group + g;
-            val = *reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8);
+    // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones); all
+    // loads of a thread are issued before the first store so their latencies overlap
+    {
+        uint4 val[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int idx = tid + i * kThreads;
+            const int chunk = idx & 15, r = idx >> 4;               // r: row within the CTA's row group
+            val[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < 4 * n_qt && r < rows_here) {
+                const int row = rg * 256 + r;
+                const int g = row / lq, j = row - g * lq;
+                const int h = kvh * group + g;
+                val[i] = __ldg(reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8));
+            }
         }
-        const int mt = r >> 7, rr = r & 127;
-        unsigned char* dst = smem + (size_t)mt * kTileBytes + (chunk >> 3) * kHalfBytes + swz(rr, chunk & 7);
-        *reinterpret_cast<uint4*>(dst) = val;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int idx = tid + i * kThreads;
+            const int chunk = idx & 15, r = idx >> 4;
+            if (i < 4 * n_qt) {
+                const int mt = r >> 7, rr = r & 127;
+                *reinterpret_cast<uint4*>(smem + (size_t)mt * kTileBytes + (chunk >> 3) * kHalfBytes + swz(rr, chunk & 7)) = val[i];
+            }
+        }
     }
     fence_proxy_async();
     tc_fence_before();
@@ -329,7 +354,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     // Work of warpgroup w: item j uses key tile kt(w, j) and query tile qt(w).
     //   side by side (two row tiles): kt = j,          n_items = n_it
     //   alternating  (one row tile):  kt = 2 j + w,    n_items = ceil((n_it - w) / 2)
-    if (warp >= 12) {
+    if (warp == 12 || warp == 13) {
         if (warp == 12 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
             for (int u = produced; u < 2 * n_it; ++u) {
@@ -339,17 +364,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             }
         } else if (warp == 13 && lane == 0) {
             // -------------------------------------------------------------- MMA issue
+            // Sequence entry n: warpgroup w = n & 1, its item j = n >> 1, key tile = n (alternating)
+            // or j (side by side).  Issue order: S(0) S(1), then PV(n) followed by S(n + 2): the
+            // next QK^T of a warpgroup follows its own PV in the pipe, so S may overwrite the P it aliases.
             const uint32_t idesc_o = instr_desc(kD, true);
-            bool ok = true;
-            // S of (warpgroup w, key tile it): D = S_w, A = Q tile, B = rotated keys
-            auto issue_s = [&](int w, int it) -> bool {
+            const int n_seq = alternate ? n_it : 2 * n_it;
+            auto issue_s = [&](int n) -> bool {
+                const int w = n & 1;
+                const int it = alternate ? n : (n >> 1);
                 const int ti = tbase + t_begin + it;
                 const int n_keys = (pv.tile_len[ti] + 15) & ~15;
                 const int stk = (2 * it) % n_stages;
-                const int kuse = (n_stages & 1) ? it / n_stages : (2 * it) / n_stages;
+                const int kuse = (n_stages & 1) ? it / n_stages : it / (n_stages >> 1);
                 if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
-                const int j = alternate ? (it >> 1) : it;
-                if (j > 0 && !mbar_wait(smem_u32(&bars->s_free[w]), (j - 1) & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t a0 = smem_desc(q_base + (alternate ? 0 : w) * kTileBytes, 16, 1024);
                 const uint64_t b0 = smem_desc(ring_base + stk * kTileBytes, 16, 1024);
@@ -360,54 +387,36 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
                 umma_commit(smem_u32(&bars->s_full[w]));
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
                 return true;
             };
-            // O_w += P_w V for key tile it
-            auto issue_pv = [&](int w, int it) -> bool {
+            auto issue_pv = [&](int n) -> bool {
+                const int w = n & 1, j = n >> 1;
+                const int it = alternate ? n : j;
                 const int ti = tbase + t_begin + it;
                 const int n_keys = (pv.tile_len[ti] + 15) & ~15;
                 const int uv = 2 * it + 1, stv = uv % n_stages;
-                const int j = alternate ? (it >> 1) : it;
                 if (!mbar_wait(smem_u32(&bars->kv_full[stv]), (uv / n_stages) & 1, abort_flag)) return false;
                 if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t a0 = smem_desc(p_base + w * kTileBytes, 16, 1024);
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
-                for (int kk = 0; kk < n_keys / 16; ++kk) {          // 16 keys per instruction
-                    const uint64_t a_off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-                    umma(tmem + 256 + w * 128, a0 + a_off, b0 + (uint64_t)(kk * 128), idesc_o, (j > 0 || kk > 0));
-                }
+                for (int kk = 0; kk < n_keys / 16; ++kk)            // 16 keys = 8 packed columns per instruction
+                    umma_ts(tmem + 256 + w * 128, tmem + w * 128 + 64 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
+                            (j > 0 || kk > 0));
                 umma_commit(smem_u32(&bars->o_done[w]));
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 return true;
             };
-            if (!alternate) {
-                for (int it = 0; it < n_it && ok; ++it) {
-                    ok = issue_s(0, it) && issue_s(1, it);
-                    if (!ok) break;
-                    umma_commit(smem_u32(&bars->kv_empty[(2 * it) % n_stages]));
-                    ok = issue_pv(0, it) && issue_pv(1, it);
-                    if (!ok) break;
-                    umma_commit(smem_u32(&bars->kv_empty[(2 * it + 1) % n_stages]));
-                }
-            } else {
-                // S(it) is issued one tile ahead of PV(it-1): the two warpgroups overlap
-                for (int it = 0; it <= n_it && ok; ++it) {
-                    if (it < n_it) {
-                        ok = issue_s(it & 1, it);
-                        if (!ok) break;
-                        umma_commit(smem_u32(&bars->kv_empty[(2 * it) % n_stages]));
-                    }
-                    if (it > 0) {
-                        ok = issue_pv((it - 1) & 1, it - 1);
-                        if (!ok) break;
-                        umma_commit(smem_u32(&bars->kv_empty[(2 * it - 1) % n_stages]));
-                    }
-                }
+            bool ok = issue_s(0);
+            if (ok && n_seq > 1) ok = issue_s(1);
+            for (int n = 0; n < n_seq && ok; ++n) {
+                ok = issue_pv(n);
+                if (ok && n + 2 < n_seq) ok = issue_s(n + 2);
             }
         }
     } else if (warp >= 8) {
         // ------------------------------------------------------------------ key rotation (Eq. 5)
-        const int t = tid - 256;                                    // 0..127
+        const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
         const int chunk = t & 7, rsub = t >> 3;
         for (int it = 0; it < n_it; ++it) {
             const int ti = tbase + t_begin + it;
@@ -428,7 +437,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             if (!mbar_wait(smem_u32(&bars->kv_full[st]), (u / n_stages) & 1, abort_flag)) break;
             unsigned char* buf = smem + (ring_base - smem_base) + (size_t)st * kTileBytes;
 #pragma unroll 2
-            for (int r = rsub; r < len; r += 16) {
+            for (int r = rsub; r < len; r += kRotateThreads / 8) {
                 uint4* pa = reinterpret_cast<uint4*>(buf + swz(r, chunk));
                 uint4* pb = reinterpret_cast<uint4*>(buf + kHalfBytes + swz(r, chunk));
                 uint4 va = *pa, vb = *pb;
@@ -475,7 +484,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             const uint32_t s_addr = tmem + lane_addr + w * 128;
             const uint32_t o_addr = tmem + lane_addr + 256 + w * 128;
             const bool row_valid = row_in_group < rows_here;
-            unsigned char* p_buf = smem + (p_base - smem_base) + (size_t)w * kTileBytes;
+            const uint32_t p_addr = s_addr + 64;                    // P (bf16 pairs) aliases S columns 64..127
             const size_t tile_row = (size_t)kvh * rows + rg * 256 + row_in_group;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
@@ -486,7 +495,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const int n_keys = (len + 15) & ~15;
                 const bool two_halves = len > 64;
                 // row maximum: first half, then second half (whose values stay in registers)
                 uint32_t v[64];
@@ -509,7 +517,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     if (!ok) break;
                     tc_fence_after();
                     if (__any_sync(0xffffffffu, move)) {            // rare after the first tiles
-                        // (the S values in registers are dropped and read again below)
                         for (int c = 0; c < 4; ++c) {
                             uint32_t o[32];
                             tmem_ld32(o_addr + c * 32, o);
@@ -522,18 +529,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     }
                 }
                 float tile_sum = 0.f;
-                if (two_halves) {
-                    tile_sum = len == kTile ? exp_and_store<false>(v, 64, 64, scale_log2, -m_ref, p_buf + kHalfBytes, r)
-                                            : exp_and_store<true>(v, len - 64, n_keys - 64, scale_log2, -m_ref,
-                                                                  p_buf + kHalfBytes, r);
+                if (two_halves) {                                   // keys 64..127 -> P columns 32..63
+                    tile_sum = len == kTile ? exp_and_pack<false>(v, 64, scale_log2, -m_ref)
+                                            : exp_and_pack<true>(v, len - 64, scale_log2, -m_ref);
+                    tmem_st32_from64(p_addr + 32, v);
                     tmem_ld64(s_addr, v);
                 }
-                // S is no longer needed in tensor memory: the next QK^T for this warpgroup may start
+                tile_sum += len >= 64 ? exp_and_pack<false>(v, 64, scale_log2, -m_ref)
+                                      : exp_and_pack<true>(v, len, scale_log2, -m_ref);
+                tmem_st32_from64(p_addr, v);                        // keys 0..63 -> P columns 0..31
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
-                mbar_arrive(smem_u32(&bars->s_free[w]));
-                tile_sum += len >= 64 ? exp_and_store<false>(v, 64, 64, scale_log2, -m_ref, p_buf, r)
-                                      : exp_and_store<true>(v, len, n_keys, scale_log2, -m_ref, p_buf, r);
-                fence_proxy_async();
                 mbar_arrive(smem_u32(&bars->p_ready[w]));
                 l_run += tile_sum;
                 if (row_valid) ws.tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
