@@ -133,13 +133,22 @@ int tiles_per_request_bound(const cf_batch* b) {
 }
 
 // Parts the key-tile list of a request is cut into.  The tensor-core kernel runs one CTA per
-// (request, kv head, group of 256 query rows, pair of parts): enough CTAs for every SM, never more
-// CTAs than tiles.  The count is always even.
+// (request, kv head, group of 256 query rows, pair of parts): as many CTAs as fit one wave over the
+// SMs, never more CTAs than tiles.  The count is always even.
 int choose_splits(const cf_geom* g, const cf_batch* b) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_groups = (rows + 255) / 256;
     const long long units = (long long)b->n_requests * g->n_kv_heads * row_groups;
-    long long s = (sm_count() + units - 1) / units;
+    const long long sms = sm_count();
+    long long s = sms / units;                        // whole CTAs per SM: one wave, no ragged second wave
+    if (s == 0) {                                     // more units than SMs: balance the waves instead
+        double best = 0.0;
+        for (long long c = 1; c <= 4; ++c) {
+            const long long ctas = units * c, waves = (ctas + sms - 1) / sms;
+            const double eff = (double)ctas / (double)(waves * sms);
+            if (eff > best + 0.03) { best = eff; s = c; }
+        }
+    }
     s = std::min<long long>(s, tiles_per_request_bound(b));
     s = std::min<long long>(s, CF_MAX_SPLITS / 2);
     return 2 * (int)std::max<long long>(s, 1);

@@ -161,14 +161,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
           "r"(taddr)
         : "memory");
 }
-// 64 consecutive fp32 columns of this thread's TMEM lane; returns after the data has arrived.
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&v)[64]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
-        : "r"(taddr)
-        : "memory");
+// Asynchronous 32-column load: the registers may only be used after tmem_ld_wait(v).
+__device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr)
+                 : "memory");
+}
+// Waits for all outstanding tensor-memory loads of this thread; naming the registers keeps the
+// compiler from moving their uses above the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31]) : : "memory");
+}
+// 16 columns (32 packed bf16) of the P operand; completion is awaited once per tile.
+__device__ __forceinline__ void tmem_st16_async(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+                 : : "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(taddr)
+                 : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -184,14 +193,24 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
 }
 
-// p = 2^(s*scale - ref) for 64 key columns held in v (keys at or beyond `valid` give 0), packed
-// to bf16 pairs in place: v[0..31] become 32 tensor-memory columns of the P operand.  Returns the
-// row sum.  MASKED=false assumes valid >= 64.
+// Maximum of the first `valid` of 32 logits (MASKED=false: all 32).
 template <bool MASKED>
-__device__ __forceinline__ float exp_and_pack(uint32_t (&v)[64], int valid, float scale_log2, float neg_ref) {
+__device__ __forceinline__ float chunk_max(const uint32_t (&v)[32], int valid) {
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        m0 = fmaxf(m0, (!MASKED || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
+        m1 = fmaxf(m1, (!MASKED || i + 1 < valid) ? __uint_as_float(v[i + 1]) : -INFINITY);
+    }
+    return fmaxf(m0, m1);
+}
+// p = 2^(s*scale - ref) for 32 key columns (keys at or beyond `valid` give 0), packed in place to
+// bf16 pairs: v[0..15] become 16 tensor-memory columns of the P operand.  Returns the row sum.
+template <bool MASKED>
+__device__ __forceinline__ float chunk_exp(uint32_t (&v)[32], int valid, float scale_log2, float neg_ref) {
     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < 64; i += 2) {
+    for (int i = 0; i < 32; i += 2) {
         float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref));
         float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref));
         if (MASKED) {
@@ -203,28 +222,6 @@ __device__ __forceinline__ float exp_and_pack(uint32_t (&v)[64], int valid, floa
         v[i >> 1] = pack_bf16(p0, p1);
     }
     return sum0 + sum1;
-}
-__device__ __forceinline__ void tmem_st32_from64(uint32_t taddr, const uint32_t (&v)[64]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
-          "r"(taddr)
-        : "memory");
-}
-template <bool MASKED>
-__device__ __forceinline__ float row_max(const uint32_t (&v)[64], int valid) {
-    float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < 64; i += 2) {
-        m0 = fmaxf(m0, (!MASKED || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
-        m1 = fmaxf(m1, (!MASKED || i + 1 < valid) ? __uint_as_float(v[i + 1]) : -INFINITY);
-    }
-    return fmaxf(m0, m1);
 }
 
 template <int LAYOUT>
@@ -316,7 +313,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     if (warp == 12 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
-        for (; produced < min(n_stages, 2 * n_it); ++produced) produce(produced);
+        for (; produced < 2; ++produced) produce(produced);        // first key and value tile; the rest follow below
     }
 
     // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones); all
@@ -359,7 +356,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             // -------------------------------------------------------------- TMA producer
             for (int u = produced; u < 2 * n_it; ++u) {
                 const int st = u % n_stages;
-                if (!mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
+                if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
                 produce(u);
             }
         } else if (warp == 13 && lane == 0) {
@@ -401,7 +398,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 tc_fence_after();
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
                 for (int kk = 0; kk < n_keys / 16; ++kk)            // 16 keys = 8 packed columns per instruction
-                    umma_ts(tmem + 256 + w * 128, tmem + w * 128 + 64 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
+                    umma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
                             (j > 0 || kk > 0));
                 umma_commit(smem_u32(&bars->o_done[w]));
                 if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
@@ -484,7 +481,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             const uint32_t s_addr = tmem + lane_addr + w * 128;
             const uint32_t o_addr = tmem + lane_addr + 256 + w * 128;
             const bool row_valid = row_in_group < rows_here;
-            const uint32_t p_addr = s_addr + 64;                    // P (bf16 pairs) aliases S columns 64..127
             const size_t tile_row = (size_t)kvh * rows + rg * 256 + row_in_group;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
@@ -495,14 +491,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const bool two_halves = len > 64;
-                // row maximum: first half, then second half (whose values stay in registers)
-                uint32_t v[64];
-                tmem_ld64(s_addr, v);
-                float mx = len >= 64 ? row_max<false>(v, 64) : row_max<true>(v, len);
-                if (two_halves) {
-                    tmem_ld64(s_addr + 64, v);
-                    mx = fmaxf(mx, len == kTile ? row_max<false>(v, 64) : row_max<true>(v, len - 64));
+                const int n_chunks = (len + 31) >> 5;               // 32 keys per chunk, loads double-buffered
+                uint32_t va[32], vb[32];
+                // pass 1: row maximum
+                float mx = -INFINITY;
+                tmem_ld32_async(s_addr, va);
+                tmem_ld_wait(va);
+                for (int c = 0; c < n_chunks; c += 2) {
+                    if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
+                    mx = fmaxf(mx, len - c * 32 >= 32 ? chunk_max<false>(va, 32) : chunk_max<true>(va, len - c * 32));
+                    if (c + 1 < n_chunks) {
+                        tmem_ld_wait(vb);
+                        if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
+                        mx = fmaxf(mx, len - c * 32 >= 64 ? chunk_max<false>(vb, 32) : chunk_max<true>(vb, len - c * 32 - 32));
+                        if (c + 2 < n_chunks) tmem_ld_wait(va);
+                    }
                 }
                 mx *= scale_log2;
                 const bool move = mx > m_ref + kRescaleThreshold;   // first item: m_ref = -inf, always moves
@@ -511,33 +514,42 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     alpha = fast_exp2(m_ref - mx);                  // 0 on the first item
                     m_ref = mx;
                 }
+                tmem_ld32_async(s_addr, va);                        // first chunk of pass 2, in flight during the checks
                 if (j > 0) {
-                    // PV of the previous item must be complete before P is overwritten or O rescaled
+                    // PV of the previous item must be complete before O is rescaled (and it has read P)
                     ok = mbar_wait(smem_u32(&bars->o_done[w]), (j - 1) & 1, abort_flag);
-                    if (!ok) break;
+                    if (!ok) { tmem_ld_wait(va); break; }
                     tc_fence_after();
                     if (__any_sync(0xffffffffu, move)) {            // rare after the first tiles
+                        tmem_ld_wait(va);
                         for (int c = 0; c < 4; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(o_addr + c * 32, o);
+                            tmem_ld32(o_addr + c * 32, vb);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                            tmem_st32(o_addr + c * 32, o);
+                            for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
+                            tmem_st32(o_addr + c * 32, vb);
                         }
                         l_run *= alpha;
-                        if (two_halves) tmem_ld64(s_addr + 64, v);
                     }
                 }
+                // pass 2: exponentials; P chunk c (16 packed columns) lands in S columns 16c..16c+15,
+                // which belong to S chunks already held in registers
                 float tile_sum = 0.f;
-                if (two_halves) {                                   // keys 64..127 -> P columns 32..63
-                    tile_sum = len == kTile ? exp_and_pack<false>(v, 64, scale_log2, -m_ref)
-                                            : exp_and_pack<true>(v, len - 64, scale_log2, -m_ref);
-                    tmem_st32_from64(p_addr + 32, v);
-                    tmem_ld64(s_addr, v);
+                const float neg_ref = -m_ref;
+                tmem_ld_wait(va);
+                for (int c = 0; c < n_chunks; c += 2) {
+                    if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
+                    tile_sum += len - c * 32 >= 32 ? chunk_exp<false>(va, 32, scale_log2, neg_ref)
+                                                   : chunk_exp<true>(va, len - c * 32, scale_log2, neg_ref);
+                    tmem_st16_async(s_addr + c * 16, va);
+                    if (c + 1 < n_chunks) {
+                        tmem_ld_wait(vb);
+                        if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
+                        tile_sum += len - c * 32 >= 64 ? chunk_exp<false>(vb, 32, scale_log2, neg_ref)
+                                                       : chunk_exp<true>(vb, len - c * 32 - 32, scale_log2, neg_ref);
+                        tmem_st16_async(s_addr + (c + 1) * 16, vb);
+                        if (c + 2 < n_chunks) tmem_ld_wait(va);
+                    }
                 }
-                tile_sum += len >= 64 ? exp_and_pack<false>(v, 64, scale_log2, -m_ref)
-                                      : exp_and_pack<true>(v, len, scale_log2, -m_ref);
-                tmem_st32_from64(p_addr, v);                        // keys 0..63 -> P columns 0..31
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars->p_ready[w]));
