@@ -324,13 +324,23 @@ def main():
     value = tokens_all * args.steps / (ms_max * 1e-3)
 
     # ---- the dominant kernel alone: event pairs around every attention-kernel launch ----------
+    # Launches are issued eagerly here; a spin kernel queued first keeps the GPU busy until the host
+    # has enqueued the whole step, so the event pairs time kernels running back to back and not the
+    # host's launch latency.
     prof_steps = max(1, min(args.steps, 20))
+    host_s = []
     for i in range(3):
+        torch.cuda.synchronize()
+        t_host = time.perf_counter()
         wl.step(i)
+        host_s.append(time.perf_counter() - t_host)
     torch.cuda.synchronize()
+    spin_cycles = int(max(host_s) * 1.5 * 2.0e9)
     cf.cf_profile_begin(prof_steps * cfg.n_layers)
     for i in range(prof_steps):
+        torch.cuda._sleep(spin_cycles)
         wl.step(3 + i)
+        torch.cuda.synchronize()
     durations = cf.cf_profile_end(prof_steps * cfg.n_layers).astype(np.float64)
     kv_bytes_per_token = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4) * cfg.n_kv_heads
     flops_per_token = 4 * cfg.group_size * cfg.q_len * cfg.head_dim * cfg.n_kv_heads

@@ -178,6 +178,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->tile_lse2 = reinterpret_cast<float*>(base + t);
         ws->row_lse2 = reinterpret_cast<float*>(base + r);
         ws->n_splits = n_splits;
+        ws->part_bf16 = 0;
     }
     return off;
 }
@@ -398,9 +399,10 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool timed = g_prof_used < g_prof_capacity;
     if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
-    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch))
+    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch)) {
+        ws.part_bf16 = 1;
         rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    else
+    } else
         rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
     if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);
     if (rc != CF_OK) return rc;

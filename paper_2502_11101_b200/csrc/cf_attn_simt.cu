@@ -150,41 +150,67 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
     }
 }
 
-// Merge the splits of one query row (one warp per row): out = sum_s w_s O_s / sum_s w_s l_s with
-// w_s = 2^(m_s - max m), and the row's log-sum-exp.
-template <typename T, int D>
-__global__ void __launch_bounds__(256)
-combine_kernel(AttnWorkspace ws, int n_requests, int n_q_heads, int lq, T* __restrict__ out,
-               float* __restrict__ lse) {
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
+// Merge the parts of one query row (one block per row, one thread per output dimension):
+// out = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m), and the row's log-sum-exp.
+// Parts are visited in index order, so the result does not depend on scheduling.
+template <typename T, int D, typename P>
+__global__ void __launch_bounds__(D)
+combine_kernel(AttnWorkspace ws, int n_q_heads, int lq, T* __restrict__ out, float* __restrict__ lse) {
+    __shared__ float s_w[CF_MAX_SPLITS];
+    __shared__ float s_red[2][D / 32];
     const int rows_total = n_q_heads * lq;
-    if (warp >= n_requests * rows_total) return;
-    const int b = warp / rows_total, rg = warp - b * rows_total;
+    const int b = blockIdx.x / rows_total, rg = blockIdx.x - b * rows_total;
     const int h = rg / lq, j = rg - h * lq;
-    float m_max = -INFINITY;
-    for (int s = 0; s < ws.n_splits; ++s)
-        m_max = fmaxf(m_max, ws.part_m[((size_t)b * ws.n_splits + s) * rows_total + rg]);
-    float acc[D / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_parts = ws.n_splits;
+    const size_t slot0 = (size_t)b * n_parts * rows_total + rg;       // part p sits at slot0 + p * rows_total
+
+    float m = -INFINITY, l = 0.f;
+    if (tid < n_parts) {
+        m = ws.part_m[slot0 + (size_t)tid * rows_total];
+        l = m > -INFINITY ? ws.part_l[slot0 + (size_t)tid * rows_total] : 0.f;
+    }
+    float m_max = m;
 #pragma unroll
-    for (int k = 0; k < D / 32; ++k) acc[k] = 0.f;
-    float l_sum = 0.f;
-    if (m_max > -INFINITY) {
-        for (int s = 0; s < ws.n_splits; ++s) {
-            const size_t slot = ((size_t)b * ws.n_splits + s) * rows_total + rg;
-            const float ms = ws.part_m[slot];
-            if (ms == -INFINITY) continue;
-            const float w = exp2f(ms - m_max);
-            l_sum = fmaf(ws.part_l[slot], w, l_sum);
+    for (int o = 16; o > 0; o >>= 1) m_max = fmaxf(m_max, __shfl_xor_sync(0xffffffffu, m_max, o));
+    if (lane == 0) s_red[0][warp] = m_max;
+    __syncthreads();
+    m_max = s_red[0][0];
 #pragma unroll
-            for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(ws.part_o[slot * D + lane + 32 * k], w, acc[k]);
-        }
+    for (int k = 1; k < D / 32; ++k) m_max = fmaxf(m_max, s_red[0][k]);
+    const float w = m > -INFINITY ? exp2f(m - m_max) : 0.f;
+    if (tid < n_parts) s_w[tid] = w;
+    float l_sum = l * w;                                               // fixed-shape tree: deterministic
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l_sum += __shfl_xor_sync(0xffffffffu, l_sum, o);
+    if (lane == 0) s_red[1][warp] = l_sum;
+    __syncthreads();
+    l_sum = s_red[1][0];
+#pragma unroll
+    for (int k = 1; k < D / 32; ++k) l_sum += s_red[1][k];
+
+    float acc = 0.f;
+    const P* po = reinterpret_cast<const P*>(ws.part_o) + slot0 * D + tid;
+    const size_t stride = (size_t)rows_total * D;
+    int p = 0;
+    for (; p + 4 <= n_parts; p += 4) {                                 // independent loads in flight
+        const float w0 = s_w[p], w1 = s_w[p + 1], w2 = s_w[p + 2], w3 = s_w[p + 3];
+        const float o0 = w0 > 0.f ? to_float(po[(size_t)p * stride]) : 0.f;
+        const float o1 = w1 > 0.f ? to_float(po[(size_t)(p + 1) * stride]) : 0.f;
+        const float o2 = w2 > 0.f ? to_float(po[(size_t)(p + 2) * stride]) : 0.f;
+        const float o3 = w3 > 0.f ? to_float(po[(size_t)(p + 3) * stride]) : 0.f;
+        acc = fmaf(o0, w0, acc);
+        acc = fmaf(o1, w1, acc);
+        acc = fmaf(o2, w2, acc);
+        acc = fmaf(o3, w3, acc);
+    }
+    for (; p < n_parts; ++p) {
+        const float wp = s_w[p];
+        if (wp > 0.f) acc = fmaf(to_float(po[(size_t)p * stride]), wp, acc);
     }
     const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-    T* dst = out + (((size_t)b * lq + j) * n_q_heads + h) * D;
-#pragma unroll
-    for (int k = 0; k < D / 32; ++k) dst[lane + 32 * k] = from_float<T>(acc[k] * inv);
-    if (lane == 0) {
+    out[(((size_t)b * lq + j) * n_q_heads + h) * D + tid] = from_float<T>(acc * inv);
+    if (tid == 0) {
         const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
         ws.row_lse2[(size_t)b * rows_total + rg] = lse2;
         if (lse) lse[(size_t)b * rows_total + rg] = lse2 * kLn2;
@@ -268,10 +294,12 @@ int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, co
 template <typename T, int D>
 static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const AttnWorkspace& ws, void* out,
                                 float* lse, cudaStream_t stream) {
-    const long long warps = (long long)b->n_requests * g->n_q_heads * b->q_len;
-    const long long blocks = (warps + 7) / 8;
-    combine_kernel<T, D><<<(unsigned)blocks, 256, 0, stream>>>(ws, b->n_requests, g->n_q_heads, b->q_len,
-                                                            static_cast<T*>(out), lse);
+    const long long blocks = (long long)b->n_requests * g->n_q_heads * b->q_len;
+    if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS || ws.n_splits > D) return CF_ERR_INVALID_ARG;
+    if (ws.part_bf16)
+        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+    else
+        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 

@@ -560,15 +560,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             if (ok) {
                 tc_fence_after();
                 const size_t slot = slot0 + (alternate ? (size_t)w * rows_total : 0) + row_in_group;
+                // Partial O rows leave as bf16 through shared memory so that global stores are full
+                // 256-byte rows.  Staging space: this warpgroup's own query tile (every QK^T that read
+                // it has completed), or, when both warpgroups share one query tile, the ring stage of
+                // the next unused key or value slot (its last reader completed before this point).
+                unsigned char* stage = alternate ? smem + (ring_base - smem_base) + (size_t)((2 * n_it + w) % n_stages) * kTileBytes
+                                                 : smem + (size_t)w * kTileBytes;
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
                     tmem_ld32(o_addr + c * 32, o);
-                    if (row_valid) {
-                        float4* dst = reinterpret_cast<float4*>(ws.part_o + slot * kD + c * 32);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            dst[i] = make_float4(__uint_as_float(o[4 * i]), __uint_as_float(o[4 * i + 1]),
-                                                 __uint_as_float(o[4 * i + 2]), __uint_as_float(o[4 * i + 3]));
+                    for (int i = 0; i < 4; ++i) {                   // 8 dims = one 16-byte chunk
+                        const int chunk = c * 4 + i;
+                        *reinterpret_cast<uint4*>(stage + r * 256 + ((chunk ^ (r & 15)) << 4)) =
+                            make_uint4(pack_bf16(__uint_as_float(o[8 * i]), __uint_as_float(o[8 * i + 1])),
+                                       pack_bf16(__uint_as_float(o[8 * i + 2]), __uint_as_float(o[8 * i + 3])),
+                                       pack_bf16(__uint_as_float(o[8 * i + 4]), __uint_as_float(o[8 * i + 5])),
+                                       pack_bf16(__uint_as_float(o[8 * i + 6]), __uint_as_float(o[8 * i + 7])));
+                    }
+                }
+                __syncwarp();
+                {
+                    const int warp_row0 = r & ~31;                  // this warp's 32 rows
+                    const int rows_left = rows_here - ((alternate ? 0 : w * 128) + warp_row0);
+                    unsigned char* dst = reinterpret_cast<unsigned char*>(ws.part_o) + (slot - lane) * (size_t)(kD * 2);
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {                  // two rows per step, 16 lanes each
+                        const int rr = 2 * i + (lane >> 4), chunk = lane & 15;
+                        if (rr < rows_left) {
+                            const int srow = warp_row0 + rr;
+                            const uint4 val = *reinterpret_cast<const uint4*>(stage + srow * 256 + ((chunk ^ (srow & 15)) << 4));
+                            *reinterpret_cast<uint4*>(dst + (size_t)rr * (kD * 2) + chunk * 16) = val;
+                        }
                     }
                 }
                 if (row_valid) {

@@ -64,12 +64,14 @@ int tiles_per_request_bound(const cf_batch* b);
 // Partial results of the attention kernels, one slice per split, merged by the combine kernel.
 // All logits are in base-2 units: t = (q.k) * softmax_scale * log2(e).
 struct AttnWorkspace {
-    float* part_o;     // [B][n_splits][Hq*Lq][D]   sum_t 2^(t - m) v_t, not normalised (unset if m = -inf)
+    float* part_o;     // [B][n_splits][Hq*Lq][D]   sum_t 2^(t - m) v_t, not normalised (unset if m = -inf);
+                       //                           fp32, or bf16 in the same index order when part_bf16 is set
     float* part_m;     // [B][n_splits][Hq*Lq]      reference maximum m (-inf if the part is empty)
     float* part_l;     // [B][n_splits][Hq*Lq]      sum_t 2^(t - m)
     float* tile_lse2;  // [max_tiles][Hq*Lq]        log2 of sum over the tile's tokens of 2^t
     float* row_lse2;   // [B][Hq*Lq]                log2 of the full softmax denominator
     int n_splits;
+    int part_bf16;     // the tensor-core kernel stores its partial O rows as bf16
 };
 size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,
                              void* base);

@@ -60,9 +60,10 @@ extern "C" int cf_query_prefill_attn_static(const cf_geom* geom, const cf_batch*
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (attn_path() == 0 && attn_tc_supported(geom, batch))
+    if (attn_path() == 0 && attn_tc_supported(geom, batch)) {
+        ws.part_bf16 = 1;
         rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    else
+    } else
         rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
     if (rc != CF_OK) return rc;
     return launch_combine(geom, batch, pv, ws, out, lse, doc_scores, score_accum, s);
