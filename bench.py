@@ -184,6 +184,42 @@ def time_steps(fn, steps, warmup, world):
     return start.elapsed_time(stop), t0, t1
 
 
+def reposition_roofline(device, peaks, layers=8, iters=5):
+    """Standalone cf_reposition_keys (Algorithm 2, Phase 2) over a store shaped like the largest
+    configuration (32 kv heads, 8 requests x 120 documents of 160-200 tokens): every key row of
+    `layers` layers is rotated in place.  Bytes = one read and one write of the key store."""
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=layers)
+    meta = W.make_meta(cfg, 0)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len,
+                   device=device)
+    k = torch.empty((layers, meta.total_tokens, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device=device)
+    v_scratch = torch.empty_like(k[0])
+    for layer in range(layers):
+        W.fill_kv_layer(meta, layer, k[layer], v_scratch)
+    del v_scratch
+    sess.set_live_docs(cfg.n_docs)
+    sess.init()
+    for _ in range(3):
+        sess.reposition(k, k, layers, k.stride(0))
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(iters):
+        sess.reposition(k, k, layers, k.stride(0))
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / iters
+    nbytes = 2 * k.numel() * k.element_size()
+    gbs = nbytes / ms / 1e6
+    assert sess.status() == 0
+    return {"kernel": "cf_reposition_keys", "workload": f"configs[4]-shaped key store, {layers} of 32 layers, in place",
+            "bound": "hbm", "bytes_per_launch": nbytes, "ms_per_launch": ms, "achieved": gbs, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "frac_of_8tbs_nominal": gbs / 8000.0,
+            "peak_source": peaks["source"]}
+
+
 def oracle_sample(cfg, seed):
     """The oracle, as it stands, on one request of the workload (all layers, pruning schedule)."""
     import oracle
@@ -242,6 +278,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
@@ -393,6 +430,16 @@ def main():
             dist.destroy_process_group()
         return
 
+    attn_kernel = "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05"
+    launches = wl.launches_per_step() * args.steps
+    slot_mb = sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6
+    launch_mode = "cuda graph per ring slot" if graphs is not None else "eager"
+    repo = None
+    if world == 1 and not args.skip_reposition:
+        del wl, graphs, host, q0, k0, v0
+        torch.cuda.empty_cache()
+        repo = reposition_roofline(device, peaks)
+
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
         t_total, tok_total, reps = 0.0, 0, 0
@@ -414,12 +461,12 @@ def main():
                        "schedule": [list(s) for s in cfg.schedule], "strategy": "align",
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
-                             f"{sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6:.0f} MB) cycled between steps",
-                       "launch": "cuda graph per ring slot" if graphs is not None else "eager",
-                       "attention_kernel": "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05",
+                             f"{slot_mb:.0f} MB) cycled between steps",
+                       "launch": launch_mode,
+                       "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": wl.launches_per_step() * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu}
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "reposition": repo, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
