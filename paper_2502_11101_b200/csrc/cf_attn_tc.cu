@@ -519,8 +519,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             int i = 0;                                              // sub-items done by this warpgroup
             bool ok = true;
 
-            // One 32-key chunk: lazy reference update (rare, warp-uniform), exponentials, packing.
-            auto process = [&](uint32_t (&v)[32], int valid, uint32_t s_addr, int chunk) -> bool {
+            // One 32-key chunk, step 1: lazy reference update (rare, warp-uniform).  No tensor-memory
+            // load may be in flight here: the branches below would let the compiler move registers
+            // that the hardware has not written yet.
+            auto prepare = [&](const uint32_t (&v)[32], int valid, uint32_t s_addr, int chunk) -> bool {
                 const float cmax = (valid >= 32 ? chunk_max<false>(v, 32) : chunk_max<true>(v, valid)) * scale_log2;
                 const bool move = cmax > m_ref + kRescaleThreshold; // very first chunk: m_ref = -inf, always moves
                 if (__any_sync(0xffffffffu, move)) {
@@ -552,9 +554,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     l_run *= alpha;
                     tile_sum *= alpha;
                 }
+                return true;
+            };
+            // Step 2 (straight-line): exponentials, packing, P store.
+            auto finish = [&](uint32_t (&v)[32], int valid, uint32_t s_addr, int chunk) {
                 tile_sum += valid >= 32 ? chunk_exp<false>(v, 32, scale_log2, -m_ref) : chunk_exp<true>(v, valid, scale_log2, -m_ref);
                 tmem_st16_async(s_addr + chunk * 16, v);            // P columns land on S columns already consumed
-                return true;
             };
 
             for (int it = first_it; it < n_it && ok; it += it_step) {
@@ -570,13 +575,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     uint32_t va[32], vb[32];
                     tmem_ld32_async(s_addr, va);
                     tmem_ld_wait(va);
-                    if (keys > 32) tmem_ld32_async(s_addr + 32, vb);
-                    ok = process(va, keys, s_addr, 0);
+                    ok = prepare(va, keys, s_addr, 0);
+                    if (!ok) break;
+                    if (keys > 32) tmem_ld32_async(s_addr + 32, vb);    // in flight during the exponentials of chunk 0
+                    finish(va, keys, s_addr, 0);
                     if (keys > 32) {
                         tmem_ld_wait(vb);
-                        if (ok) ok = process(vb, keys - 32, s_addr, 1);
+                        ok = prepare(vb, keys - 32, s_addr, 1);
+                        if (!ok) break;
+                        finish(vb, keys - 32, s_addr, 1);
                     }
-                    if (!ok) break;
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     tc_fence_before();
                     mbar_arrive(smem_u32(&bars->p_ready[w][buf]));
