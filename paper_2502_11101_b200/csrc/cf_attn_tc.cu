@@ -43,7 +43,7 @@ constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile
 constexpr int kBoxRows = 32;                       // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * 128;
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
-constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 256;
+constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512;   // tiles, alignment slack, barriers
 constexpr int kMaxStages = 6;
 constexpr int kRotateThreads = 192;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
@@ -51,15 +51,21 @@ constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference 
                                                    // when a tile exceeds it by more than 2^8
 
 struct Barriers {
-    unsigned long long kv_full[kMaxStages];
+    // A parity wait is only meaningful for a waiter that has seen every earlier phase of the barrier,
+    // so every barrier here has one kind of waiter that waits for each of its phases in order: the
+    // key loads and the value loads of a ring stage complete on separate barriers (the rotation warps
+    // wait for keys, the MMA warp for values), and PV completion alternates between two barriers.
+    unsigned long long kv_full[kMaxStages][2];   // [stage][0 = keys, 1 = values]
     unsigned long long kv_empty[kMaxStages];
     unsigned long long k_ready[kMaxStages];
     unsigned long long s_full[2][2];      // [warpgroup][S buffer]
     unsigned long long p_ready[2][2];
-    unsigned long long o_done[2];
+    unsigned long long o_done[2][2];      // [warpgroup][sub-item parity]
     unsigned int tmem_base;
     volatile int abort_flag;
 };
+
+static_assert(sizeof(Barriers) <= 512, "barrier block must fit its reserved shared memory");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -284,7 +290,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     if (tid == 0) {
         const int rows_t0 = min(rows_here, 128), rows_t1 = alternate ? rows_t0 : rows_here - 128;
         for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(smem_u32(&bars->kv_full[s]), 1);
+            mbar_init(smem_u32(&bars->kv_full[s][0]), 1);
+            mbar_init(smem_u32(&bars->kv_full[s][1]), 1);
             mbar_init(smem_u32(&bars->kv_empty[s]), 1);
             mbar_init(smem_u32(&bars->k_ready[s]), kRotateThreads);
         }
@@ -294,7 +301,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 mbar_init(smem_u32(&bars->s_full[w][buf]), 1);
                 mbar_init(smem_u32(&bars->p_ready[w][buf]), active);
             }
-            mbar_init(smem_u32(&bars->o_done[w]), 1);
+            mbar_init(smem_u32(&bars->o_done[w][0]), 1);
+            mbar_init(smem_u32(&bars->o_done[w][1]), 1);
         }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -313,7 +321,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const int row0 = pv.tile_row0[ti];
         const int boxes = (pv.tile_len[ti] + kBoxRows - 1) / kBoxRows;
         const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
-        const uint32_t bar = smem_u32(&bars->kv_full[st]);
+        const uint32_t bar = smem_u32(&bars->kv_full[st][u & 1]);
         const uint32_t dst = ring_base + st * kTileBytes;
         mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
         for (int bx = 0; bx < boxes; ++bx) {
@@ -410,14 +418,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 const int keys = sub == 0 ? min(len, 64) : len - 64;
                 const bool last_sub = sub == 1 || len <= 64;
                 const int uv = 2 * it + 1, stv = uv % n_stages;
-                if (!mbar_wait(smem_u32(&bars->kv_full[stv]), (uv / n_stages) & 1, abort_flag)) return false;
+                const int vuse = (n_stages & 1) ? it / n_stages : uv / n_stages;   // value loads this stage has seen
+                if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
                 if (!mbar_wait(smem_u32(&bars->p_ready[w][buf]), (i >> 1) & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes + sub * (64 * 128), kHalfBytes, 1024);
                 for (int kk = 0; kk < ((keys + 15) >> 4); ++kk)     // 16 keys = 8 packed P columns per instruction
                     umma_ts(tmem + w * 256 + 128, tmem + w * 256 + buf * 64 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
                             (i > 0 || kk > 0));
-                umma_commit(smem_u32(&bars->o_done[w]));
+                umma_commit(smem_u32(&bars->o_done[w][i & 1]));
                 if (last_sub && (alternate || w == 1)) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 if (last_sub) { p_it[w] += step; p_sub[w] = 0; } else p_sub[w] = 1;
                 ++p_idx[w];
@@ -464,7 +473,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                     cs[4 + e] = __ldg(trig + 32 + chunk * 4 + e);   // second half: dims 64 + chunk*8 ..
                 }
             }
-            if (!mbar_wait(smem_u32(&bars->kv_full[st]), (u / n_stages) & 1, abort_flag)) break;
+            const int kuse = (n_stages & 1) ? it / n_stages : u / n_stages;      // key loads this stage has seen
+            if (!mbar_wait(smem_u32(&bars->kv_full[st][0]), kuse & 1, abort_flag)) break;
             unsigned char* buf = smem + (ring_base - smem_base) + (size_t)st * kTileBytes;
 #pragma unroll 2
             for (int r = rsub; r < len; r += kRotateThreads / 8) {
@@ -532,7 +542,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                         m_ref = cmax;
                     }
                     if (i > 0) {                                    // O holds earlier sub-items: their PV must be complete
-                        if (!mbar_wait(smem_u32(&bars->o_done[w]), (i - 1) & 1, abort_flag)) return false;
+                        // PV(i-1); PV(i-3), the previous phase of that barrier, completed before S(i) was issued
+                        if (!mbar_wait(smem_u32(&bars->o_done[w][(i - 1) & 1]), ((i - 1) >> 1) & 1, abort_flag)) return false;
                         tc_fence_after();
                         for (int c = 0; c < 8; ++c) {
                             uint32_t o[16];
@@ -594,7 +605,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 if (row_valid) ws.tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
                 tile_sum = 0.f;
             }
-            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (i - 1) & 1, abort_flag);
+            // the last PV (the pipe is in order, so every earlier one is complete as well)
+            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w][(i - 1) & 1]), ((i - 1) >> 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after();
                 const size_t slot = slot0 + (alternate ? (size_t)w * rows_total : 0) + row_in_group;
@@ -647,9 +659,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         // a wait expired: let loads already in flight land before the shared memory is given back
         if (warp == 12 && lane == 0) {
             for (int u = 0; u < 2 * n_it; ++u) {
-                const uint32_t bar = smem_u32(&bars->kv_full[u % n_stages]);
+                const int use = (n_stages & 1) ? (u >> 1) / n_stages : u / n_stages;
+                const uint32_t bar = smem_u32(&bars->kv_full[u % n_stages][u & 1]);
                 const long long t0 = clock64();
-                while (!mbar_try_wait(bar, (u / n_stages) & 1) && clock64() - t0 < kWaitLimitCycles / 16) {}
+                while (!mbar_try_wait(bar, use & 1) && clock64() - t0 < kWaitLimitCycles / 16) {}
             }
         }
         if (tid == 0) atomicCAS(pv.status, 0, CF_ERR_TIMEOUT);
