@@ -4,11 +4,10 @@
 // 128B-swizzled shared memory, every key is rotated by its document's delta in registers and
 // written back in place, QK^T and PV run as tcgen05.mma with fp32 accumulators in tensor memory,
 // the softmax runs one query row per thread out of tensor memory and hands P back through tensor
-// memory (bf16, aliased onto S columns already consumed).  The cache is read once.
+// memory (bf16, aliased onto the upper half of S).  The cache is read once.
 //
-// One CTA owns a (request, kv head, group of <=256 query rows, range of key tiles).  Keys are
-// consumed in sub-tiles of 64: each of the two softmax warpgroups has two S buffers (so the next
-// QK^T runs while it exponentiates the current one) and one O accumulator in tensor memory:
+// One CTA owns a (request, kv head, group of <=256 query rows, range of key tiles).  Two softmax
+// warpgroups work side by side, each with its own S and O accumulators in tensor memory:
 //   - with more than 128 query rows in the group, warpgroup w owns row tile w and both see every
 //     key tile of the CTA's range;
 //   - with at most 128 rows, both own the same rows and take alternate key tiles, i.e. the CTA
@@ -19,10 +18,8 @@
 //   warps 4-7    softmax warpgroup 1
 //   warps 8-11, 14, 15  key rotation in shared memory
 //   warp 12      TMA producer (one lane)     warp 13  TMEM allocation and MMA issue (one lane)
-// The softmax is single-pass: the reference maximum of a row only moves when a 32-key chunk
-// exceeds it by more than 2^8, in which case O, the sums and the P columns already written are
-// rescaled (rare after the first chunk); any reference within the exponent range is exact enough
-// because P (bf16) and the sums (fp32) keep their relative precision.
+// The MMA warp interleaves the two warpgroups (PV of one, then the next QK^T of the same one), so
+// one warpgroup's exponentials overlap the other's tensor-core work.
 // Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
 // plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
 #include <cuda.h>
@@ -51,16 +48,15 @@ constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference 
                                                    // when a tile exceeds it by more than 2^8
 
 struct Barriers {
-    // A parity wait is only meaningful for a waiter that has seen every earlier phase of the barrier,
-    // so every barrier here has one kind of waiter that waits for each of its phases in order: the
-    // key loads and the value loads of a ring stage complete on separate barriers (the rotation warps
-    // wait for keys, the MMA warp for values), and PV completion alternates between two barriers.
+    // A parity wait is only meaningful for a waiter that has seen every earlier phase of the barrier.
+    // Key loads and value loads of a ring stage therefore complete on separate barriers: the rotation
+    // warps wait for every key load, the MMA warp for every value load.
     unsigned long long kv_full[kMaxStages][2];   // [stage][0 = keys, 1 = values]
     unsigned long long kv_empty[kMaxStages];
     unsigned long long k_ready[kMaxStages];
-    unsigned long long s_full[2][2];      // [warpgroup][S buffer]
-    unsigned long long p_ready[2][2];
-    unsigned long long o_done[2][2];      // [warpgroup][sub-item parity]
+    unsigned long long s_full[2];
+    unsigned long long p_ready[2];
+    unsigned long long o_done[2];
     unsigned int tmem_base;
     volatile int abort_flag;
 };
@@ -157,6 +153,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};\n"
+        "tcgen05.wait::st.sync.aligned;"
+        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
+          "r"(taddr)
+        : "memory");
+}
 // Asynchronous 32-column load: the registers may only be used after tmem_ld_wait(v).
 __device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -169,26 +178,7 @@ __device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31]) : : "memory");
 }
-// 16 columns, synchronous (used on the rare rescaling path).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};\n"
-        "tcgen05.wait::st.sync.aligned;"
-        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(taddr)
-        : "memory");
-}
-// 16 columns (32 packed bf16) of the P operand; completion is awaited once per sub-tile.
+// 16 columns (32 packed bf16) of the P operand; completion is awaited once per tile.
 __device__ __forceinline__ void tmem_st16_async(uint32_t taddr, const uint32_t (&v)[32]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
                  : : "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(taddr)
@@ -297,12 +287,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         }
         for (int w = 0; w < 2; ++w) {
             const int active = 32 * (((w ? rows_t1 : rows_t0) + 31) / 32);   // threads of warps that own rows
-            for (int buf = 0; buf < 2; ++buf) {
-                mbar_init(smem_u32(&bars->s_full[w][buf]), 1);
-                mbar_init(smem_u32(&bars->p_ready[w][buf]), active);
-            }
-            mbar_init(smem_u32(&bars->o_done[w][0]), 1);
-            mbar_init(smem_u32(&bars->o_done[w][1]), 1);
+            mbar_init(smem_u32(&bars->s_full[w]), 1);
+            mbar_init(smem_u32(&bars->p_ready[w]), active);
+            mbar_init(smem_u32(&bars->o_done[w]), 1);
         }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -380,77 +367,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             }
         } else if (warp == 13 && lane == 0) {
             // -------------------------------------------------------------- MMA issue
-            // Each warpgroup consumes a stream of sub-items (key tile, 64-key half).  Per stream the
-            // QK^T of sub-item i+2 follows the PV of sub-item i in the pipe (it reuses that S buffer,
-            // whose lower columns hold P(i): the tensor pipe runs them in issue order), so up to two
-            // QK^T results are ahead of the softmax.  The two streams are interleaved.
+            // Sequence entry n: warpgroup w = n & 1, its item j = n >> 1, key tile = n (alternating)
+            // or j (side by side).  Issue order: S(0) S(1), then PV(n) followed by S(n + 2): the
+            // next QK^T of a warpgroup follows its own PV in the pipe, so S may overwrite the P it aliases.
             const uint32_t idesc_o = instr_desc(kD, true);
-            const int step = alternate ? 2 : 1;
-            int s_it[2] = {0, alternate ? 1 : 0}, s_sub[2] = {0, 0}, s_idx[2] = {0, 0};   // next QK^T per stream
-            int p_it[2] = {0, alternate ? 1 : 0}, p_sub[2] = {0, 0}, p_idx[2] = {0, 0};   // next PV per stream
-            bool ok = true;
-            auto issue_s = [&](int w) -> bool {
-                const int it = s_it[w], sub = s_sub[w], buf = s_idx[w] & 1;
-                const int len = pv.tile_len[tbase + t_begin + it];
-                const int keys = sub == 0 ? min(len, 64) : len - 64;
-                const bool last_sub = sub == 1 || len <= 64;
+            const int n_seq = alternate ? n_it : 2 * n_it;
+            auto issue_s = [&](int n) -> bool {
+                const int w = n & 1;
+                const int it = alternate ? n : (n >> 1);
+                const int ti = tbase + t_begin + it;
+                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
                 const int stk = (2 * it) % n_stages;
                 const int kuse = (n_stages & 1) ? it / n_stages : it / (n_stages >> 1);
                 if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t a0 = smem_desc(q_base + (alternate ? 0 : w) * kTileBytes, 16, 1024);
-                const uint64_t b0 = smem_desc(ring_base + stk * kTileBytes + sub * (64 * 128), 16, 1024);
-                const uint32_t idesc_s = instr_desc((keys + 15) & ~15, false);
+                const uint64_t b0 = smem_desc(ring_base + stk * kTileBytes, 16, 1024);
+                const uint32_t idesc_s = instr_desc(n_keys, false);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {                    // 16 dims per instruction
                     const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-                    umma(tmem + w * 256 + buf * 64, a0 + off, b0 + off, idesc_s, kk > 0);
+                    umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
-                umma_commit(smem_u32(&bars->s_full[w][buf]));
-                if (last_sub && (alternate || w == 1)) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
-                if (last_sub) { s_it[w] += step; s_sub[w] = 0; } else s_sub[w] = 1;
-                ++s_idx[w];
+                umma_commit(smem_u32(&bars->s_full[w]));
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
                 return true;
             };
-            auto issue_pv = [&](int w) -> bool {
-                const int it = p_it[w], sub = p_sub[w], i = p_idx[w], buf = i & 1;
-                const int len = pv.tile_len[tbase + t_begin + it];
-                const int keys = sub == 0 ? min(len, 64) : len - 64;
-                const bool last_sub = sub == 1 || len <= 64;
+            auto issue_pv = [&](int n) -> bool {
+                const int w = n & 1, j = n >> 1;
+                const int it = alternate ? n : j;
+                const int ti = tbase + t_begin + it;
+                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
                 const int uv = 2 * it + 1, stv = uv % n_stages;
                 const int vuse = (n_stages & 1) ? it / n_stages : uv / n_stages;   // value loads this stage has seen
                 if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
-                if (!mbar_wait(smem_u32(&bars->p_ready[w][buf]), (i >> 1) & 1, abort_flag)) return false;
+                if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes + sub * (64 * 128), kHalfBytes, 1024);
-                for (int kk = 0; kk < ((keys + 15) >> 4); ++kk)     // 16 keys = 8 packed P columns per instruction
-                    umma_ts(tmem + w * 256 + 128, tmem + w * 256 + buf * 64 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
-                            (i > 0 || kk > 0));
-                umma_commit(smem_u32(&bars->o_done[w][i & 1]));
-                if (last_sub && (alternate || w == 1)) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
-                if (last_sub) { p_it[w] += step; p_sub[w] = 0; } else p_sub[w] = 1;
-                ++p_idx[w];
+                const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
+                for (int kk = 0; kk < n_keys / 16; ++kk)            // 16 keys = 8 packed columns per instruction
+                    umma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
+                            (j > 0 || kk > 0));
+                umma_commit(smem_u32(&bars->o_done[w]));
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 return true;
             };
-            // Scheduling: always serve the stream whose pending PV is on the earliest key tile, and let
-            // QK^T run at most two sub-items ahead of a stream's PV and at most two key tiles ahead of
-            // the oldest tile still in use (what the ring can hold) -- one in-order issuer must never
-            // wait for a tile whose ring slot depends on work it has not issued yet.
-            constexpr int kBig = 0x3fffffff;
-            auto top_up = [&]() -> bool {
-                const int oldest = min(p_it[0] < n_it ? p_it[0] : kBig, p_it[1] < n_it ? p_it[1] : kBig);
-                for (int w = 0; w < 2; ++w)
-                    while (s_idx[w] < p_idx[w] + 2 && s_it[w] < n_it && s_it[w] <= oldest + 2)
-                        if (!issue_s(w)) return false;
-                return true;
-            };
-            ok = top_up();
-            while (ok && (p_it[0] < n_it || p_it[1] < n_it)) {
-                const int t0 = p_it[0] < n_it ? p_it[0] : kBig, t1 = p_it[1] < n_it ? p_it[1] : kBig;
-                const int w = (t1 < t0 || (t1 == t0 && p_idx[1] < p_idx[0])) ? 1 : 0;
-                if (s_idx[w] <= p_idx[w]) ok = issue_s(w);          // its own QK^T was held back by the window
-                if (ok) ok = issue_pv(w);
-                if (ok) ok = top_up();
+            bool ok = issue_s(0);
+            if (ok && n_seq > 1) ok = issue_s(1);
+            for (int n = 0; n < n_seq && ok; ++n) {
+                ok = issue_pv(n);
+                if (ok && n + 2 < n_seq) ok = issue_s(n + 2);
             }
         }
     } else if (warp >= 8) {
@@ -516,97 +481,90 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const int w = warp >> 2;                                    // warpgroup
         const int r = tid & 127;                                    // row within the tile = TMEM lane
         const int row_in_group = (alternate ? 0 : w * 128) + r;
-        const int first_it = alternate ? w : 0, it_step = alternate ? 2 : 1;
+        const int n_items = alternate ? (n_it - w + 1) / 2 : n_it;
         // a warp none of whose rows exist does not take part (the barrier counts exclude it)
         const bool warp_active = (alternate ? 0 : w * 128) + (warp & 3) * 32 < rows_here;
-        if (warp_active && first_it < n_it) {
+        if (warp_active && n_items > 0) {
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t wg_addr = tmem + lane_addr + w * 256;    // S buffers at +0 and +64, O at +128
-            const uint32_t o_addr = wg_addr + 128;
+            const uint32_t s_addr = tmem + lane_addr + w * 128;
+            const uint32_t o_addr = tmem + lane_addr + 256 + w * 128;
             const bool row_valid = row_in_group < rows_here;
             const size_t tile_row = (size_t)kvh * rows + rg * 256 + row_in_group;
-            float m_ref = -INFINITY, l_run = 0.f, tile_sum = 0.f;
-            int i = 0;                                              // sub-items done by this warpgroup
+            float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
-
-            // One 32-key chunk, step 1: lazy reference update (rare, warp-uniform).  No tensor-memory
-            // load may be in flight here: the branches below would let the compiler move registers
-            // that the hardware has not written yet.
-            auto prepare = [&](const uint32_t (&v)[32], int valid, uint32_t s_addr, int chunk) -> bool {
-                const float cmax = (valid >= 32 ? chunk_max<false>(v, 32) : chunk_max<true>(v, valid)) * scale_log2;
-                const bool move = cmax > m_ref + kRescaleThreshold; // very first chunk: m_ref = -inf, always moves
-                if (__any_sync(0xffffffffu, move)) {
-                    float alpha = 1.f;
-                    if (move) {
-                        alpha = fast_exp2(m_ref - cmax);            // 0 when nothing has been accumulated yet
-                        m_ref = cmax;
-                    }
-                    if (i > 0) {                                    // O holds earlier sub-items: their PV must be complete
-                        // PV(i-1); PV(i-3), the previous phase of that barrier, completed before S(i) was issued
-                        if (!mbar_wait(smem_u32(&bars->o_done[w][(i - 1) & 1]), ((i - 1) >> 1) & 1, abort_flag)) return false;
-                        tc_fence_after();
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t o[16];
-                            tmem_ld16(o_addr + c * 16, o);
-#pragma unroll
-                            for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                            tmem_st16(o_addr + c * 16, o);
-                        }
-                    }
-                    if (chunk == 1) {                               // P of the first chunk of this sub-item
-                        uint32_t pk[16];
-                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");   // its store is still in flight
-                        tmem_ld16(s_addr, pk);
-#pragma unroll
-                        for (int k = 0; k < 16; ++k)
-                            pk[k] = pack_bf16(__uint_as_float(pk[k] << 16) * alpha, __uint_as_float(pk[k] & 0xffff0000u) * alpha);
-                        tmem_st16(s_addr, pk);
-                    }
-                    l_run *= alpha;
-                    tile_sum *= alpha;
-                }
-                return true;
-            };
-            // Step 2 (straight-line): exponentials, packing, P store.
-            auto finish = [&](uint32_t (&v)[32], int valid, uint32_t s_addr, int chunk) {
-                tile_sum += valid >= 32 ? chunk_exp<false>(v, 32, scale_log2, -m_ref) : chunk_exp<true>(v, valid, scale_log2, -m_ref);
-                tmem_st16_async(s_addr + chunk * 16, v);            // P columns land on S columns already consumed
-            };
-
-            for (int it = first_it; it < n_it && ok; it += it_step) {
+            for (int j = 0; j < n_items; ++j) {
+                const int it = alternate ? 2 * j + w : j;
                 const int ti = tbase + t_begin + it;
                 const int len = pv.tile_len[ti];
-                for (int sub = 0; sub * 64 < len && ok; ++sub, ++i) {
-                    const int keys = min(len - sub * 64, 64);
-                    const int buf = i & 1;
-                    const uint32_t s_addr = wg_addr + buf * 64;
-                    ok = mbar_wait(smem_u32(&bars->s_full[w][buf]), (i >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    uint32_t va[32], vb[32];
-                    tmem_ld32_async(s_addr, va);
-                    tmem_ld_wait(va);
-                    ok = prepare(va, keys, s_addr, 0);
-                    if (!ok) break;
-                    if (keys > 32) tmem_ld32_async(s_addr + 32, vb);    // in flight during the exponentials of chunk 0
-                    finish(va, keys, s_addr, 0);
-                    if (keys > 32) {
-                        tmem_ld_wait(vb);
-                        ok = prepare(vb, keys - 32, s_addr, 1);
-                        if (!ok) break;
-                        finish(vb, keys - 32, s_addr, 1);
-                    }
-                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(&bars->p_ready[w][buf]));
-                }
+                ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
+                tc_fence_after();
+                const int n_chunks = (len + 31) >> 5;               // 32 keys per chunk, loads double-buffered
+                uint32_t va[32], vb[32];
+                // pass 1: row maximum
+                float mx = -INFINITY;
+                tmem_ld32_async(s_addr, va);
+                tmem_ld_wait(va);
+                for (int c = 0; c < n_chunks; c += 2) {
+                    if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
+                    mx = fmaxf(mx, len - c * 32 >= 32 ? chunk_max<false>(va, 32) : chunk_max<true>(va, len - c * 32));
+                    if (c + 1 < n_chunks) {
+                        tmem_ld_wait(vb);
+                        if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
+                        mx = fmaxf(mx, len - c * 32 >= 64 ? chunk_max<false>(vb, 32) : chunk_max<true>(vb, len - c * 32 - 32));
+                        if (c + 2 < n_chunks) tmem_ld_wait(va);
+                    }
+                }
+                mx *= scale_log2;
+                const bool move = mx > m_ref + kRescaleThreshold;   // first item: m_ref = -inf, always moves
+                float alpha = 1.f;
+                if (move) {
+                    alpha = fast_exp2(m_ref - mx);                  // 0 on the first item
+                    m_ref = mx;
+                }
+                tmem_ld32_async(s_addr, va);                        // first chunk of pass 2, in flight during the checks
+                if (j > 0) {
+                    // PV of the previous item must be complete before O is rescaled (and it has read P)
+                    ok = mbar_wait(smem_u32(&bars->o_done[w]), (j - 1) & 1, abort_flag);
+                    if (!ok) { tmem_ld_wait(va); break; }
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, move)) {            // rare after the first tiles
+                        tmem_ld_wait(va);
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(o_addr + c * 32, vb);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
+                            tmem_st32(o_addr + c * 32, vb);
+                        }
+                        l_run *= alpha;
+                    }
+                }
+                // pass 2: exponentials; P chunk c (16 packed columns) lands in S columns 16c..16c+15,
+                // which belong to S chunks already held in registers
+                float tile_sum = 0.f;
+                const float neg_ref = -m_ref;
+                tmem_ld_wait(va);
+                for (int c = 0; c < n_chunks; c += 2) {
+                    if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
+                    tile_sum += len - c * 32 >= 32 ? chunk_exp<false>(va, 32, scale_log2, neg_ref)
+                                                   : chunk_exp<true>(va, len - c * 32, scale_log2, neg_ref);
+                    tmem_st16_async(s_addr + c * 16, va);
+                    if (c + 1 < n_chunks) {
+                        tmem_ld_wait(vb);
+                        if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
+                        tile_sum += len - c * 32 >= 64 ? chunk_exp<false>(vb, 32, scale_log2, neg_ref)
+                                                       : chunk_exp<true>(vb, len - c * 32 - 32, scale_log2, neg_ref);
+                        tmem_st16_async(s_addr + (c + 1) * 16, vb);
+                        if (c + 2 < n_chunks) tmem_ld_wait(va);
+                    }
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars->p_ready[w]));
                 l_run += tile_sum;
                 if (row_valid) ws.tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
-                tile_sum = 0.f;
             }
-            // the last PV (the pipe is in order, so every earlier one is complete as well)
-            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w][(i - 1) & 1]), ((i - 1) >> 1) & 1, abort_flag);
+            if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (n_items - 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after();
                 const size_t slot = slot0 + (alternate ? (size_t)w * rows_total : 0) + row_in_group;
