@@ -220,6 +220,22 @@ def reposition_roofline(device, peaks, layers=8, iters=5):
             "peak_source": peaks["source"]}
 
 
+def whole_job(ms, tokens_per_step, steps, world, device):
+    """Whole-job numbers of a replica run: every rank processed `tokens_per_step` tokens per step in `ms`
+    milliseconds for `steps` steps; the job's time is the slowest rank's, its work the sum over ranks.
+    Returns (ms_max, tokens_all_per_step, tokens_per_second)."""
+    stats = torch.tensor([ms, float(tokens_per_step)], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        mx, sm = stats.clone(), stats.clone()
+        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms_max, tokens_all = float(mx[0]), float(sm[1])
+    else:
+        ms_max, tokens_all = float(ms), float(tokens_per_step)
+    return ms_max, tokens_all, tokens_all * steps / (ms_max * 1e-3)
+
+
 def oracle_sample(cfg, seed):
     """The oracle, as it stands, on one request of the workload (all layers, pruning schedule)."""
     import oracle
@@ -349,16 +365,7 @@ def main():
     clocks = sampler.stop(t0, t1) if sampler else None
     assert wl.sess.status() == 0
 
-    stats = torch.tensor([ms, float(tokens_per_step)], dtype=torch.float64, device=device)
-    if world > 1:
-        mx = stats.clone()
-        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = stats.clone()
-        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        ms_max, tokens_all = float(mx[0]), float(sm[1])
-    else:
-        ms_max, tokens_all = ms, float(tokens_per_step)
-    value = tokens_all * args.steps / (ms_max * 1e-3)
+    ms_max, tokens_all, value = whole_job(ms, tokens_per_step, args.steps, world, device)
 
     # ---- the dominant kernel alone: event pairs around every attention-kernel launch ----------
     # Launches are issued eagerly here; a spin kernel queued first keeps the GPU busy until the host
@@ -417,12 +424,10 @@ def main():
 
     e2e_steps = max(1, min(args.steps, 20))
     e2e_ms, _, _ = time_steps(e2e_step, e2e_steps, 3, world)
-    e2e_stats = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(e2e_stats, op=dist.ReduceOp.MAX)
+    e2e_ms_max, _, e2e_value = whole_job(e2e_ms, tokens_per_step, e2e_steps, world, device)
     h2d = sum(t.numel() * t.element_size() for t in host)
     d2h = sum(t.numel() * t.element_size() for t in (out_h, acc_h, kept_h))
-    e2e = {"value": tokens_all * e2e_steps / (float(e2e_stats[0]) * 1e-3), "unit": UNIT,
+    e2e = {"value": e2e_value, "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
     if rank != 0:

@@ -1,0 +1,93 @@
+"""Full-size runs in the launch configuration bench.py times (Session.run_stack), checked on sampled
+outputs the oracle computes one by one and on properties that hold at any size.
+
+Nothing the oracle consumes comes from the CUDA path: layer 1 attends every document in retrieval
+order, so its allocation and outputs are fixed by the inputs alone."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2502_11101_b200 import workloads as W
+from paper_2502_11101_b200.session import Session
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_full(cfg, samples):
+    meta = W.make_meta(cfg, 0)
+    dev = "cuda:0"
+    q = W.make_q(meta, dev)
+    k, v = W.make_kv(meta, dev)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len, device=dev)
+    # integer state after Init: bit-exact against the oracle's allocation, every request
+    sess.init()
+    plan0 = sess.read_plan()
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        dst, grp, n_reuse, qs = oracle.allocate_positions(meta.doc_len[lo:hi], range(hi - lo), cfg.pos_range, 0, cfg.q_len)
+        assert np.array_equal(plan0["dst_start"][lo:hi], dst) and np.array_equal(plan0["group"][lo:hi], grp)
+        assert int(plan0["n_reuse"][b]) == n_reuse and int(plan0["query_start"][b]) == qs
+    out = torch.empty_like(q)
+    lse = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), device=dev)
+    scores = torch.empty((cfg.n_layers, meta.n_docs_total), device=dev)
+    sess.run_stack(q, k, v, cfg.schedule, oracle.ALLOC_ALIGN, out, lse, None, scores)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    # ---- sampled outputs of layer 1 (all documents kept, retrieval order)
+    g = cfg.group_size
+    for b, h in samples:
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        n = hi - lo
+        r0, r1 = int(meta.doc_offsets[lo]), int(meta.doc_offsets[hi])
+        kvh = h // g
+        k_req = k[0, r0:r1, kvh:kvh + 1].double().cpu().numpy()
+        v_req = v[0, r0:r1, kvh:kvh + 1].double().cpu().numpy()
+        off = meta.doc_offsets[lo:hi + 1] - r0
+        dst, _, _, _ = oracle.allocate_positions(meta.doc_len[lo:hi], range(n), cfg.pos_range, 0, cfg.q_len)
+        k_rot = oracle.reposition_keys(k_req, off, meta.doc_src_start[lo:hi], dst, range(n), cfg.rope_theta)
+        q_h = q[0, b, :, h:h + 1].double().cpu().numpy()
+        o_ref, lse_ref, mass, _ = oracle.query_prefill_attn(q_h, k_rot, v_req, off, range(n), n)
+        o_got = out[0, b, :, h].float().cpu().numpy()
+        assert np.all(np.abs(o_got - o_ref[:, 0]) <= 1e-2 + 2e-2 * np.abs(o_ref[:, 0])), (b, h)
+        assert np.all(np.abs(lse[0, b, h].cpu().numpy() - lse_ref[0]) <= 1e-2), (b, h)
+    # ---- properties that hold at any size
+    sc = scores.cpu().numpy()
+    for layer in range(1, cfg.n_layers + 1):
+        for b in range(cfg.batch):
+            lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+            s = sc[layer - 1, lo:hi]
+            assert abs(float(s.sum()) - 1.0) < 2e-3, (layer, b)                 # masses of a request sum to 1
+            assert int((s > 0).sum()) == cfg.kept_at_layer(layer), (layer, b)   # pruned documents score exactly 0
+    plan = sess.read_plan()
+    final_keep = cfg.schedule[-1][1]
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        order = plan["order"][b]
+        assert len(order) == final_keep and len(set(order)) == final_keep
+        assert set(meta.planted[b]) <= set(order), "planted documents must survive every pruning layer"
+        qs = int(plan["query_start"][b])
+        spans = {}
+        for i in order:                                                          # allocation invariants
+            d0 = int(plan["dst_start"][lo + i])
+            assert 0 <= d0 and d0 + int(meta.doc_len[lo + i]) <= qs
+            spans.setdefault(int(plan["group"][lo + i]), []).append((d0, d0 + int(meta.doc_len[lo + i])))
+        for win in spans.values():
+            win.sort()
+            assert win[-1][1] == qs and all(a[1] == c[0] for a, c in zip(win, win[1:]))
+        pruned = np.setdiff1d(np.arange(hi - lo), order)
+        assert np.all(plan["dst_start"][lo + pruned] == -1)
+    return plan0
+
+
+def test_config4_full_size_sampled():
+    _run_full(W.CONFIGS[4], samples=[(0, 0), (1, 13), (3, 27)])
+
+
+def test_config5_four_layers_full_batch_sampled():
+    # the full 32-layer store is 90 GB; four layers keep the per-layer launch configuration (8 requests x
+    # 120 documents x 32 heads, six parallel windows) and hold 11 GB
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=4, schedule=((1, 60), (2, 30), (3, 15)))
+    plan0 = _run_full(cfg, samples=[(0, 0), (5, 17), (7, 31)])
+    assert all(int(x) == 6 for x in plan0["n_reuse"])
