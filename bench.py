@@ -159,8 +159,8 @@ class GpuWorkload:
 
     def launches_per_step(self):
         cfg = self.cfg
-        # plan init + per layer (attention, merge + scores) + prune/plan kernels + final re-positioning
-        return 1 + 2 * cfg.n_layers + len(cfg.schedule) + 1
+        # plan init + per layer (attention, merge, scores) + prune/plan kernels + final re-positioning
+        return 1 + 3 * cfg.n_layers + len(cfg.schedule) + 1
 
 
 def time_steps(fn, steps, warmup, world):

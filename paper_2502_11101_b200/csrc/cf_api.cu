@@ -171,16 +171,12 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
     size_t l = take(nb * n_splits * rows);
     size_t t = take(max_tiles * rows);
     size_t r = take(nb * rows);
-    size_t f = take(2 * (size_t)b->n_docs_total);
-    size_t k = take(nb);
     if (ws) {
         ws->part_o = reinterpret_cast<float*>(base + o);
         ws->part_m = reinterpret_cast<float*>(base + m);
         ws->part_l = reinterpret_cast<float*>(base + l);
         ws->tile_lse2 = reinterpret_cast<float*>(base + t);
         ws->row_lse2 = reinterpret_cast<float*>(base + r);
-        ws->doc_fixed = reinterpret_cast<unsigned long long*>(base + f);
-        ws->ticket = reinterpret_cast<int*>(base + k);
         ws->n_splits = n_splits;
         ws->part_bf16 = 0;
     }

@@ -55,10 +55,6 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
     }
 
     const int doc0 = bv.req_doc_begin[b];
-    if (blockIdx.x == 0 && blockIdx.y == 0) {                      // reset this request's score accumulators
-        for (int i = doc0 + tid; i < bv.req_doc_begin[b + 1]; i += kSimtThreads) ws.doc_fixed[i] = 0ull;
-        if (tid == 0) ws.ticket[b] = 0;
-    }
     const int base = tile_base(doc0, bv.doc_offsets[doc0]);
     const int n_tiles = pv.n_tiles[b];
     const int t_begin = (int)((long long)n_tiles * split / ws.n_splits);
@@ -157,19 +153,11 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
 // Merge the parts of one query row (one block per row, one thread per output dimension):
 // out = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m), and the row's log-sum-exp.
 // Parts are visited in index order, so the result does not depend on scheduling.
-//
-// Document scores (footnote of Sec. 2.4; Algorithm 2: S <- S + s^l) are finished here as well: every
-// row adds its masses 2^(tile_lse - row_lse) to one integer per document (units of 2^-40, so the sum
-// is exact and independent of the order of the atomic additions), and the block that finishes last
-// for a request turns the integers into doc_scores, adds them to score_accum and clears them.
 template <typename T, int D, typename P>
 __global__ void __launch_bounds__(D)
-combine_kernel(AttnWorkspace ws, BatchView bv, PlanView pv, int n_q_heads, int lq, T* __restrict__ out,
-               float* __restrict__ lse, float* __restrict__ doc_scores, float* __restrict__ score_accum) {
+combine_kernel(AttnWorkspace ws, int n_q_heads, int lq, T* __restrict__ out, float* __restrict__ lse) {
     __shared__ float s_w[CF_MAX_SPLITS];
     __shared__ float s_red[2][D / 32];
-    __shared__ float s_lse2;
-    __shared__ int s_last;
     const int rows_total = n_q_heads * lq;
     const int b = blockIdx.x / rows_total, rg = blockIdx.x - b * rows_total;
     const int h = rg / lq, j = rg - h * lq;
@@ -226,31 +214,44 @@ combine_kernel(AttnWorkspace ws, BatchView bv, PlanView pv, int n_q_heads, int l
         const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
         ws.row_lse2[(size_t)b * rows_total + rg] = lse2;
         if (lse) lse[(size_t)b * rows_total + rg] = lse2 * kLn2;
-        s_lse2 = lse2;
     }
-    if (!doc_scores && !score_accum) return;
-    __syncthreads();
-    const float lse2 = s_lse2;
-    const int tbase = pv.tile_begin[b], n_tiles = pv.n_tiles[b];
-    if (lse2 > -INFINITY) {
-        for (int t = tid; t < n_tiles; t += D) {
-            const float mass = exp2f(ws.tile_lse2[(size_t)(tbase + t) * rows_total + rg] - lse2);
-            atomicAdd(ws.doc_fixed + pv.tile_doc[tbase + t], (unsigned long long)(mass * 1099511627776.0f + 0.5f));
-        }
+}
+
+// Document scores (footnote of Sec. 2.4; Algorithm 2: S <- S + s^l): one block per document sums
+// 2^(tile_lse - row_lse) over the document's tiles and all query rows, in a fixed order.
+__global__ void __launch_bounds__(256)
+score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float* __restrict__ doc_scores,
+             float* __restrict__ score_accum) {
+    __shared__ float s_red[256];
+    const int doc = blockIdx.x;
+    const int count = pv.doc_tile_count[doc];
+    if (count == 0) {
+        if (threadIdx.x == 0 && doc_scores) doc_scores[doc] = 0.f;
+        return;
     }
-    __threadfence();
+    int lo = 0, hi = bv.n_requests;                 // request that owns the document
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (bv.req_doc_begin[mid] <= doc) lo = mid; else hi = mid;
+    }
+    const float* row_lse2 = ws.row_lse2 + (size_t)lo * rows_total;
+    const float* tile_lse2 = ws.tile_lse2 + (size_t)pv.doc_tile_begin[doc] * rows_total;
+    float sum = 0.f;
+    for (int idx = threadIdx.x; idx < count * rows_total; idx += 256) {
+        const int rg = idx % rows_total;
+        sum += exp2f(tile_lse2[idx] - row_lse2[rg]);
+    }
+    s_red[threadIdx.x] = sum;
     __syncthreads();
-    if (tid == 0) s_last = atomicAdd(ws.ticket + b, 1) == rows_total - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const double unit = 1.0 / (1099511627776.0 * (double)rows_total);
-    for (int doc = bv.req_doc_begin[b] + tid; doc < bv.req_doc_begin[b + 1]; doc += D) {
-        const float score = (float)((double)atomicExch(ws.doc_fixed + doc, 0ull) * unit);
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) s_red[threadIdx.x] += s_red[threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const float score = s_red[0] / (float)rows_total;
         if (doc_scores) doc_scores[doc] = score;
         if (score_accum) score_accum[doc] += score;
     }
-    if (tid == 0) ws.ticket[b] = 0;
 }
 
 template <typename T, int D>
@@ -291,27 +292,34 @@ int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, co
 }
 
 template <typename T, int D>
-static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
-                                void* out, float* lse, float* doc_scores, float* score_accum, cudaStream_t stream) {
+static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const AttnWorkspace& ws, void* out,
+                                float* lse, cudaStream_t stream) {
     const long long blocks = (long long)b->n_requests * g->n_q_heads * b->q_len;
     if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS || ws.n_splits > D) return CF_ERR_INVALID_ARG;
-    BatchView bv = make_batch_view(b);
     if (ws.part_bf16)
-        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, bv, pv, g->n_q_heads, b->q_len,
-                                                                              static_cast<T*>(out), lse, doc_scores, score_accum);
+        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     else
-        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, bv, pv, g->n_q_heads, b->q_len,
-                                                                      static_cast<T*>(out), lse, doc_scores, score_accum);
+        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
 int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
                    void* out, float* lse, float* doc_scores, float* score_accum, cudaStream_t stream) {
+    int rc;
     if (g->dtype == CF_BF16)
-        return g->head_dim == 128 ? launch_combine_typed<__nv_bfloat16, 128>(g, b, pv, ws, out, lse, doc_scores, score_accum, stream)
-                                  : launch_combine_typed<__nv_bfloat16, 64>(g, b, pv, ws, out, lse, doc_scores, score_accum, stream);
-    return g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, pv, ws, out, lse, doc_scores, score_accum, stream)
-                              : launch_combine_typed<float, 64>(g, b, pv, ws, out, lse, doc_scores, score_accum, stream);
+        rc = g->head_dim == 128 ? launch_combine_typed<__nv_bfloat16, 128>(g, b, ws, out, lse, stream)
+                                : launch_combine_typed<__nv_bfloat16, 64>(g, b, ws, out, lse, stream);
+    else
+        rc = g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, ws, out, lse, stream)
+                                : launch_combine_typed<float, 64>(g, b, ws, out, lse, stream);
+    if (rc != CF_OK) return rc;
+    if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
+        score_kernel<<<(unsigned)b->n_docs_total, 256, 0, stream>>>(make_batch_view(b), pv, ws,
+                                                                   g->n_q_heads * b->q_len, doc_scores,
+                                                                   score_accum);
+        if (cudaGetLastError() != cudaSuccess) return CF_ERR_CUDA;
+    }
+    return CF_OK;
 }
 
 }  // namespace cf

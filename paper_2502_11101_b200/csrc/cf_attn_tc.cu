@@ -270,11 +270,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     // first workspace row of this CTA in part 2*pair
     const size_t slot0 = ((size_t)b * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * 256;
 
-    if (blockIdx.x == 0 && blockIdx.y == 0) {                       // reset this request's score accumulators
-        const int d0 = bv.req_doc_begin[b], d1 = bv.req_doc_begin[b + 1];
-        for (int i = d0 + tid; i < d1; i += kThreads) ws.doc_fixed[i] = 0ull;
-        if (tid == 0) ws.ticket[b] = 0;
-    }
     // rows that will carry no data in one of the two parts: mark them neutral (m = -inf)
     for (int r = tid; r < rows_here; r += kThreads) {
         if (n_it <= 0) ws.part_m[slot0 + r] = -INFINITY;

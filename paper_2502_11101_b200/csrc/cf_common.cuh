@@ -70,10 +70,6 @@ struct AttnWorkspace {
     float* part_l;     // [B][n_splits][Hq*Lq]      sum_t 2^(t - m)
     float* tile_lse2;  // [max_tiles][Hq*Lq]        log2 of sum over the tile's tokens of 2^t
     float* row_lse2;   // [B][Hq*Lq]                log2 of the full softmax denominator
-    unsigned long long* doc_fixed;   // [n_docs_total] attention mass per document summed over rows, in
-                                     // units of 2^-40 (integer sums do not depend on the order of addition);
-                                     // zeroed by the attention kernel, consumed and re-zeroed by the merge
-    int* ticket;       // [B]                       merge blocks of a request that have finished
     int n_splits;
     int part_bf16;     // the tensor-core kernel stores its partial O rows as bf16
 };
