@@ -20,6 +20,10 @@
 //   warp 12      TMA producer (one lane)     warp 13  TMEM allocation and MMA issue (one lane)
 // The MMA warp interleaves the two warpgroups (PV of one, then the next QK^T of the same one), so
 // one warpgroup's exponentials overlap the other's tensor-core work.
+// The softmax is single-pass: the reference maximum of a row only moves when a 32-key chunk exceeds
+// it by more than 2^8, in which case O, the sums and the P columns already written are rescaled
+// (rare after the first chunk); any reference within the exponent range is exact enough because
+// P (bf16) and the sums (fp32) keep their relative precision.
 // Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
 // plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
 #include <cuda.h>
@@ -153,19 +157,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};\n"
-        "tcgen05.wait::st.sync.aligned;"
-        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
-          "r"(taddr)
-        : "memory");
-}
 // Asynchronous 32-column load: the registers may only be used after tmem_ld_wait(v).
 __device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -177,6 +168,25 @@ __device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32
 // compiler from moving their uses above the wait.
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31]) : : "memory");
+}
+// 16 columns, synchronous (used on the rare rescaling path).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};\n"
+        "tcgen05.wait::st.sync.aligned;"
+        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(taddr)
+        : "memory");
 }
 // 16 columns (32 packed bf16) of the P operand; completion is awaited once per tile.
 __device__ __forceinline__ void tmem_st16_async(uint32_t taddr, const uint32_t (&v)[32]) {
@@ -499,62 +509,68 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const int n_chunks = (len + 31) >> 5;               // 32 keys per chunk, loads double-buffered
+                if (j > 0) {
+                    // PV(j-1) sits before S(j) in the tensor pipe, so it is complete; waiting here keeps
+                    // this thread's view of the barrier in step (every phase is waited for, in order)
+                    ok = mbar_wait(smem_u32(&bars->o_done[w]), (j - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                // Single pass over S in 32-key chunks, loads double-buffered.  The reference maximum only
+                // moves when a chunk exceeds it by more than 2^8; then O, the sums and the P chunks of this
+                // tile that are already written are rescaled (rare after the first chunk of the first tile).
+                const int n_chunks = (len + 31) >> 5;
+                float tile_sum = 0.f;
                 uint32_t va[32], vb[32];
-                // pass 1: row maximum
-                float mx = -INFINITY;
+                // step 1 of a chunk; no tensor-memory load may be in flight across these branches
+                auto prepare = [&](const uint32_t (&v)[32], int valid, int c) {
+                    const float cmax = (valid >= 32 ? chunk_max<false>(v, 32) : chunk_max<true>(v, valid)) * scale_log2;
+                    const bool move = cmax > m_ref + kRescaleThreshold;       // very first chunk: m_ref = -inf
+                    if (__any_sync(0xffffffffu, move)) {
+                        float alpha = 1.f;
+                        if (move) {
+                            alpha = fast_exp2(m_ref - cmax);                  // 0 when nothing is accumulated yet
+                            m_ref = cmax;
+                        }
+                        if (j > 0) {
+                            for (int cc = 0; cc < 8; ++cc) {
+                                uint32_t o[16];
+                                tmem_ld16(o_addr + cc * 16, o);
+#pragma unroll
+                                for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                                tmem_st16(o_addr + cc * 16, o);
+                            }
+                        }
+                        if (c > 0) asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");   // P stores in flight
+                        for (int cc = 0; cc < c; ++cc) {
+                            uint32_t pk[16];
+                            tmem_ld16(s_addr + cc * 16, pk);
+#pragma unroll
+                            for (int k = 0; k < 16; ++k)
+                                pk[k] = pack_bf16(__uint_as_float(pk[k] << 16) * alpha, __uint_as_float(pk[k] & 0xffff0000u) * alpha);
+                            tmem_st16(s_addr + cc * 16, pk);
+                        }
+                        l_run *= alpha;
+                        tile_sum *= alpha;
+                    }
+                };
+                // step 2 (straight-line): exponentials, packing; P chunk c lands in S columns 16c..16c+15,
+                // which belong to S chunks already held in registers
+                auto finish = [&](uint32_t (&v)[32], int valid, int c) {
+                    tile_sum += valid >= 32 ? chunk_exp<false>(v, 32, scale_log2, -m_ref) : chunk_exp<true>(v, valid, scale_log2, -m_ref);
+                    tmem_st16_async(s_addr + c * 16, v);
+                };
                 tmem_ld32_async(s_addr, va);
                 tmem_ld_wait(va);
                 for (int c = 0; c < n_chunks; c += 2) {
+                    prepare(va, len - c * 32, c);
                     if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
-                    mx = fmaxf(mx, len - c * 32 >= 32 ? chunk_max<false>(va, 32) : chunk_max<true>(va, len - c * 32));
+                    finish(va, len - c * 32, c);
                     if (c + 1 < n_chunks) {
                         tmem_ld_wait(vb);
+                        prepare(vb, len - c * 32 - 32, c + 1);
                         if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
-                        mx = fmaxf(mx, len - c * 32 >= 64 ? chunk_max<false>(vb, 32) : chunk_max<true>(vb, len - c * 32 - 32));
-                        if (c + 2 < n_chunks) tmem_ld_wait(va);
-                    }
-                }
-                mx *= scale_log2;
-                const bool move = mx > m_ref + kRescaleThreshold;   // first item: m_ref = -inf, always moves
-                float alpha = 1.f;
-                if (move) {
-                    alpha = fast_exp2(m_ref - mx);                  // 0 on the first item
-                    m_ref = mx;
-                }
-                tmem_ld32_async(s_addr, va);                        // first chunk of pass 2, in flight during the checks
-                if (j > 0) {
-                    // PV of the previous item must be complete before O is rescaled (and it has read P)
-                    ok = mbar_wait(smem_u32(&bars->o_done[w]), (j - 1) & 1, abort_flag);
-                    if (!ok) { tmem_ld_wait(va); break; }
-                    tc_fence_after();
-                    if (__any_sync(0xffffffffu, move)) {            // rare after the first tiles
-                        tmem_ld_wait(va);
-                        for (int c = 0; c < 4; ++c) {
-                            tmem_ld32(o_addr + c * 32, vb);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
-                            tmem_st32(o_addr + c * 32, vb);
-                        }
-                        l_run *= alpha;
-                    }
-                }
-                // pass 2: exponentials; P chunk c (16 packed columns) lands in S columns 16c..16c+15,
-                // which belong to S chunks already held in registers
-                float tile_sum = 0.f;
-                const float neg_ref = -m_ref;
-                tmem_ld_wait(va);
-                for (int c = 0; c < n_chunks; c += 2) {
-                    if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
-                    tile_sum += len - c * 32 >= 32 ? chunk_exp<false>(va, 32, scale_log2, neg_ref)
-                                                   : chunk_exp<true>(va, len - c * 32, scale_log2, neg_ref);
-                    tmem_st16_async(s_addr + c * 16, va);
-                    if (c + 1 < n_chunks) {
-                        tmem_ld_wait(vb);
-                        if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
-                        tile_sum += len - c * 32 >= 64 ? chunk_exp<false>(vb, 32, scale_log2, neg_ref)
-                                                       : chunk_exp<true>(vb, len - c * 32 - 32, scale_log2, neg_ref);
-                        tmem_st16_async(s_addr + (c + 1) * 16, vb);
+                        finish(vb, len - c * 32 - 32, c + 1);
                         if (c + 2 < n_chunks) tmem_ld_wait(va);
                     }
                 }
