@@ -209,3 +209,51 @@ def test_argument_errors_are_reported_not_faulted():
                     cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
     tight.init()
     assert tight.status() == cf.CF_ERR_RANGE
+
+
+def test_degenerate_batches():
+    """A request without documents, a one-token document, keep = 0: results are defined, nothing faults."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    lens = np.array([1, 130, 17], dtype=np.int32)                    # request 0: one token; request 1: none; request 2: two docs
+    req = np.array([0, 1, 1, 3], dtype=np.int32)
+    src = np.zeros(3, dtype=np.int32)
+    hq, hkv, d, lq = 4, 2, 128, 5
+    sess = Session(hq, hkv, d, torch.bfloat16, 4096, 1e4, lq, lens, req, src, tail_reserve=lq)
+    gen = torch.Generator().manual_seed(0)
+    total = int(lens.sum())
+    q = torch.randn((3, lq, hq, d), generator=gen).bfloat16().cuda()
+    k = torch.randn((total, hkv, d), generator=gen).bfloat16().cuda()
+    v = torch.randn((total, hkv, d), generator=gen).bfloat16().cuda()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((3, hq, lq), float("nan"), device="cuda")
+    for path in (0, 1):
+        cf.cf_set_attn_path(path)
+        try:
+            sess.init()
+            sess.attend(q, k, v, out, lse)
+            torch.cuda.synchronize()
+        finally:
+            cf.cf_set_attn_path(0)
+        assert sess.status() == 0
+        o = out.float().cpu().numpy()
+        # one-token document: the softmax has a single term, the output is that value row
+        for h in range(hq):
+            assert np.allclose(o[0, :, h], v[0, h // 2].float().cpu().numpy(), atol=1e-2)
+        assert np.all(o[1] == 0.0) and np.all(np.isneginf(lse[1].cpu().numpy()))   # nothing to attend
+        s = sess.doc_scores.cpu().numpy()
+        assert abs(s[0] - 1.0) < 1e-4 and abs(s[1] + s[2] - 1.0) < 1e-3
+        # oracle for request 2 (no position change matters for the check of masses: compare outputs)
+        dst, _, _, _ = oracle.allocate_positions(lens[1:], [0, 1], 4096, 0, lq)
+        off = np.array([0, 130, 147])
+        kr = oracle.reposition_keys(k[1:].double().cpu().numpy(), off, [0, 0], dst, [0, 1], 1e4)
+        o_ref, lse_ref, _, s_ref = oracle.query_prefill_attn(q[2].double().cpu().numpy(), kr, v[1:].double().cpu().numpy(),
+                                                             off, [0, 1], 2)
+        assert np.all(np.abs(o[2] - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
+        assert np.allclose(s[1:], s_ref, rtol=2e-2, atol=1e-3)
+    # keep = 0 empties every request; the next layer then attends nothing
+    sess.prune(0, oracle.ALLOC_ALIGN)
+    sess.attend(q, k, v, out, lse)
+    torch.cuda.synchronize()
+    assert sess.status() == 0 and sess.read_plan()["order"] == [[], [], []]
+    assert np.all(out.float().cpu().numpy() == 0.0) and np.all(sess.doc_scores.cpu().numpy() == 0.0)
