@@ -23,8 +23,6 @@ __global__ void __launch_bounds__(kSimtThreads)
 attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads,
                  float scale_log2, const T* __restrict__ q, const T* __restrict__ k_cache,
                  const T* __restrict__ v_cache) {
-    pdl_wait();
-    pdl_trigger();
     extern __shared__ float smem[];
     float (*Qs)[D + 1] = reinterpret_cast<float (*)[D + 1]>(smem);
     float (*Ks)[D + 1] = reinterpret_cast<float (*)[D + 1]>(smem + kSimtRows * (D + 1));
@@ -160,8 +158,6 @@ __global__ void __launch_bounds__(D)
 combine_kernel(AttnWorkspace ws, int n_q_heads, int lq, T* __restrict__ out, float* __restrict__ lse) {
     __shared__ float s_w[CF_MAX_SPLITS];
     __shared__ float s_red[2][D / 32];
-    pdl_wait();
-    pdl_trigger();
     const int rows_total = n_q_heads * lq;
     const int b = blockIdx.x / rows_total, rg = blockIdx.x - b * rows_total;
     const int h = rg / lq, j = rg - h * lq;
@@ -227,8 +223,6 @@ __global__ void __launch_bounds__(256)
 score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float* __restrict__ doc_scores,
              float* __restrict__ score_accum) {
     __shared__ float s_red[256];
-    pdl_wait();
-    pdl_trigger();
     const int doc = blockIdx.x;
     const int count = pv.doc_tile_count[doc];
     if (count == 0) {
@@ -277,9 +271,10 @@ static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView
                 return CF_ERR_CUDA;
             configured[which] = true;
         }
-        return launch_pdl(kernel, grid, dim3(kSimtThreads), smem, stream, bv, pv, ws, g->n_q_heads, g->n_kv_heads,
-                          scale_log2, static_cast<const T*>(q), static_cast<const T*>(k),
-                          static_cast<const T*>(v)) == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+        kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, g->n_q_heads, g->n_kv_heads, scale_log2,
+                                                     static_cast<const T*>(q), static_cast<const T*>(k),
+                                                     static_cast<const T*>(v));
+        return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
     if (g->rope_layout == CF_ROPE_HALF) return run(attn_simt_kernel<T, D, CF_ROPE_HALF>, 0);
     return run(attn_simt_kernel<T, D, CF_ROPE_INTERLEAVED>, 1);
@@ -301,14 +296,11 @@ static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const AttnW
                                 float* lse, cudaStream_t stream) {
     const long long blocks = (long long)b->n_requests * g->n_q_heads * b->q_len;
     if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS || ws.n_splits > D) return CF_ERR_INVALID_ARG;
-    cudaError_t err;
     if (ws.part_bf16)
-        err = launch_pdl(combine_kernel<T, D, __nv_bfloat16>, dim3((unsigned)blocks), dim3(D), 0, stream, ws, g->n_q_heads,
-                         b->q_len, static_cast<T*>(out), lse);
+        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     else
-        err = launch_pdl(combine_kernel<T, D, float>, dim3((unsigned)blocks), dim3(D), 0, stream, ws, g->n_q_heads,
-                         b->q_len, static_cast<T*>(out), lse);
-    return err == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
 int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
@@ -322,9 +314,10 @@ int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                                 : launch_combine_typed<float, 64>(g, b, ws, out, lse, stream);
     if (rc != CF_OK) return rc;
     if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
-        if (launch_pdl(score_kernel, dim3((unsigned)b->n_docs_total), dim3(256), 0, stream, make_batch_view(b), pv, ws,
-                       g->n_q_heads * b->q_len, doc_scores, score_accum) != cudaSuccess)
-            return CF_ERR_CUDA;
+        score_kernel<<<(unsigned)b->n_docs_total, 256, 0, stream>>>(make_batch_view(b), pv, ws,
+                                                                   g->n_q_heads * b->q_len, doc_scores,
+                                                                   score_accum);
+        if (cudaGetLastError() != cudaSuccess) return CF_ERR_CUDA;
     }
     return CF_OK;
 }

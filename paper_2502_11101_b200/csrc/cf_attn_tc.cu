@@ -244,8 +244,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads, float scale_log2,
                const __nv_bfloat16* __restrict__ q) {
-    pdl_wait();          // everything queued before this launch is complete and visible from here on
-    pdl_trigger();       // the merge kernel may be scheduled; it waits for this grid before it reads
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -707,9 +705,9 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                 return CF_ERR_CUDA;
             configured[which] = true;
         }
-        return launch_pdl(kernel, grid, dim3(kThreads), (size_t)kSmemBytes, stream, map_k, map_v, bv, pv, ws, g->n_q_heads,
-                          g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q)) == cudaSuccess ? CF_OK
-                                                                                                          : CF_ERR_CUDA;
+        kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_k, map_v, bv, pv, ws, g->n_q_heads, g->n_kv_heads,
+                                                       scale_log2, static_cast<const __nv_bfloat16*>(q));
+        return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
     if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);
     return run(attn_tc_kernel<CF_ROPE_INTERLEAVED>, 1);

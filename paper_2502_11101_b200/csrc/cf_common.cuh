@@ -93,30 +93,6 @@ int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                    void* out, float* lse, float* doc_scores, float* score_accum,
                    cudaStream_t stream);
 
-// ---- programmatic dependent launch ---------------------------------------------------------
-// The per-layer kernels (attention, merge, scores) are launched so that the next one may be
-// scheduled while its predecessor is still running.  Each of them starts with pdl_wait() -- which
-// returns once every earlier grid of the stream has completed and its writes are visible -- before
-// its first global-memory access, and then lets its own successor be scheduled.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                              Args&&... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 // ---- device helpers -----------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
