@@ -115,9 +115,10 @@ class GpuWorkload:
     """A ring of resident input sets (distinct seeds) so that consecutive steps never find their
     inputs in L2, plus the session and output buffers of the library."""
 
-    def __init__(self, cfg, seed, device, ring):
+    def __init__(self, cfg, seed, device, ring, batch_layers=True):
         from paper_2502_11101_b200.session import Session
         self.cfg, self.device = cfg, device
+        self.batch_layers = batch_layers
         self.meta = W.make_meta(cfg, seed)
         m = self.meta
         self.sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range,
@@ -138,7 +139,22 @@ class GpuWorkload:
 
     def step(self, slot):
         q, k, v = self.slots[slot % len(self.slots)]
-        self.sess.run_stack(q, k, v, self.cfg.schedule, STRATEGY_ALIGN, self.out, self.lse, self.k_final)
+        self.sess.run_stack(q, k, v, self.cfg.schedule, STRATEGY_ALIGN, self.out, self.lse, self.k_final,
+                            batch_layers=self.batch_layers)
+
+    def calls(self):
+        """(first, last) layer ranges of the attention calls of one step."""
+        from paper_2502_11101_b200 import binding as B
+        n = self.cfg.n_layers
+        if not self.batch_layers:
+            return [(i, i + 1) for i in range(n)]
+        cuts = sorted(l for l, _ in self.cfg.schedule if l < n) + [n]
+        out, first = [], 0
+        for last in cuts:
+            for lo in range(first, last, B.CF_MAX_LAYERS_PER_CALL):
+                out.append((lo, min(last, lo + B.CF_MAX_LAYERS_PER_CALL)))
+            first = last
+        return out
 
     def kept_per_layer(self, slot=0):
         """One instrumented step: the kept sets seen by every layer."""
@@ -159,8 +175,8 @@ class GpuWorkload:
 
     def launches_per_step(self):
         cfg = self.cfg
-        # plan init + per layer (attention, merge, scores) + prune/plan kernels + final re-positioning
-        return 1 + 3 * cfg.n_layers + len(cfg.schedule) + 1
+        # plan init + per attention call (attention, merge, scores) + prune/plan kernels + final re-positioning
+        return 1 + 3 * len(self.calls()) + len(cfg.schedule) + 1
 
 
 def time_steps(fn, steps, warmup, world):
@@ -293,6 +309,8 @@ def main():
     ap.add_argument("--ring", type=int, default=3, help="distinct resident input sets cycled between steps")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="one attention call per layer instead of one per run of layers between two pruning layers")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
@@ -328,7 +346,7 @@ def main():
         cf.cf_set_attn_path(1)
     peaks = load_peaks()
 
-    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring)
+    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer)
     kept, survivors = wl.kept_per_layer()
     per_layer_tokens = token_layers(cfg, wl.meta, kept)
     tokens_per_step = sum(per_layer_tokens)
@@ -337,22 +355,26 @@ def main():
     assert wl.sess.status() == 0
 
     # ---- CUDA graphs: one per ring slot (pointers differ) -------------------------------------
-    graphs = None
-    if not args.no_graph:
+    def capture():
+        if args.no_graph:
+            return None
         try:
             wl.step(0)
             torch.cuda.synchronize()
-            graphs = []
+            made = []
             side = torch.cuda.Stream()
             for r in range(args.ring):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=side):
                     wl.step(r)
-                graphs.append(g)
+                made.append(g)
+            return made
         except Exception as exc:  # capture not possible: time eager launches and say so
-            graphs = None
             sys.stderr.write(f"[bench] graph capture failed, timing eager launches: {exc}\n")
             torch.cuda.synchronize()
+            return None
+
+    graphs = capture()
 
     def run(i):
         if graphs is not None:
@@ -367,6 +389,21 @@ def main():
 
     ms_max, tokens_all, value = whole_job(ms, tokens_per_step, args.steps, world, device)
 
+    # ---- the same step with one attention call per layer (what a running model can issue) ------
+    per_layer = None
+    if wl.batch_layers and world == 1:
+        main_graphs = graphs
+        wl.batch_layers = False
+        graphs = capture()
+        pl_steps = max(1, min(args.steps, 100))
+        pl_ms, _, _ = time_steps(run, pl_steps, 3, world)
+        assert wl.sess.status() == 0
+        per_layer = {"value": tokens_per_step * pl_steps / (pl_ms * 1e-3), "unit": UNIT, "ms_per_step": pl_ms / pl_steps,
+                     "steps": pl_steps, "gpu_launches_per_step": wl.launches_per_step(),
+                     "note": "one cf_query_prefill_attn call per layer"}
+        wl.batch_layers = True
+        graphs, main_graphs = main_graphs, None
+
     # ---- the dominant kernel alone: event pairs around every attention-kernel launch ----------
     # Launches are issued eagerly here; a spin kernel queued first keeps the GPU busy until the host
     # has enqueued the whole step, so the event pairs time kernels running back to back and not the
@@ -380,17 +417,23 @@ def main():
         host_s.append(time.perf_counter() - t_host)
     torch.cuda.synchronize()
     spin_cycles = int(max(host_s) * 1.5 * 2.0e9)
-    cf.cf_profile_begin(prof_steps * cfg.n_layers)
+    calls = wl.calls()
+    cf.cf_profile_begin(prof_steps * len(calls))
     for i in range(prof_steps):
         torch.cuda._sleep(spin_cycles)
         wl.step(3 + i)
         torch.cuda.synchronize()
-    durations = cf.cf_profile_end(prof_steps * cfg.n_layers).astype(np.float64)
+    durations = cf.cf_profile_end(prof_steps * len(calls)).astype(np.float64)
+    per_call_tokens = [sum(per_layer_tokens[lo:hi]) for lo, hi in calls]
     kv_bytes_per_token = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4) * cfg.n_kv_heads
     flops_per_token = 4 * cfg.group_size * cfg.q_len * cfg.head_dim * cfg.n_kv_heads
-    launch_bytes = np.tile(np.array(per_layer_tokens, dtype=np.float64) * kv_bytes_per_token, prof_steps)
-    launch_flops = np.tile(np.array(per_layer_tokens, dtype=np.float64) * flops_per_token, prof_steps)
+    launch_bytes = np.tile(np.array(per_call_tokens, dtype=np.float64) * kv_bytes_per_token, prof_steps)
+    launch_flops = np.tile(np.array(per_call_tokens, dtype=np.float64) * flops_per_token, prof_steps)
     n = min(len(durations), len(launch_bytes))
+    if n == prof_steps * len(calls):
+        per_call = durations[:n].reshape(prof_steps, len(calls)).mean(axis=0) * 1e3
+        sys.stderr.write("[bench] attention launches of a step, mean us (layers first-last): " +
+                         " ".join(f"{lo + 1}-{hi}:{x:.1f}" for (lo, hi), x in zip(calls, per_call)) + "\n")
     dur_s = durations[:n].sum() * 1e-3
     gbs = launch_bytes[:n].sum() / dur_s / 1e9
     tfs = launch_flops[:n].sum() / dur_s / 1e12
@@ -437,8 +480,11 @@ def main():
 
     attn_kernel = "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05"
     launches = wl.launches_per_step() * args.steps
+    n_calls = len(wl.calls())
     slot_mb = sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6
     launch_mode = "cuda graph per ring slot" if graphs is not None else "eager"
+    call_mode = ("one attention call per run of layers between two pruning layers (every layer's query states "
+                 "are inputs of the step)") if wl.batch_layers else "one attention call per layer"
     repo = None
     if world == 1 and not args.skip_reposition:
         del wl, graphs, host, q0, k0, v0
@@ -467,11 +513,12 @@ def main():
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
                              f"{slot_mb:.0f} MB) cycled between steps",
-                       "launch": launch_mode,
+                       "launch": launch_mode, "attention_calls": call_mode,
+                       "attention_calls_per_step": n_calls,
                        "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "reposition": repo, "cpu_baseline": cpu}
+            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -58,6 +58,7 @@ extern "C" {
 #define CF_TILE_TOKENS 128      /* key tiles never straddle two documents                       */
 #define CF_MAX_DOCS_PER_REQUEST 1024
 #define CF_MAX_SPLITS 64
+#define CF_MAX_LAYERS_PER_CALL 64 /* layers one cf_query_prefill_attn_layers call may batch       */
 #define CF_STATIC_WORKSPACE_BYTES (32u << 20)   /* scratch carried by cf_query_prefill_attn_static */
 
 /* Model-side geometry.  head_dim 64 or 128; pos_range = the model's positional range L of
@@ -198,6 +199,31 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
                           float softmax_scale, void* out, float* lse, float* doc_scores,
                           float* score_accum, void* workspace, size_t workspace_bytes,
                           void* stream);
+
+/* Several consecutive layers that attend the same kept documents, in one call (Algorithm 2:
+ * between two pruning layers the set ids, and with it the allocation, does not change, so
+ * layer_l ... layer_{l+m-1} read one plan).  Equivalent to n_layers successive calls of
+ * cf_query_prefill_attn on layer slices of the arguments, S <- S + s^l accumulated in layer
+ * order; the layers run side by side on the device.  A caller can use it when the query states
+ * of those layers are available together (replay, benchmarking, scoring passes with stored
+ * queries); inside a running model each layer's queries depend on the previous layer's output,
+ * and the single-layer call is the one that applies.
+ *   n_layers          1 .. CF_MAX_LAYERS_PER_CALL, and n_layers * n_requests <= 65535
+ *   q, out            layer i at q + i * q_layer_stride, out + i * out_layer_stride (elements);
+ *                     each layer laid out as in cf_query_prefill_attn
+ *   k_cache, v_cache  layer i of the store at + i * kv_layer_stride elements (a multiple of 8
+ *                     bf16 / 4 fp32 elements, at least total_tokens * token_stride if n_layers > 1)
+ *   lse               float [n_layers][n_requests][n_q_heads][q_len] or NULL
+ *   doc_scores        float [n_layers][n_docs_total] or NULL (every layer's s^l)
+ *   score_accum       float [n_docs_total] or NULL
+ *   workspace         at least cf_attn_workspace_bytes_layers(geom, batch, n_layers) bytes */
+size_t cf_attn_workspace_bytes_layers(const cf_geom* geom, const cf_batch* batch, int32_t n_layers);
+int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                                 int32_t n_layers, const void* q, int64_t q_layer_stride,
+                                 const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                                 float softmax_scale, void* out, int64_t out_layer_stride,
+                                 float* lse, float* doc_scores, float* score_accum,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* The same computation as cf_query_prefill_attn for callers that cannot allocate device memory
  * (the paper has no counterpart; this is a property of the library, not of the method).

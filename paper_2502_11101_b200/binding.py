@@ -16,13 +16,14 @@ CF_BF16, CF_F32 = 0, 1
 CF_ROPE_HALF, CF_ROPE_INTERLEAVED = 0, 1
 CF_ALLOC_NONE, CF_ALLOC_ALIGN, CF_ALLOC_SORT = 0, 1, 2
 CF_TILE_TOKENS = 128
+CF_MAX_LAYERS_PER_CALL = 64
 TC_KERNEL_BUILT = True      # bf16 / head_dim 128 batches take the tcgen05 attention kernel
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefocus.so")
 
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
-           "cf_query_prefill_attn", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -79,13 +80,17 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes.argtypes = [gp, bp]
     lib.cf_query_prefill_attn.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
+    lib.cf_attn_workspace_bytes_layers.restype = ctypes.c_size_t
+    lib.cf_attn_workspace_bytes_layers.argtypes = [gp, bp, i32]
+    lib.cf_query_prefill_attn_layers.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64,
+                                                 vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_query_prefill_attn_static.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
     lib.cf_profile_end.argtypes = [vp, i32, vp]
     for name in EXPORTS:
-        if name not in ("cf_error_string", "cf_attn_workspace_bytes"):
+        if name not in ("cf_error_string", "cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers"):
             getattr(lib, name).restype = ctypes.c_int
     _LIB = lib
     return lib
@@ -201,6 +206,31 @@ def cf_query_prefill_attn(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q:
                                               _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
                                               workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn")
+
+
+def cf_attn_workspace_bytes_layers(geom: cf_geom, batch: cf_batch, n_layers: int) -> int:
+    return int(load_library().cf_attn_workspace_bytes_layers(ctypes.byref(geom), ctypes.byref(batch), n_layers))
+
+
+def cf_query_prefill_attn_layers(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,
+                                 k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+                                 workspace: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                                 doc_scores: Optional[torch.Tensor] = None,
+                                 score_accum: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                                 stream=None) -> None:
+    """`q`, `out` [n_layers, B, Lq, Hq, D]; `k_cache`, `v_cache` [n_layers, T, ...]; `lse` [n_layers, B, Hq, Lq];
+    `doc_scores` [n_layers, n_docs_total].  Dimension 0 may be strided, the rest of a layer is dense."""
+    n_layers = q.shape[0]
+    assert k_cache.shape[0] == n_layers and v_cache.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k_cache.stride(0) == v_cache.stride(0)
+    for t in (lse, doc_scores):
+        assert t is None or (t.shape[0] == n_layers and t.is_contiguous())
+    rc = load_library().cf_query_prefill_attn_layers(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), n_layers, q.data_ptr(), q.stride(0),
+        k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(0), softmax_scale, out.data_ptr(), out.stride(0),
+        _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn_layers")
 
 
 def cf_query_prefill_attn_static(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,

@@ -132,13 +132,24 @@ int tiles_per_request_bound(const cf_batch* b) {
     return (int)std::min<long long>(t, 1 << 20);
 }
 
-// Parts the key-tile list of a request is cut into.  The tensor-core kernel runs one CTA per
-// (request, kv head, group of 256 query rows, pair of parts): as many CTAs as fit one wave over the
-// SMs, never more CTAs than tiles.  The count is always even.
-int choose_splits(const cf_geom* g, const cf_batch* b) {
+// Query rows one CTA of the tensor-core kernel owns.  A CTA holds two 128-row tiles; when the rows
+// that share a kv head fill an odd number of such tiles (and more than one), CTAs of one tile each
+// -- whose two warpgroups then take alternate key tiles -- split the work evenly, where pairs would
+// leave a half-empty CTA on the critical path.
+int choose_row_group(const cf_geom* g, const cf_batch* b) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
-    const int row_groups = (rows + 255) / 256;
-    const long long units = (long long)b->n_requests * g->n_kv_heads * row_groups;
+    const int row_tiles = (rows + 127) / 128;
+    return (row_tiles > 1 && (row_tiles & 1)) ? 128 : 256;
+}
+
+// Parts the key-tile list of a request is cut into.  The tensor-core kernel runs one CTA per
+// (layer, request, kv head, group of query rows, pair of parts): as many CTAs as fit one wave over
+// the SMs, never more CTAs than tiles.  The count is always even.
+int choose_splits(const cf_geom* g, const cf_batch* b, int n_layers) {
+    const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
+    const int rg_rows = choose_row_group(g, b);
+    const int row_groups = (rows + rg_rows - 1) / rg_rows;
+    const long long units = (long long)n_layers * b->n_requests * g->n_kv_heads * row_groups;
     const long long sms = sm_count();
     long long s = sms / units;                        // whole CTAs per SM: one wave, no ragged second wave
     if (s == 0) {                                     // more units than SMs: balance the waves instead
@@ -154,10 +165,10 @@ int choose_splits(const cf_geom* g, const cf_batch* b) {
     return 2 * (int)std::max<long long>(s, 1);
 }
 
-size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,
-                             void* base_ptr) {
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers,
+                             AttnWorkspace* ws, void* base_ptr) {
     const size_t rows = (size_t)g->n_q_heads * b->q_len;
-    const size_t nb = (size_t)b->n_requests;
+    const size_t nlb = (size_t)b->n_requests * (size_t)n_layers;
     const size_t max_tiles = (size_t)b->n_docs_total + (size_t)(b->total_tokens / kTile) + 1;
     char* base = static_cast<char*>(base_ptr);
     size_t off = 0;
@@ -166,11 +177,11 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         off = align_up(off + count * 4, 256);
         return at;
     };
-    size_t o = take(nb * n_splits * rows * g->head_dim);
-    size_t m = take(nb * n_splits * rows);
-    size_t l = take(nb * n_splits * rows);
-    size_t t = take(max_tiles * rows);
-    size_t r = take(nb * rows);
+    size_t o = take(nlb * n_splits * rows * g->head_dim);
+    size_t m = take(nlb * n_splits * rows);
+    size_t l = take(nlb * n_splits * rows);
+    size_t t = take((size_t)n_layers * max_tiles * rows);
+    size_t r = take(nlb * rows);
     if (ws) {
         ws->part_o = reinterpret_cast<float*>(base + o);
         ws->part_m = reinterpret_cast<float*>(base + m);
@@ -179,6 +190,9 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->row_lse2 = reinterpret_cast<float*>(base + r);
         ws->n_splits = n_splits;
         ws->part_bf16 = 0;
+        ws->n_layers = n_layers;
+        ws->max_tiles = (int)max_tiles;
+        ws->rg_rows = choose_row_group(g, b);
     }
     return off;
 }
@@ -190,6 +204,55 @@ int attn_path() { return g_attn_path.load(); }
 static std::vector<cudaEvent_t> g_prof_events;
 static int g_prof_capacity = 0;
 static int g_prof_used = 0;
+
+static int check_plan(const cf_geom* geom, const cf_batch* batch, const void* plan) {
+    if (!batch || !plan) return CF_ERR_INVALID_ARG;
+    int rc = validate(geom, batch);
+    if (rc != CF_OK) return rc;
+    if (reinterpret_cast<uintptr_t>(plan) % 256 != 0) return CF_ERR_WORKSPACE;
+    return CF_OK;
+}
+
+int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan, const LayerSpan& span,
+                    const void* q, const void* k_cache, const void* v_cache, float softmax_scale,
+                    void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
+                    size_t workspace_bytes, cudaStream_t s) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (!q || !k_cache || !v_cache || !out || !workspace) return CF_ERR_INVALID_ARG;
+    if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return CF_ERR_INVALID_ARG;
+    if (span.n_layers <= 0 || span.n_layers > CF_MAX_LAYERS_PER_CALL ||
+        (long long)span.n_layers * batch->n_requests > 65535)
+        return CF_ERR_INVALID_ARG;
+    const int esize = geom->dtype == CF_BF16 ? 2 : 4;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return CF_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(q) % 16 || reinterpret_cast<uintptr_t>(out) % 16 ||
+        reinterpret_cast<uintptr_t>(k_cache) % 16 || reinterpret_cast<uintptr_t>(v_cache) % 16)
+        return CF_ERR_INVALID_ARG;
+    if (span.n_layers > 1) {
+        const long long layer_rows = (long long)batch->n_requests * batch->q_len * geom->n_q_heads * geom->head_dim;
+        if (span.q_stride < layer_rows || span.out_stride < layer_rows ||
+            span.kv_stride < batch->total_tokens * batch->token_stride || (span.q_stride * esize) % 16 ||
+            (span.out_stride * esize) % 16 || (span.kv_stride * esize) % 16)
+            return CF_ERR_INVALID_ARG;
+    }
+    const int n_splits = choose_splits(geom, batch, span.n_layers);
+    AttnWorkspace ws;
+    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, &ws, workspace);
+    if (workspace_bytes < need) return CF_ERR_WORKSPACE;
+    const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
+    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    const bool timed = g_prof_used < g_prof_capacity;
+    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
+    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch)) {
+        ws.part_bf16 = 1;
+        rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
+    } else
+        rc = launch_attn_simt(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
+    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);
+    if (rc != CF_OK) return rc;
+    return launch_combine(geom, batch, pv, span, ws, out, lse, doc_scores, score_accum, s);
+}
 
 }  // namespace cf
 
@@ -284,14 +347,6 @@ int cf_plan_layout_of(const cf_geom* geom, const cf_batch* batch, cf_plan_layout
     return CF_OK;
 }
 
-static int check_plan(const cf_geom* geom, const cf_batch* batch, const void* plan) {
-    if (!batch || !plan) return CF_ERR_INVALID_ARG;
-    int rc = validate(geom, batch);
-    if (rc != CF_OK) return rc;
-    if (reinterpret_cast<uintptr_t>(plan) % 256 != 0) return CF_ERR_WORKSPACE;
-    return CF_OK;
-}
-
 int cf_plan_init(const cf_geom* geom, const cf_batch* batch, const int32_t* order,
                  const int32_t* kept_count, int32_t query_start, void* plan, size_t plan_bytes,
                  void* stream) {
@@ -338,9 +393,13 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
                              static_cast<cudaStream_t>(stream));
 }
 
+size_t cf_attn_workspace_bytes_layers(const cf_geom* geom, const cf_batch* batch, int32_t n_layers) {
+    if (!batch || validate(geom, batch) != CF_OK || n_layers <= 0 || n_layers > CF_MAX_LAYERS_PER_CALL) return 0;
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, n_layers), n_layers, nullptr, nullptr);
+}
+
 size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch) {
-    if (!batch || validate(geom, batch) != CF_OK) return 0;
-    return attn_workspace_layout(geom, batch, choose_splits(geom, batch), nullptr, nullptr);
+    return cf_attn_workspace_bytes_layers(geom, batch, 1);
 }
 
 int cf_profile_begin(int32_t max_records) {
@@ -382,31 +441,21 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
                           float softmax_scale, void* out, float* lse, float* doc_scores,
                           float* score_accum, void* workspace, size_t workspace_bytes,
                           void* stream) {
-    int rc = check_plan(geom, batch, plan);
-    if (rc != CF_OK) return rc;
-    if (!q || !k_cache || !v_cache || !out || !workspace) return CF_ERR_INVALID_ARG;
-    if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return CF_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return CF_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(q) % 16 || reinterpret_cast<uintptr_t>(out) % 16 ||
-        reinterpret_cast<uintptr_t>(k_cache) % 16 || reinterpret_cast<uintptr_t>(v_cache) % 16)
-        return CF_ERR_INVALID_ARG;
-    const int n_splits = choose_splits(geom, batch);
-    AttnWorkspace ws;
-    const size_t need = attn_workspace_layout(geom, batch, n_splits, &ws, workspace);
-    if (workspace_bytes < need) return CF_ERR_WORKSPACE;
-    const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
-    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool timed = g_prof_used < g_prof_capacity;
-    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
-    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch)) {
-        ws.part_bf16 = 1;
-        rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    } else
-        rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);
-    if (rc != CF_OK) return rc;
-    return launch_combine(geom, batch, pv, ws, out, lse, doc_scores, score_accum, s);
+    const LayerSpan span = {1, 0, 0, 0};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
+                           score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                                 int32_t n_layers, const void* q, int64_t q_layer_stride,
+                                 const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                                 float softmax_scale, void* out, int64_t out_layer_stride,
+                                 float* lse, float* doc_scores, float* score_accum,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (q_layer_stride < 0 || kv_layer_stride < 0 || out_layer_stride < 0) return CF_ERR_INVALID_ARG;
+    const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
+                           score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,

@@ -20,7 +20,7 @@ constexpr size_t simt_smem_bytes() {
 
 template <typename T, int D, int LAYOUT>
 __global__ void __launch_bounds__(kSimtThreads)
-attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads,
+attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, LayerSpan span, int n_q_heads, int n_kv_heads,
                  float scale_log2, const T* __restrict__ q, const T* __restrict__ k_cache,
                  const T* __restrict__ v_cache) {
     extern __shared__ float smem[];
@@ -35,7 +35,12 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
     const int lq = bv.q_len;
     const int rows = group * lq;                                   // query rows sharing one kv head
     const int row_chunks = (rows + kSimtRows - 1) / kSimtRows;
-    const int b = blockIdx.z;
+    const int lb = blockIdx.z;                                     // layer * B + request
+    const int layer = lb / bv.n_requests;
+    const int b = lb - layer * bv.n_requests;
+    q += (size_t)layer * span.q_stride;
+    k_cache += (size_t)layer * span.kv_stride;
+    v_cache += (size_t)layer * span.kv_stride;
     const int kvh = blockIdx.y / row_chunks;
     const int r0 = (blockIdx.y - kvh * row_chunks) * kSimtRows;
     const int n_rows = min(kSimtRows, rows - r0);
@@ -137,10 +142,10 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
             }
         }
         if (q4 == 0 && r < n_rows)
-            ws.tile_lse2[(size_t)(base + ti) * rows_total + row_global] = m + log2f(l_tile);
+            ws.tile_lse2[((size_t)layer * ws.max_tiles + base + ti) * rows_total + row_global] = m + log2f(l_tile);
     }
     if (r < n_rows) {
-        const size_t slot = ((size_t)b * ws.n_splits + split) * rows_total + row_global;
+        const size_t slot = ((size_t)lb * ws.n_splits + split) * rows_total + row_global;
         if (q4 == 0) {
             ws.part_m[slot] = m;
             ws.part_l[slot] = l;
@@ -155,15 +160,17 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int
 // Parts are visited in index order, so the result does not depend on scheduling.
 template <typename T, int D, typename P>
 __global__ void __launch_bounds__(D)
-combine_kernel(AttnWorkspace ws, int n_q_heads, int lq, T* __restrict__ out, float* __restrict__ lse) {
+combine_kernel(AttnWorkspace ws, int n_requests, long long out_layer_stride, int n_q_heads, int lq,
+               T* __restrict__ out, float* __restrict__ lse) {
     __shared__ float s_w[CF_MAX_SPLITS];
     __shared__ float s_red[2][D / 32];
     const int rows_total = n_q_heads * lq;
-    const int b = blockIdx.x / rows_total, rg = blockIdx.x - b * rows_total;
+    const int lb = blockIdx.x / rows_total, rg = blockIdx.x - lb * rows_total;   // lb = layer * B + request
+    const int layer = lb / n_requests, b = lb - layer * n_requests;
     const int h = rg / lq, j = rg - h * lq;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_parts = ws.n_splits;
-    const size_t slot0 = (size_t)b * n_parts * rows_total + rg;       // part p sits at slot0 + p * rows_total
+    const size_t slot0 = (size_t)lb * n_parts * rows_total + rg;      // part p sits at slot0 + p * rows_total
 
     float m = -INFINITY, l = 0.f;
     if (tid < n_parts) {
@@ -209,24 +216,29 @@ combine_kernel(AttnWorkspace ws, int n_q_heads, int lq, T* __restrict__ out, flo
         if (wp > 0.f) acc = fmaf(to_float(po[(size_t)p * stride]), wp, acc);
     }
     const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-    out[(((size_t)b * lq + j) * n_q_heads + h) * D + tid] = from_float<T>(acc * inv);
+    out[(size_t)layer * out_layer_stride + (((size_t)b * lq + j) * n_q_heads + h) * D + tid] = from_float<T>(acc * inv);
     if (tid == 0) {
         const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
-        ws.row_lse2[(size_t)b * rows_total + rg] = lse2;
-        if (lse) lse[(size_t)b * rows_total + rg] = lse2 * kLn2;
+        ws.row_lse2[(size_t)lb * rows_total + rg] = lse2;
+        if (lse) lse[(size_t)lb * rows_total + rg] = lse2 * kLn2;
     }
 }
 
 // Document scores (footnote of Sec. 2.4; Algorithm 2: S <- S + s^l): one block per document sums
-// 2^(tile_lse - row_lse) over the document's tiles and all query rows, in a fixed order.
+// 2^(tile_lse - row_lse) over the document's tiles and all query rows of every layer of the call,
+// each layer in a fixed order, then adds the layers' scores to S in layer order.  Up to eight
+// layers are reduced side by side by groups of threads.
 __global__ void __launch_bounds__(256)
 score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float* __restrict__ doc_scores,
              float* __restrict__ score_accum) {
     __shared__ float s_red[256];
+    __shared__ float s_layer[CF_MAX_LAYERS_PER_CALL];
     const int doc = blockIdx.x;
+    const int n_layers = ws.n_layers;
     const int count = pv.doc_tile_count[doc];
     if (count == 0) {
-        if (threadIdx.x == 0 && doc_scores) doc_scores[doc] = 0.f;
+        if (doc_scores)
+            for (int l = threadIdx.x; l < n_layers; l += 256) doc_scores[(size_t)l * bv.n_docs_total + doc] = 0.f;
         return;
     }
     int lo = 0, hi = bv.n_requests;                 // request that owns the document
@@ -234,34 +246,51 @@ score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float*
         const int mid = (lo + hi) >> 1;
         if (bv.req_doc_begin[mid] <= doc) lo = mid; else hi = mid;
     }
-    const float* row_lse2 = ws.row_lse2 + (size_t)lo * rows_total;
-    const float* tile_lse2 = ws.tile_lse2 + (size_t)pv.doc_tile_begin[doc] * rows_total;
-    float sum = 0.f;
-    for (int idx = threadIdx.x; idx < count * rows_total; idx += 256) {
-        const int rg = idx % rows_total;
-        sum += exp2f(tile_lse2[idx] - row_lse2[rg]);
-    }
-    s_red[threadIdx.x] = sum;
-    __syncthreads();
-    for (int w = 128; w > 0; w >>= 1) {
-        if (threadIdx.x < w) s_red[threadIdx.x] += s_red[threadIdx.x + w];
+    int groups = 1;                                 // power of two, at most min(n_layers, 8)
+    while (groups * 2 <= n_layers && groups < 8) groups *= 2;
+    const int gs = 256 / groups;
+    const int g = threadIdx.x / gs, t = threadIdx.x - g * gs;
+    const int rounds = (n_layers + groups - 1) / groups;
+    const size_t tile0 = (size_t)pv.doc_tile_begin[doc];
+    for (int rd = 0; rd < rounds; ++rd) {
+        const int layer = rd * groups + g;
+        float sum = 0.f;
+        if (layer < n_layers) {
+            const float* row_lse2 = ws.row_lse2 + ((size_t)layer * bv.n_requests + lo) * rows_total;
+            const float* tile_lse2 = ws.tile_lse2 + ((size_t)layer * ws.max_tiles + tile0) * rows_total;
+            for (int idx = t; idx < count * rows_total; idx += gs) {
+                const int rg = idx % rows_total;
+                sum += exp2f(tile_lse2[idx] - row_lse2[rg]);
+            }
+        }
+        s_red[threadIdx.x] = sum;
+        __syncthreads();
+        for (int w = gs >> 1; w > 0; w >>= 1) {
+            if (t < w) s_red[threadIdx.x] += s_red[threadIdx.x + w];
+            __syncthreads();
+        }
+        if (t == 0 && layer < n_layers) s_layer[layer] = s_red[threadIdx.x] / (float)rows_total;
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        const float score = s_red[0] / (float)rows_total;
-        if (doc_scores) doc_scores[doc] = score;
-        if (score_accum) score_accum[doc] += score;
+        float acc = score_accum ? score_accum[doc] : 0.f;
+        for (int l = 0; l < n_layers; ++l) {
+            if (doc_scores) doc_scores[(size_t)l * bv.n_docs_total + doc] = s_layer[l];
+            acc += s_layer[l];
+        }
+        if (score_accum) score_accum[doc] = acc;
     }
 }
 
 template <typename T, int D>
-static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
-                             const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
-                             cudaStream_t stream) {
+static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                             const void* q, const void* k, const void* v, float scale_log2,
+                             const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_chunks = (rows + kSimtRows - 1) / kSimtRows;
-    if ((long long)g->n_kv_heads * row_chunks > 65535 || b->n_requests > 65535) return CF_ERR_INVALID_ARG;
-    dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_chunks), (unsigned)b->n_requests);
+    if ((long long)g->n_kv_heads * row_chunks > 65535 || (long long)b->n_requests * span.n_layers > 65535)
+        return CF_ERR_INVALID_ARG;
+    dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_chunks), (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
     const size_t smem = simt_smem_bytes<D>();
     static bool configured[2] = {false, false};      // per (T, D) instantiation and slice layout
@@ -271,7 +300,7 @@ static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView
                 return CF_ERR_CUDA;
             configured[which] = true;
         }
-        kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, g->n_q_heads, g->n_kv_heads, scale_log2,
+        kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, span, g->n_q_heads, g->n_kv_heads, scale_log2,
                                                      static_cast<const T*>(q), static_cast<const T*>(k),
                                                      static_cast<const T*>(v));
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
@@ -280,38 +309,39 @@ static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView
     return run(attn_simt_kernel<T, D, CF_ROPE_INTERLEAVED>, 1);
 }
 
-int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
-                     const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
-                     cudaStream_t stream) {
+int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                     const void* q, const void* k, const void* v, float scale_log2,
+                     const AttnWorkspace& ws, cudaStream_t stream) {
     if (g->dtype == CF_BF16) {
-        if (g->head_dim == 128) return launch_simt_typed<__nv_bfloat16, 128>(g, b, pv, q, k, v, scale_log2, ws, stream);
-        return launch_simt_typed<__nv_bfloat16, 64>(g, b, pv, q, k, v, scale_log2, ws, stream);
+        if (g->head_dim == 128) return launch_simt_typed<__nv_bfloat16, 128>(g, b, pv, span, q, k, v, scale_log2, ws, stream);
+        return launch_simt_typed<__nv_bfloat16, 64>(g, b, pv, span, q, k, v, scale_log2, ws, stream);
     }
-    if (g->head_dim == 128) return launch_simt_typed<float, 128>(g, b, pv, q, k, v, scale_log2, ws, stream);
-    return launch_simt_typed<float, 64>(g, b, pv, q, k, v, scale_log2, ws, stream);
+    if (g->head_dim == 128) return launch_simt_typed<float, 128>(g, b, pv, span, q, k, v, scale_log2, ws, stream);
+    return launch_simt_typed<float, 64>(g, b, pv, span, q, k, v, scale_log2, ws, stream);
 }
 
 template <typename T, int D>
-static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const AttnWorkspace& ws, void* out,
-                                float* lse, cudaStream_t stream) {
-    const long long blocks = (long long)b->n_requests * g->n_q_heads * b->q_len;
+static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const LayerSpan& span, const AttnWorkspace& ws,
+                                void* out, float* lse, cudaStream_t stream) {
+    const long long blocks = (long long)span.n_layers * b->n_requests * g->n_q_heads * b->q_len;
     if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS || ws.n_splits > D) return CF_ERR_INVALID_ARG;
     if (ws.part_bf16)
-        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, b->n_requests, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     else
-        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, b->n_requests, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
-int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
-                   void* out, float* lse, float* doc_scores, float* score_accum, cudaStream_t stream) {
+int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                   const AttnWorkspace& ws, void* out, float* lse, float* doc_scores, float* score_accum,
+                   cudaStream_t stream) {
     int rc;
     if (g->dtype == CF_BF16)
-        rc = g->head_dim == 128 ? launch_combine_typed<__nv_bfloat16, 128>(g, b, ws, out, lse, stream)
-                                : launch_combine_typed<__nv_bfloat16, 64>(g, b, ws, out, lse, stream);
+        rc = g->head_dim == 128 ? launch_combine_typed<__nv_bfloat16, 128>(g, b, span, ws, out, lse, stream)
+                                : launch_combine_typed<__nv_bfloat16, 64>(g, b, span, ws, out, lse, stream);
     else
-        rc = g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, ws, out, lse, stream)
-                                : launch_combine_typed<float, 64>(g, b, ws, out, lse, stream);
+        rc = g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, span, ws, out, lse, stream)
+                                : launch_combine_typed<float, 64>(g, b, span, ws, out, lse, stream);
     if (rc != CF_OK) return rc;
     if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
         score_kernel<<<(unsigned)b->n_docs_total, 256, 0, stream>>>(make_batch_view(b), pv, ws,

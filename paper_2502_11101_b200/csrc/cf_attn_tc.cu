@@ -6,7 +6,7 @@
 // the softmax runs one query row per thread out of tensor memory and hands P back through tensor
 // memory (bf16, aliased onto the upper half of S).  The cache is read once.
 //
-// One CTA owns a (request, kv head, group of <=256 query rows, range of key tiles).  Two softmax
+// One CTA owns a (layer, request, kv head, group of <=256 query rows, range of key tiles).  Two softmax
 // warpgroups work side by side, each with its own S and O accumulators in tensor memory:
 //   - with more than 128 query rows in the group, warpgroup w owns row tile w and both see every
 //     key tile of the CTA's range;
@@ -107,10 +107,10 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
         : "memory");
 }
 
@@ -242,8 +242,8 @@ __device__ __forceinline__ float chunk_exp(uint32_t (&v)[32], int valid, float s
 template <int LAYOUT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-               BatchView bv, PlanView pv, AttnWorkspace ws, int n_q_heads, int n_kv_heads, float scale_log2,
-               const __nv_bfloat16* __restrict__ q) {
+               BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
+               float scale_log2, const __nv_bfloat16* __restrict__ q) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -253,11 +253,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int group = n_q_heads / n_kv_heads;
     const int lq = bv.q_len;
     const int rows = group * lq;
-    const int row_groups = (rows + 255) / 256;
-    const int b = blockIdx.z;
+    const int rg_rows = ws.rg_rows;                                 // 256, or 128 (one row tile per CTA)
+    const int row_groups = (rows + rg_rows - 1) / rg_rows;
+    const int lb = blockIdx.z;                                      // layer * B + request
+    const int layer = lb / bv.n_requests;
+    const int b = lb - layer * bv.n_requests;
+    q += (size_t)layer * q_layer_stride;
     const int kvh = blockIdx.y / row_groups;
     const int rg = blockIdx.y - kvh * row_groups;
-    const int rows_here = min(256, rows - rg * 256);
+    const int rows_here = min(rg_rows, rows - rg * rg_rows);
     const bool alternate = rows_here <= 128;                        // both warpgroups on the same rows
     const int n_qt = alternate ? 1 : 2;                             // query tiles in shared memory
     const int n_stages = kSmemTiles - n_qt;                         // 6 or 5
@@ -278,7 +282,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int t_end = (int)((long long)n_tiles * (pair + 1) / n_pairs);
     const int n_it = t_end - t_begin;                               // key tiles of this CTA
     // first workspace row of this CTA in part 2*pair
-    const size_t slot0 = ((size_t)b * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * 256;
+    const size_t slot0 = ((size_t)lb * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * rg_rows;
 
     // rows that will carry no data in one of the two parts: mark them neutral (m = -inf)
     for (int r = tid; r < rows_here; r += kThreads) {
@@ -322,8 +326,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const uint32_t dst = ring_base + st * kTileBytes;
         mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
         for (int bx = 0; bx < boxes; ++bx) {
-            tma_load_3d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, bar);
-            tma_load_3d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, bar);
+            tma_load_4d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, layer, bar);
+            tma_load_4d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, layer, bar);
         }
     };
     if (warp == 12 && lane == 0) {
@@ -342,7 +346,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             const int chunk = idx & 15, r = idx >> 4;               // r: row within the CTA's row group
             val[i] = make_uint4(0u, 0u, 0u, 0u);
             if (i < 4 * n_qt && r < rows_here) {
-                const int row = rg * 256 + r;
+                const int row = rg * rg_rows + r;
                 const int g = row / lq, j = row - g * lq;
                 const int h = kvh * group + g;
                 val[i] = __ldg(reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8));
@@ -499,7 +503,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             const uint32_t s_addr = tmem + lane_addr + w * 128;
             const uint32_t o_addr = tmem + lane_addr + 256 + w * 128;
             const bool row_valid = row_in_group < rows_here;
-            const size_t tile_row = (size_t)kvh * rows + rg * 256 + row_in_group;
+            const size_t tile_row = (size_t)kvh * rows + rg * rg_rows + row_in_group;
+            float* tile_lse2 = ws.tile_lse2 + (size_t)layer * ws.max_tiles * rows_total;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
             for (int j = 0; j < n_items; ++j) {
@@ -578,7 +583,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars->p_ready[w]));
                 l_run += tile_sum;
-                if (row_valid) ws.tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
+                if (row_valid) tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
             }
             if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (n_items - 1) & 1, abort_flag);
             if (ok) {
@@ -665,15 +670,19 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// One layer of the store as a 3-D tensor (head_dim, kv heads, rows); boxes of 64 x 1 x 32.
-int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b) {
+// The store as a 4-D tensor (head_dim, kv heads, rows, layers); boxes of 64 x 1 x 32 x 1.  Rows past
+// the end of a layer read as zero, they never reach into the next layer.
+int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return CF_ERR_CUDA;
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, (cuuint64_t)b->total_tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)b->token_stride * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kBoxRows};
-    const cuuint32_t elem[3] = {1, 1, 1};
-    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+    const cuuint64_t layer_bytes = span.n_layers > 1 ? (cuuint64_t)span.kv_stride * 2
+                                                     : (cuuint64_t)b->total_tokens * (cuuint64_t)b->token_stride * 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, (cuuint64_t)b->total_tokens,
+                                (cuuint64_t)span.n_layers};
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)b->token_stride * 2, layer_bytes};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kBoxRows, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
@@ -685,18 +694,20 @@ bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
     return g->dtype == CF_BF16 && g->head_dim == 128 && b->total_tokens > 0;
 }
 
-int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q, const void* k,
-                   const void* v, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
+int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span, const void* q,
+                   const void* k, const void* v, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
-    const int row_groups = (rows + 255) / 256;
-    if ((long long)g->n_kv_heads * row_groups > 65535 || b->n_requests > 65535 || (ws.n_splits & 1))
+    const int row_groups = (rows + ws.rg_rows - 1) / ws.rg_rows;
+    if ((long long)g->n_kv_heads * row_groups > 65535 || (long long)b->n_requests * span.n_layers > 65535 ||
+        (ws.n_splits & 1) || (ws.rg_rows != 128 && ws.rg_rows != 256))
         return CF_ERR_INVALID_ARG;
     CUtensorMap map_k, map_v;
-    int rc = make_store_map(&map_k, k, g, b);
+    int rc = make_store_map(&map_k, k, g, b, span);
     if (rc != CF_OK) return rc;
-    rc = make_store_map(&map_v, v, g, b);
+    rc = make_store_map(&map_v, v, g, b, span);
     if (rc != CF_OK) return rc;
-    dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups), (unsigned)b->n_requests);
+    dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
+              (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
     static bool configured[2] = {false, false};
     auto run = [&](auto kernel, int which) {
@@ -705,8 +716,8 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                 return CF_ERR_CUDA;
             configured[which] = true;
         }
-        kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_k, map_v, bv, pv, ws, g->n_q_heads, g->n_kv_heads,
-                                                       scale_log2, static_cast<const __nv_bfloat16*>(q));
+        kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_k, map_v, bv, pv, ws, span.q_stride, g->n_q_heads,
+                                                       g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q));
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
     if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);

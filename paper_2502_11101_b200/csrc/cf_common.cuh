@@ -58,23 +58,34 @@ BatchView make_batch_view(const cf_batch* b);
 PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan);
 int validate(const cf_geom* g, const cf_batch* b);
 int sm_count();
-int choose_splits(const cf_geom* g, const cf_batch* b);
+int choose_splits(const cf_geom* g, const cf_batch* b, int n_layers);
+int choose_row_group(const cf_geom* g, const cf_batch* b);
 int tiles_per_request_bound(const cf_batch* b);
 
 // Partial results of the attention kernels, one slice per split, merged by the combine kernel.
 // All logits are in base-2 units: t = (q.k) * softmax_scale * log2(e).
+// A call covers n_layers layers; (layer, request) pairs are numbered lb = layer * B + request.
 struct AttnWorkspace {
-    float* part_o;     // [B][n_splits][Hq*Lq][D]   sum_t 2^(t - m) v_t, not normalised (unset if m = -inf);
+    float* part_o;     // [L*B][n_splits][Hq*Lq][D] sum_t 2^(t - m) v_t, not normalised (unset if m = -inf);
                        //                           fp32, or bf16 in the same index order when part_bf16 is set
-    float* part_m;     // [B][n_splits][Hq*Lq]      reference maximum m (-inf if the part is empty)
-    float* part_l;     // [B][n_splits][Hq*Lq]      sum_t 2^(t - m)
-    float* tile_lse2;  // [max_tiles][Hq*Lq]        log2 of sum over the tile's tokens of 2^t
-    float* row_lse2;   // [B][Hq*Lq]                log2 of the full softmax denominator
+    float* part_m;     // [L*B][n_splits][Hq*Lq]    reference maximum m (-inf if the part is empty)
+    float* part_l;     // [L*B][n_splits][Hq*Lq]    sum_t 2^(t - m)
+    float* tile_lse2;  // [L][max_tiles][Hq*Lq]     log2 of sum over the tile's tokens of 2^t
+    float* row_lse2;   // [L*B][Hq*Lq]              log2 of the full softmax denominator
     int n_splits;
     int part_bf16;     // the tensor-core kernel stores its partial O rows as bf16
+    int n_layers;
+    int max_tiles;     // tile slots per layer in tile_lse2
+    int rg_rows;       // query rows per CTA of the tensor-core kernel: 256 (two row tiles) or 128
 };
-size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, AttnWorkspace* ws,
-                             void* base);
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers,
+                             AttnWorkspace* ws, void* base);
+
+// Where the layers of a call sit (element strides between consecutive layers).
+struct LayerSpan {
+    int n_layers;
+    long long q_stride, kv_stride, out_stride;
+};
 
 // ---- launchers (each returns a CF_* code) -------------------------------------------------
 int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
@@ -82,16 +93,21 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream);
 int launch_reposition(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers,
                       long long layer_stride, const void* k_in, void* k_out, cudaStream_t stream);
-int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
-                     const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
-                     cudaStream_t stream);
-int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const void* q,
-                   const void* k, const void* v, float scale_log2, const AttnWorkspace& ws,
-                   cudaStream_t stream);
+int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                     const void* q, const void* k, const void* v, float scale_log2,
+                     const AttnWorkspace& ws, cudaStream_t stream);
+int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                   const void* q, const void* k, const void* v, float scale_log2,
+                   const AttnWorkspace& ws, cudaStream_t stream);
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b);
-int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws,
-                   void* out, float* lse, float* doc_scores, float* score_accum,
-                   cudaStream_t stream);
+int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
+                   const AttnWorkspace& ws, void* out, float* lse, float* doc_scores,
+                   float* score_accum, cudaStream_t stream);
+// Shared body of the attention entry points.
+int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan, const LayerSpan& span,
+                    const void* q, const void* k_cache, const void* v_cache, float softmax_scale,
+                    void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
+                    size_t workspace_bytes, cudaStream_t stream);
 
 // ---- device helpers -----------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float x) { return x; }

@@ -7,7 +7,6 @@
 
 namespace cf {
 
-int attn_path();   // cf_api.cu: 0 = automatic, 1 = CUDA-core kernel forced
 
 // The scratch itself.  Every GPU that loads this library holds these bytes until the process
 // exits.  In host code `g_static_scratch` is only a handle: the device address comes from
@@ -43,28 +42,14 @@ extern "C" int cf_query_prefill_attn_static(const cf_geom* geom, const cf_batch*
     if (!batch || !plan) return CF_ERR_INVALID_ARG;
     int rc = validate(geom, batch);
     if (rc != CF_OK) return rc;
-    if (reinterpret_cast<uintptr_t>(plan) % 256 != 0) return CF_ERR_WORKSPACE;
-    if (!q || !k_cache || !v_cache || !out) return CF_ERR_INVALID_ARG;
-    if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return CF_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(q) % 16 || reinterpret_cast<uintptr_t>(out) % 16 ||
-        reinterpret_cast<uintptr_t>(k_cache) % 16 || reinterpret_cast<uintptr_t>(v_cache) % 16)
-        return CF_ERR_INVALID_ARG;
-    const int n_splits = choose_splits(geom, batch);
-    if (attn_workspace_layout(geom, batch, n_splits, nullptr, nullptr) > (size_t)CF_STATIC_WORKSPACE_BYTES)
+    if (attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), 1, nullptr, nullptr) >
+        (size_t)CF_STATIC_WORKSPACE_BYTES)
         return CF_ERR_WORKSPACE;            // this batch needs more scratch than the library carries
     void* scratch = nullptr;
     rc = static_scratch_address(&scratch);
     if (rc != CF_OK) return rc;
-    AttnWorkspace ws;
-    attn_workspace_layout(geom, batch, n_splits, &ws, scratch);
-    const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
-    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (attn_path() == 0 && attn_tc_supported(geom, batch)) {
-        ws.part_bf16 = 1;
-        rc = launch_attn_tc(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    } else
-        rc = launch_attn_simt(geom, batch, pv, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    if (rc != CF_OK) return rc;
-    return launch_combine(geom, batch, pv, ws, out, lse, doc_scores, score_accum, s);
+    const LayerSpan span = {1, 0, 0, 0};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
+                           score_accum, scratch, (size_t)CF_STATIC_WORKSPACE_BYTES,
+                           static_cast<cudaStream_t>(stream));
 }

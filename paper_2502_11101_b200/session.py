@@ -39,8 +39,8 @@ class Session:
         self.layout = B.cf_plan_layout_of(self.geom, self.batch)
         self.plan = torch.zeros(self.layout.total_bytes, dtype=torch.uint8, device=self.device)
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()) if self.n_requests else 0)
-        self.workspace = torch.empty(max(256, B.cf_attn_workspace_bytes(self.geom, self.batch)), dtype=torch.uint8,
-                                     device=self.device)
+        self.workspace = torch.empty(256, dtype=torch.uint8, device=self.device)
+        self.reserve_workspace(1)
         self.doc_scores = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
         self.score_accum = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
 
@@ -54,6 +54,13 @@ class Session:
             worst = max(worst, int(tiles[:kept_per_request].sum()))
         self.batch.tiles_hint = worst
 
+    def reserve_workspace(self, n_layers: int) -> None:
+        """Grow the attention workspace to what a call over `n_layers` layers needs with the current
+        live-document hint (allocation happens here, never inside a library call)."""
+        need = B.cf_attn_workspace_bytes_layers(self.geom, self.batch, n_layers)
+        if need > self.workspace.numel():
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+
     def init(self, order: Optional[torch.Tensor] = None, kept_count: Optional[torch.Tensor] = None,
              query_start: int = -1) -> None:
         self.score_accum.zero_()
@@ -63,6 +70,15 @@ class Session:
                lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0) -> None:
         B.cf_query_prefill_attn(self.geom, self.batch, self.plan, q, k_layer, v_layer, out, self.workspace, lse,
                                 self.doc_scores, self.score_accum, softmax_scale)
+
+    def attend_layers(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                      lse: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
+                      softmax_scale: float = 0.0) -> None:
+        """Consecutive layers that attend the same kept documents, in one library call: q, out
+        [m, B, Lq, Hq, D]; k, v [m, T, Hkv, D]; lse [m, B, Hq, Lq]; layer_scores [m, n_docs_total]."""
+        self.reserve_workspace(q.shape[0])
+        B.cf_query_prefill_attn_layers(self.geom, self.batch, self.plan, q, k, v, out, self.workspace, lse,
+                                       layer_scores, self.score_accum, softmax_scale)
 
     def prune(self, keep: int, strategy: int) -> None:
         B.cf_prune_topk(self.geom, self.batch, self.plan, self.score_accum, keep, strategy)
@@ -90,19 +106,35 @@ class Session:
 
     def run_stack(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, schedule: Sequence[Tuple[int, int]],
                   strategy: int, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
-                  k_final: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None) -> None:
+                  k_final: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
+                  batch_layers: bool = False) -> None:
         """Algorithm 2, Phases 1 and 2, as library calls: q, out [L, B, Lq, Hq, D]; k, v [L, T, Hkv, D];
-        lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores."""
+        lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores.
+
+        With `batch_layers` the layers between two pruning layers go to the library in one call
+        (possible here because every layer's query states are given up front)."""
         sched = dict(schedule)
         n_layers = q.shape[0]
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))
         self.init()
-        for layer in range(1, n_layers + 1):
-            i = layer - 1
-            self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
-            if layer_scores is not None:
-                layer_scores[i].copy_(self.doc_scores)
-            if layer in sched:
-                self.prune(sched[layer], strategy)
+        if batch_layers:
+            cuts = sorted(l for l in sched if l < n_layers) + [n_layers]
+            first = 0
+            for last in cuts:                               # layers first+1 .. last (1-based) share one plan
+                for lo in range(first, last, B.CF_MAX_LAYERS_PER_CALL):
+                    hi = min(last, lo + B.CF_MAX_LAYERS_PER_CALL)
+                    self.attend_layers(q[lo:hi], k[lo:hi], v[lo:hi], out[lo:hi], None if lse is None else lse[lo:hi],
+                                       None if layer_scores is None else layer_scores[lo:hi])
+                if last in sched:
+                    self.prune(sched[last], strategy)
+                first = last
+        else:
+            for layer in range(1, n_layers + 1):
+                i = layer - 1
+                self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
+                if layer_scores is not None:
+                    layer_scores[i].copy_(self.doc_scores)
+                if layer in sched:
+                    self.prune(sched[layer], strategy)
         if k_final is not None:
             self.reposition(k, k_final, n_layers, k.stride(0))

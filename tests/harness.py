@@ -57,7 +57,7 @@ def cut_margins(meta: W.WorkloadMeta, ref: List[Dict], strategy: int, schedule=N
 
 
 def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, device="cuda:0", n_reuse: int = 0,
-              with_final: bool = True):
+              with_final: bool = True, batch_layers: bool = False):
     from paper_2502_11101_b200.session import Session
     cfg = meta.cfg
     sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
@@ -70,7 +70,7 @@ def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, devic
     scores = torch.full((n_layers, meta.n_docs_total), float("nan"), device=device)
     k_final = kg.clone() if with_final else None
     sched = cfg.schedule if schedule is None else schedule
-    sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores)
+    sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores, batch_layers=batch_layers)
     torch.cuda.synchronize()
     status = sess.status()
     return {"out": out.float().cpu().numpy(), "lse": lse.cpu().numpy(), "scores": scores.cpu().numpy(),
@@ -143,14 +143,14 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
 
 
 def run_and_compare(cfg: W.WorkloadConfig, seed: int, strategy: int, device="cuda:0", n_reuse: int = 0,
-                    min_margin: float = 2e-3, doc_len_override=None) -> Dict[str, float]:
+                    min_margin: float = 2e-3, doc_len_override=None, batch_layers: bool = False) -> Dict[str, float]:
     meta = W.make_meta(cfg, seed, doc_len_override)
     q = W.make_q(meta)
     k, v = W.make_kv(meta)
     ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse)
     margin = cut_margins(meta, ref, strategy)
     assert margin >= min_margin, f"workload rejected: decisive score gap {margin:.2e} below {min_margin:.0e}"
-    got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse)
+    got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse, batch_layers=batch_layers)
     report = compare(meta, ref, got, k)
     report["margin"] = margin
     return report

@@ -102,6 +102,7 @@ def test_results_are_bitwise_reproducible():
     ((4, 4), 16, [40, 128, 7]),                            # ragged tiles
     ((12, 2), 48, [130, 160, 192, 128, 150]),              # two row tiles (288 rows), two-tile documents
     ((28, 4), 64, [128, 192, 161, 140, 177, 133]),         # 448 rows: two row groups per kv head
+    ((20, 2), 60, [130, 160, 128]),                        # 600 rows: five row tiles, one per CTA
 ])
 def test_tensor_core_kernel_matches_cuda_core_kernel(heads, q_len, lens):
     """Same inputs through both attention kernels of the library."""
@@ -130,6 +131,67 @@ def test_tensor_core_kernel_matches_cuda_core_kernel(heads, q_len, lens):
     assert torch.all((o_a - o_b).abs() <= 1e-2 + 2e-2 * o_a.abs()), float((o_a - o_b).abs().max())
     assert torch.all((l_a - l_b).abs() <= 1e-3), float((l_a - l_b).abs().max())
     assert torch.all((s_a - s_b).abs() <= 1e-3 * s_a.abs() + 1e-6)
+
+
+@pytest.mark.parametrize("which", ["config3", "config4-reduced", "ragged-f32-d64", "ragged-bf16-d64"])
+def test_layer_batched_calls_match_oracle(which):
+    """Layers between two pruning layers in one library call (cf_query_prefill_attn_layers)."""
+    if which == "config3":                                 # segments of 4, 8, 8 and 8 layers
+        cfg = W.CONFIGS[3]
+    elif which == "config4-reduced":                       # two requests x segments of 2, 2 and 1 layers
+        cfg = W.scaled_config(W.CONFIGS[4], n_layers=5, batch=2, schedule=((2, 50), (4, 25)))
+    else:                                                  # CUDA-core kernel, ragged tiles, segments of 3 and 2
+        lens = [1, 63, 64, 65, 127, 128, 129, 200, 300, 17, 256, 31]
+        dtype = "f32" if "f32" in which else "bf16"
+        cfg = W.WorkloadConfig("ragged", 5, 8, 2, 64, dtype, 1e4, 4096, len(lens), 1, 300, 5, 1, 2, ((3, 7),))
+        harness.run_and_compare(cfg, 1, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=1e-3, batch_layers=True)
+        return
+    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3,
+                            batch_layers=True)
+
+
+def test_layer_batched_call_is_reproducible_and_agrees_with_single_layer_calls():
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[3], n_layers=3, n_docs=20, schedule=())
+    meta = W.make_meta(cfg, 0)
+    q = W.make_q(meta).cuda()
+    k, v = [t.cuda() for t in W.make_kv(meta)]
+    # the store with a gap between layers: the layer stride is an argument of its own
+    pad = 24
+    k_wide = torch.zeros((3, meta.total_tokens + pad, cfg.n_kv_heads, 128), dtype=torch.bfloat16, device="cuda")
+    v_wide = torch.zeros_like(k_wide)
+    k_wide[:, :meta.total_tokens] = k
+    v_wide[:, :meta.total_tokens] = v
+    runs = []
+    for mode in ("layers", "layers", "layers-strided", "single"):
+        sess = Session(cfg.n_q_heads, cfg.n_kv_heads, 128, torch.bfloat16, cfg.pos_range, cfg.rope_theta, cfg.q_len,
+                       meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+        sess.init()
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((3, 1, cfg.n_q_heads, cfg.q_len), float("nan"), device="cuda")
+        scores = torch.full((3, meta.n_docs_total), float("nan"), device="cuda")
+        if mode == "layers":
+            sess.attend_layers(q, k, v, out, lse, scores)
+        elif mode == "layers-strided":
+            sess.attend_layers(q, k_wide[:, :meta.total_tokens], v_wide[:, :meta.total_tokens], out, lse, scores)
+        else:
+            for i in range(3):
+                sess.attend(q[i], k[i], v[i], out[i], lse[i])
+                scores[i].copy_(sess.doc_scores)
+        torch.cuda.synchronize()
+        assert sess.status() == 0
+        runs.append([t.float().cpu() for t in (out, lse, scores, sess.score_accum)])
+    for a, b in zip(runs[0], runs[1]):
+        assert torch.equal(a, b)                                        # run to run
+    for a, b in zip(runs[0], runs[2]):
+        assert torch.equal(a, b)                                        # a layer stride changes nothing
+    o_a, l_a, s_a, acc_a = runs[0]
+    o_b, l_b, s_b, acc_b = runs[3]
+    assert torch.all((o_a - o_b).abs() <= 1e-2 + 2e-2 * o_b.abs())
+    assert torch.all((l_a - l_b).abs() <= 1e-3)
+    assert torch.all((s_a - s_b).abs() <= 1e-3 * s_b.abs() + 1e-6)
+    assert torch.allclose(acc_a, s_a.sum(0), rtol=1e-5) and torch.allclose(acc_a, acc_b, rtol=1e-3)
 
 
 def test_interleaved_slice_layout():
@@ -200,6 +262,16 @@ def test_argument_errors_are_reported_not_faulted():
     with pytest.raises(cf.CacheFocusError) as e:
         cf.cf_plan_init(sess.geom, sess.batch, small)
     assert e.value.code == cf.CF_ERR_WORKSPACE
+    q3, k3, v3 = q[:1].expand(3, *q.shape[1:]), k[:1].expand(3, *k.shape[1:]), v[:1].expand(3, *v.shape[1:])
+    out3 = torch.empty((3,) + tuple(out.shape), dtype=out.dtype, device="cuda")
+    with pytest.raises(cf.CacheFocusError) as e:             # layers that overlap (stride 0)
+        cf.cf_query_prefill_attn_layers(sess.geom, sess.batch, sess.plan, q3, k3, v3, out3, sess.workspace)
+    assert e.value.code == cf.CF_ERR_INVALID_ARG
+    with pytest.raises(cf.CacheFocusError) as e:
+        cf.cf_query_prefill_attn_layers(sess.geom, sess.batch, sess.plan, q3.contiguous(), k3.contiguous(),
+                                        v3.contiguous(), out3, small)
+    assert e.value.code == cf.CF_ERR_WORKSPACE
+    assert cf.cf_attn_workspace_bytes_layers(sess.geom, sess.batch, cf.CF_MAX_LAYERS_PER_CALL + 1) == 0
     bad = cf.make_geom(5, 2, 128, cf.CF_BF16, 4096, 1e4)
     with pytest.raises(cf.CacheFocusError) as e:
         cf.cf_plan_layout_of(bad, sess.batch)
