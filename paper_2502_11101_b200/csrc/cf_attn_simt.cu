@@ -155,90 +155,128 @@ attn_simt_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, LayerSpan span, in
     }
 }
 
-// Merge the parts of one query row (one block per row, one thread per output dimension):
+// D/32 consecutive elements of a partial O row (fp32 or bf16) as floats.
+template <int V>
+__device__ __forceinline__ void load_part(const float* p, float (&x)[V]) {
+    if (V == 4) {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        x[0] = t.x; x[1] = t.y; x[V - 2] = t.z; x[V - 1] = t.w;
+    } else {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        x[0] = t.x; x[1] = t.y;
+    }
+}
+template <int V>
+__device__ __forceinline__ void load_part(const __nv_bfloat16* p, float (&x)[V]) {
+    if (V == 4) {
+        const uint2 t = *reinterpret_cast<const uint2*>(p);
+        x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xffff0000u);
+        x[V - 2] = __uint_as_float(t.y << 16); x[V - 1] = __uint_as_float(t.y & 0xffff0000u);
+    } else {
+        const uint32_t t = *reinterpret_cast<const uint32_t*>(p);
+        x[0] = __uint_as_float(t << 16); x[1] = __uint_as_float(t & 0xffff0000u);
+    }
+}
+template <int V>
+__device__ __forceinline__ void store_row(float* p, const float (&x)[V]) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) p[i] = x[i];
+}
+template <int V>
+__device__ __forceinline__ void store_row(__nv_bfloat16* p, const float (&x)[V]) {
+#pragma unroll
+    for (int i = 0; i < V; i += 2)
+        *reinterpret_cast<__nv_bfloat162*>(p + i) = __floats2bfloat162_rn(x[i], x[i + 1]);
+}
+
+constexpr int kCombineRows = 8;       // query rows (warps) per block of the merge kernel
+
+// Merge the parts of one query row (one warp per row, D/32 output dimensions per lane):
 // out = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m), and the row's log-sum-exp.
-// Parts are visited in index order, so the result does not depend on scheduling.
+// Parts are visited in index order and the warp reductions have a fixed shape, so the result does
+// not depend on scheduling.
 template <typename T, int D, typename P>
-__global__ void __launch_bounds__(D)
-combine_kernel(AttnWorkspace ws, int n_requests, long long out_layer_stride, int n_q_heads, int lq,
-               T* __restrict__ out, float* __restrict__ lse) {
-    __shared__ float s_w[CF_MAX_SPLITS];
-    __shared__ float s_red[2][D / 32];
+__global__ void __launch_bounds__(32 * kCombineRows)
+combine_kernel(AttnWorkspace ws, int n_requests, long long n_rows_all, long long out_layer_stride, int n_q_heads,
+               int lq, T* __restrict__ out, float* __restrict__ lse) {
+    constexpr int V = D / 32;
+    static_assert(CF_MAX_SPLITS <= 64, "two parts per lane");
+    const int lane = threadIdx.x & 31;
+    const long long row_all = (long long)blockIdx.x * kCombineRows + (threadIdx.x >> 5);
+    if (row_all >= n_rows_all) return;
     const int rows_total = n_q_heads * lq;
-    const int lb = blockIdx.x / rows_total, rg = blockIdx.x - lb * rows_total;   // lb = layer * B + request
+    const int lb = (int)(row_all / rows_total), rg = (int)(row_all - (long long)lb * rows_total);   // lb = layer * B + request
     const int layer = lb / n_requests, b = lb - layer * n_requests;
     const int h = rg / lq, j = rg - h * lq;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_parts = ws.n_splits;
     const size_t slot0 = (size_t)lb * n_parts * rows_total + rg;      // part p sits at slot0 + p * rows_total
 
-    float m = -INFINITY, l = 0.f;
-    if (tid < n_parts) {
-        m = ws.part_m[slot0 + (size_t)tid * rows_total];
-        l = m > -INFINITY ? ws.part_l[slot0 + (size_t)tid * rows_total] : 0.f;
+    float m[2], l[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int p = lane + 32 * k;
+        m[k] = p < n_parts ? ws.part_m[slot0 + (size_t)p * rows_total] : -INFINITY;
+        l[k] = m[k] > -INFINITY ? ws.part_l[slot0 + (size_t)p * rows_total] : 0.f;
     }
-    float m_max = m;
+    float m_max = fmaxf(m[0], m[1]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m_max = fmaxf(m_max, __shfl_xor_sync(0xffffffffu, m_max, o));
-    if (lane == 0) s_red[0][warp] = m_max;
-    __syncthreads();
-    m_max = s_red[0][0];
+    float w[2];
 #pragma unroll
-    for (int k = 1; k < D / 32; ++k) m_max = fmaxf(m_max, s_red[0][k]);
-    const float w = m > -INFINITY ? exp2f(m - m_max) : 0.f;
-    if (tid < n_parts) s_w[tid] = w;
-    float l_sum = l * w;                                               // fixed-shape tree: deterministic
+    for (int k = 0; k < 2; ++k) w[k] = m[k] > -INFINITY ? exp2f(m[k] - m_max) : 0.f;
+    float l_sum = fmaf(l[1], w[1], l[0] * w[0]);                      // fixed-shape tree: deterministic
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) l_sum += __shfl_xor_sync(0xffffffffu, l_sum, o);
-    if (lane == 0) s_red[1][warp] = l_sum;
-    __syncthreads();
-    l_sum = s_red[1][0];
-#pragma unroll
-    for (int k = 1; k < D / 32; ++k) l_sum += s_red[1][k];
 
-    float acc = 0.f;
-    const P* po = reinterpret_cast<const P*>(ws.part_o) + slot0 * D + tid;
+    float acc[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = 0.f;
+    const P* po = reinterpret_cast<const P*>(ws.part_o) + slot0 * D + lane * V;
     const size_t stride = (size_t)rows_total * D;
-    int p = 0;
-    for (; p + 4 <= n_parts; p += 4) {                                 // independent loads in flight
-        const float w0 = s_w[p], w1 = s_w[p + 1], w2 = s_w[p + 2], w3 = s_w[p + 3];
-        const float o0 = w0 > 0.f ? to_float(po[(size_t)p * stride]) : 0.f;
-        const float o1 = w1 > 0.f ? to_float(po[(size_t)(p + 1) * stride]) : 0.f;
-        const float o2 = w2 > 0.f ? to_float(po[(size_t)(p + 2) * stride]) : 0.f;
-        const float o3 = w3 > 0.f ? to_float(po[(size_t)(p + 3) * stride]) : 0.f;
-        acc = fmaf(o0, w0, acc);
-        acc = fmaf(o1, w1, acc);
-        acc = fmaf(o2, w2, acc);
-        acc = fmaf(o3, w3, acc);
-    }
-    for (; p < n_parts; ++p) {
-        const float wp = s_w[p];
-        if (wp > 0.f) acc = fmaf(to_float(po[(size_t)p * stride]), wp, acc);
+    for (int p0 = 0; p0 < n_parts; p0 += 4) {                         // four independent loads in flight
+        float wp[4], x[4][V];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int p = p0 + u;
+            wp[u] = __shfl_sync(0xffffffffu, (p & 32) ? w[1] : w[0], p & 31);
+            if (p >= n_parts) wp[u] = 0.f;
+            if (wp[u] > 0.f) load_part<V>(po + (size_t)p * stride, x[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (wp[u] > 0.f) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] = fmaf(x[u][i], wp[u], acc[i]);
+            }
     }
     const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-    out[(size_t)layer * out_layer_stride + (((size_t)b * lq + j) * n_q_heads + h) * D + tid] = from_float<T>(acc * inv);
-    if (tid == 0) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] *= inv;
+    store_row<V>(out + (size_t)layer * out_layer_stride + (((size_t)b * lq + j) * n_q_heads + h) * D + lane * V, acc);
+    if (lane == 0) {
         const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
         ws.row_lse2[(size_t)lb * rows_total + rg] = lse2;
         if (lse) lse[(size_t)lb * rows_total + rg] = lse2 * kLn2;
     }
 }
 
+constexpr int kScoreThreads = 1024;
+
 // Document scores (footnote of Sec. 2.4; Algorithm 2: S <- S + s^l): one block per document sums
 // 2^(tile_lse - row_lse) over the document's tiles and all query rows of every layer of the call,
 // each layer in a fixed order, then adds the layers' scores to S in layer order.  Up to eight
 // layers are reduced side by side by groups of threads.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kScoreThreads)
 score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float* __restrict__ doc_scores,
              float* __restrict__ score_accum) {
-    __shared__ float s_red[256];
+    __shared__ float s_red[kScoreThreads / 32];
     __shared__ float s_layer[CF_MAX_LAYERS_PER_CALL];
     const int doc = blockIdx.x;
     const int n_layers = ws.n_layers;
     const int count = pv.doc_tile_count[doc];
     if (count == 0) {
         if (doc_scores)
-            for (int l = threadIdx.x; l < n_layers; l += 256) doc_scores[(size_t)l * bv.n_docs_total + doc] = 0.f;
+            for (int l = threadIdx.x; l < n_layers; l += kScoreThreads) doc_scores[(size_t)l * bv.n_docs_total + doc] = 0.f;
         return;
     }
     int lo = 0, hi = bv.n_requests;                 // request that owns the document
@@ -248,28 +286,31 @@ score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float*
     }
     int groups = 1;                                 // power of two, at most min(n_layers, 8)
     while (groups * 2 <= n_layers && groups < 8) groups *= 2;
-    const int gs = 256 / groups;
+    const int gs = kScoreThreads / groups;          // threads per group, a multiple of 128
     const int g = threadIdx.x / gs, t = threadIdx.x - g * gs;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int warps_per_group = gs >> 5;
     const int rounds = (n_layers + groups - 1) / groups;
     const size_t tile0 = (size_t)pv.doc_tile_begin[doc];
+    const int n = count * rows_total;
     for (int rd = 0; rd < rounds; ++rd) {
         const int layer = rd * groups + g;
         float sum = 0.f;
         if (layer < n_layers) {
-            const float* row_lse2 = ws.row_lse2 + ((size_t)layer * bv.n_requests + lo) * rows_total;
-            const float* tile_lse2 = ws.tile_lse2 + ((size_t)layer * ws.max_tiles + tile0) * rows_total;
-            for (int idx = t; idx < count * rows_total; idx += gs) {
-                const int rg = idx % rows_total;
-                sum += exp2f(tile_lse2[idx] - row_lse2[rg]);
-            }
+            const float* __restrict__ row_lse2 = ws.row_lse2 + ((size_t)layer * bv.n_requests + lo) * rows_total;
+            const float* __restrict__ tile_lse2 = ws.tile_lse2 + ((size_t)layer * ws.max_tiles + tile0) * rows_total;
+#pragma unroll 4
+            for (int idx = t; idx < n; idx += gs) sum += exp2f(tile_lse2[idx] - row_lse2[idx % rows_total]);
         }
-        s_red[threadIdx.x] = sum;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) s_red[warp] = sum;
         __syncthreads();
-        for (int w = gs >> 1; w > 0; w >>= 1) {
-            if (t < w) s_red[threadIdx.x] += s_red[threadIdx.x + w];
-            __syncthreads();
+        if (t == 0 && layer < n_layers) {
+            float total = 0.f;
+            for (int k = 0; k < warps_per_group; ++k) total += s_red[g * warps_per_group + k];
+            s_layer[layer] = total / (float)rows_total;
         }
-        if (t == 0 && layer < n_layers) s_layer[layer] = s_red[threadIdx.x] / (float)rows_total;
         __syncthreads();
     }
     if (threadIdx.x == 0) {
@@ -323,12 +364,15 @@ int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, co
 template <typename T, int D>
 static int launch_combine_typed(const cf_geom* g, const cf_batch* b, const LayerSpan& span, const AttnWorkspace& ws,
                                 void* out, float* lse, cudaStream_t stream) {
-    const long long blocks = (long long)span.n_layers * b->n_requests * g->n_q_heads * b->q_len;
-    if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS || ws.n_splits > D) return CF_ERR_INVALID_ARG;
+    const long long rows_all = (long long)span.n_layers * b->n_requests * g->n_q_heads * b->q_len;
+    const long long blocks = (rows_all + kCombineRows - 1) / kCombineRows;
+    if (blocks > 0x7fffffffLL || ws.n_splits > CF_MAX_SPLITS) return CF_ERR_INVALID_ARG;
     if (ws.part_bf16)
-        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, D, 0, stream>>>(ws, b->n_requests, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+        combine_kernel<T, D, __nv_bfloat16><<<(unsigned)blocks, 32 * kCombineRows, 0, stream>>>(
+            ws, b->n_requests, rows_all, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     else
-        combine_kernel<T, D, float><<<(unsigned)blocks, D, 0, stream>>>(ws, b->n_requests, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
+        combine_kernel<T, D, float><<<(unsigned)blocks, 32 * kCombineRows, 0, stream>>>(
+            ws, b->n_requests, rows_all, span.out_stride, g->n_q_heads, b->q_len, static_cast<T*>(out), lse);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -344,7 +388,7 @@ int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                                 : launch_combine_typed<float, 64>(g, b, span, ws, out, lse, stream);
     if (rc != CF_OK) return rc;
     if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
-        score_kernel<<<(unsigned)b->n_docs_total, 256, 0, stream>>>(make_batch_view(b), pv, ws,
+        score_kernel<<<(unsigned)b->n_docs_total, kScoreThreads, 0, stream>>>(make_batch_view(b), pv, ws,
                                                                    g->n_q_heads * b->q_len, doc_scores,
                                                                    score_accum);
         if (cudaGetLastError() != cudaSuccess) return CF_ERR_CUDA;

@@ -8,21 +8,28 @@
 namespace cf {
 
 constexpr int kPlanThreads = 256;
+static_assert(4 * kPlanThreads >= kMaxDocs, "the tile scan gives four ranks to every thread");
 
 __device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
 // mode 0: initialise from (order, kept_count); mode 1: prune by score, then rebuild.
+// Everything a later step needs from global memory is staged in shared memory at the start, so
+// the steps below do not each wait for a round trip of their own.
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restrict__ order,
             const int* __restrict__ kept_count_in, int query_start_arg,
             const float* __restrict__ score_accum, int keep, const int* __restrict__ keep_per_request,
             int strategy) {
     __shared__ int s_ids[kMaxDocs];       // kept local ids by rank
-    __shared__ int s_tmp[kMaxDocs];       // new order / per-rank tile counts / window cursors
+    __shared__ int s_tmp[kMaxDocs];       // new order, then the first tile of every rank
+    __shared__ int s_row[kMaxDocs + 1];   // first store row of every document (by local id), and the end
+    __shared__ int s_dst[kMaxDocs];       // start positions by local id
+    __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
     __shared__ float s_score[kMaxDocs];
     __shared__ unsigned char s_flag[kMaxDocs];
     __shared__ double s_inv_freq[64];
-    __shared__ int s_longest, s_min_cursor;
+    __shared__ int s_longest, s_min_cursor, s_fail;
+    __shared__ int s_warp_sum[kPlanThreads / 32];
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
@@ -38,15 +45,9 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
         return;
     }
     const int half = gv.head_dim / 2;
-    for (int p = tid; p < half; p += kPlanThreads)
-        s_inv_freq[p] = pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
-    if (tid == 0) {
-        s_longest = 0;
-        s_min_cursor = 0x7fffffff;
-    }
 
-    // ---- the kept list, in rank order -------------------------------------------------------
-    int n_kept;
+    // ---- stage the inputs -------------------------------------------------------------------
+    int n_old = 0, keep_b = 0, n_kept = 0;
     if (mode == 0) {
         n_kept = kept_count_in ? kept_count_in[b] : n_docs;
         n_kept = max(0, min(n_kept, n_docs));
@@ -58,24 +59,43 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
             }
             s_ids[r] = id;
         }
-        __syncthreads();
     } else {
-        const int n_old = max(0, min(pv.kept_count[b], n_docs));
-        int keep_b = keep_per_request ? keep_per_request[b] : keep;
+        n_old = max(0, min(pv.kept_count[b], n_docs));
+        keep_b = keep_per_request ? keep_per_request[b] : keep;
         keep_b = max(0, min(keep_b, n_old));
         for (int r = tid; r < n_old; r += kPlanThreads) {
-            s_ids[r] = pv.kept[doc0 + r];
-            s_score[r] = score_accum[doc0 + s_ids[r]];
+            const int id = max(0, min(pv.kept[doc0 + r], n_docs - 1));
+            s_ids[r] = id;
+            s_score[r] = score_accum[doc0 + id];
         }
-        __syncthreads();
+    }
+    for (int i = tid; i <= n_docs; i += kPlanThreads) s_row[i] = bv.doc_offsets[doc0 + i];
+    for (int i = tid; i < n_docs; i += kPlanThreads) {
+        s_src[i] = bv.doc_src_start[doc0 + i];
+        s_dst[i] = mode == 0 ? -1 : pv.dst_start[doc0 + i];
+    }
+    int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
+                                : pv.query_start[b];
+    int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
+    for (int p = tid; p < half; p += kPlanThreads)
+        s_inv_freq[p] = pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
+    if (tid == 0) {
+        s_longest = 0;
+        s_min_cursor = 0x7fffffff;
+        s_fail = 0;
+    }
+    __syncthreads();
+
+    // ---- the kept list, in rank order -------------------------------------------------------
+    if (mode != 0) {
         // rank by counting: how many kept documents beat this one (ties: lower id wins)
         for (int r = tid; r < n_old; r += kPlanThreads) {
-            const float s = s_score[r];
+            const float sc = s_score[r];
             const int id = s_ids[r];
             int better = 0;
             for (int o = 0; o < n_old; ++o) {
                 const float so = s_score[o];
-                better += (so > s) || (so == s && s_ids[o] < id);
+                better += (so > sc) || (so == sc && s_ids[o] < id);
             }
             s_flag[r] = better < keep_b;
             if (strategy == CF_ALLOC_SORT && better < keep_b) s_tmp[better] = id;
@@ -113,15 +133,9 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
     }
 
     // ---- positional allocation ----------------------------------------------------------------
-    int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
-                                : pv.query_start[b];
-    int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
     if (reallocate && n_kept > 0) {
         int longest = 0;
-        for (int r = tid; r < n_kept; r += kPlanThreads) {
-            const int i = doc0 + s_ids[r];
-            longest = max(longest, bv.doc_offsets[i + 1] - bv.doc_offsets[i]);
-        }
+        for (int r = tid; r < n_kept; r += kPlanThreads) longest = max(longest, s_row[s_ids[r] + 1] - s_row[s_ids[r]]);
         atomicMax(&s_longest, longest);
         __syncthreads();
         longest = s_longest;
@@ -140,10 +154,11 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
         for (int w = tid; w < windows && w < n_kept; w += kPlanThreads) {
             int cursor = query_start;
             for (int r = w; r < n_kept; r += windows) {
-                const int i = doc0 + s_ids[r];
-                cursor -= bv.doc_offsets[i + 1] - bv.doc_offsets[i];
-                pv.dst_start[i] = cursor;
-                pv.group[i] = w;
+                const int id = s_ids[r];
+                cursor -= s_row[id + 1] - s_row[id];
+                s_dst[id] = cursor;
+                pv.dst_start[doc0 + id] = cursor;
+                pv.group[doc0 + id] = w;
             }
             atomicMin(&s_min_cursor, cursor);
         }
@@ -153,38 +168,56 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
     }
 
     // ---- key tiles: document-aligned runs of at most kTile rows -------------------------------
-    for (int r = tid; r < n_kept; r += kPlanThreads) {
-        const int i = doc0 + s_ids[r];
-        s_tmp[r] = (bv.doc_offsets[i + 1] - bv.doc_offsets[i] + kTile - 1) / kTile;
+    // exclusive prefix sum of the per-rank tile counts: four consecutive ranks per thread
+    int cnt[4], local = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = 4 * tid + k;
+        cnt[k] = r < n_kept ? (s_row[s_ids[r] + 1] - s_row[s_ids[r]] + kTile - 1) / kTile : 0;
+        local += cnt[k];
     }
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((tid & 31) >= o) incl += up;
+    }
+    if ((tid & 31) == 31) s_warp_sum[tid >> 5] = incl;
     __syncthreads();
-    const int base = tile_base(doc0, bv.doc_offsets[doc0]);
+    int run = incl - local, total = 0;
+    for (int w = 0; w < kPlanThreads / 32; ++w) {
+        if (w < (tid >> 5)) run += s_warp_sum[w];
+        total += s_warp_sum[w];
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = 4 * tid + k;
+        if (r < n_kept) s_tmp[r] = run;
+        run += cnt[k];
+    }
+    const int base = tile_base(doc0, s_row[0]);
     if (tid == 0) {
-        int run = 0;
-        for (int r = 0; r < n_kept; ++r) {
-            const int c = s_tmp[r];
-            s_tmp[r] = run;
-            run += c;
-        }
-        if (base + run > pv.max_tiles) {      // cannot happen with a plan sized by cf_plan_layout_of
+        if (base + total > pv.max_tiles) {    // cannot happen with a plan sized by cf_plan_layout_of
             raise_status(pv.status, CF_ERR_WORKSPACE);
-            s_longest = -1;
+            s_fail = 1;
         }
-        pv.n_tiles[b] = s_longest < 0 ? 0 : run;
-        pv.kept_count[b] = s_longest < 0 ? 0 : n_kept;
+        const bool fail = base + total > pv.max_tiles;
+        pv.n_tiles[b] = fail ? 0 : total;
+        pv.kept_count[b] = fail ? 0 : n_kept;
         pv.tile_begin[b] = base;
         pv.n_reuse[b] = windows;
         pv.query_start[b] = query_start;
     }
     __syncthreads();
-    if (s_longest < 0) return;
+    if (s_fail) return;
     for (int r = tid; r < n_kept; r += kPlanThreads) {
-        const int i = doc0 + s_ids[r];
-        const int row0 = bv.doc_offsets[i];
-        const int len = bv.doc_offsets[i + 1] - row0;
+        const int id = s_ids[r];
+        const int i = doc0 + id;
+        const int row0 = s_row[id];
+        const int len = s_row[id + 1] - row0;
         const int first = base + s_tmp[r];
         const int count = (len + kTile - 1) / kTile;
-        pv.kept[doc0 + r] = s_ids[r];
+        pv.kept[doc0 + r] = id;
         pv.doc_tile_begin[i] = first;
         pv.doc_tile_count[i] = count;
         for (int k = 0; k < count; ++k) {
@@ -195,14 +228,13 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
     }
 
     // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D), angle in fp64 --------------
-    // (dst_start was written by other threads of this block: the barriers above order it)
     for (int idx = tid; idx < n_kept * half; idx += kPlanThreads) {
         const int r = idx / half, p = idx - r * half;
-        const int i = doc0 + s_ids[r];
-        const double delta = (double)(pv.dst_start[i] - bv.doc_src_start[i]);
+        const int id = s_ids[r];
+        const double delta = (double)(s_dst[id] - s_src[id]);
         double sn, cs;
         sincos(delta * s_inv_freq[p], &sn, &cs);
-        pv.trig[(size_t)i * half + p] = make_float2((float)cs, (float)sn);
+        pv.trig[(size_t)(doc0 + id) * half + p] = make_float2((float)cs, (float)sn);
     }
 }
 
