@@ -189,7 +189,8 @@ __device__ __forceinline__ void store_row(__nv_bfloat16* p, const float (&x)[V])
         *reinterpret_cast<__nv_bfloat162*>(p + i) = __floats2bfloat162_rn(x[i], x[i + 1]);
 }
 
-constexpr int kCombineRows = 8;       // query rows (warps) per block of the merge kernel
+constexpr int kCombineRows = 4;       // query rows (warps) per block of the merge kernel
+constexpr int kCombineDepth = 8;      // parts whose loads are in flight together
 
 // Merge the parts of one query row (one warp per row, D/32 output dimensions per lane):
 // out = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m), and the row's log-sum-exp.
@@ -233,17 +234,17 @@ combine_kernel(AttnWorkspace ws, int n_requests, long long n_rows_all, long long
     for (int i = 0; i < V; ++i) acc[i] = 0.f;
     const P* po = reinterpret_cast<const P*>(ws.part_o) + slot0 * D + lane * V;
     const size_t stride = (size_t)rows_total * D;
-    for (int p0 = 0; p0 < n_parts; p0 += 4) {                         // four independent loads in flight
-        float wp[4], x[4][V];
+    for (int p0 = 0; p0 < n_parts; p0 += kCombineDepth) {             // independent loads in flight
+        float wp[kCombineDepth], x[kCombineDepth][V];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kCombineDepth; ++u) {
             const int p = p0 + u;
             wp[u] = __shfl_sync(0xffffffffu, (p & 32) ? w[1] : w[0], p & 31);
             if (p >= n_parts) wp[u] = 0.f;
             if (wp[u] > 0.f) load_part<V>(po + (size_t)p * stride, x[u]);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < kCombineDepth; ++u)
             if (wp[u] > 0.f) {
 #pragma unroll
                 for (int i = 0; i < V; ++i) acc[i] = fmaf(x[u][i], wp[u], acc[i]);

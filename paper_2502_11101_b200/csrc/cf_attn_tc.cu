@@ -44,7 +44,8 @@ constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile
 constexpr int kBoxRows = 32;                       // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * 128;
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
-constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512;   // tiles, alignment slack, barriers
+constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
+constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512 + kMetaTiles * 8;   // tiles, alignment slack, barriers, tile list
 constexpr int kMaxStages = 6;
 constexpr int kRotateThreads = 192;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
@@ -66,6 +67,27 @@ struct Barriers {
 };
 
 static_assert(sizeof(Barriers) <= 512, "barrier block must fit its reserved shared memory");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
+
+// A key tile of the CTA's range: first store row, length, document.  The first kMetaTiles come
+// from shared memory (copied there once), later ones from the plan.
+struct TileInfo {
+    int row0, len, doc;
+};
+__device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView& pv, int ti0, int it) {
+    TileInfo t;
+    if (it < kMetaTiles) {
+        const int2 m = s_meta[it];
+        t.row0 = m.x;
+        t.len = m.y & 0xff;
+        t.doc = m.y >> 8;
+    } else {
+        t.row0 = pv.tile_row0[ti0 + it];
+        t.len = pv.tile_len[ti0 + it];
+        t.doc = pv.tile_doc[ti0 + it];
+    }
+    return t;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -273,6 +295,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const uint32_t q_base = smem_base;
     const uint32_t ring_base = q_base + n_qt * kTileBytes;
     Barriers* bars = reinterpret_cast<Barriers*>(smem + kSmemTiles * kTileBytes);
+    int2* s_meta = reinterpret_cast<int2*>(smem + kSmemTiles * kTileBytes + 512);
     volatile int* abort_flag = &bars->abort_flag;
 
     const int tbase = pv.tile_begin[b];
@@ -290,6 +313,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         if (n_it <= 0 || !alternate || n_it < 2) ws.part_m[slot0 + rows_total + r] = -INFINITY;
     }
     if (n_it <= 0) return;
+    const int ti0 = tbase + t_begin;                                // first tile of this CTA in the plan's list
+    if (tid < min(n_it, kMetaTiles)) {
+        const int len = pv.tile_len[ti0 + tid], doc = pv.tile_doc[ti0 + tid];
+        s_meta[tid] = make_int2(pv.tile_row0[ti0 + tid], (len & 0xff) | (doc << 8));   // len 1..128 -> 0x80 at most
+    }
+    // query rows of this CTA: the loads are issued now so that their latency overlaps the set-up below
+    uint4 qval[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int idx = tid + i * kThreads;
+        const int chunk = idx & 15, r = idx >> 4;                   // r: row within the CTA's row group
+        qval[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (i < 4 * n_qt && r < rows_here) {
+            const int row = rg * rg_rows + r;
+            const int g = row / lq, j = row - g * lq;
+            const int h = kvh * group + g;
+            qval[i] = __ldg(reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8));
+        }
+    }
 
     if (tid == 0) {
         const int rows_t0 = min(rows_here, 128), rows_t1 = alternate ? rows_t0 : rows_here - 128;
@@ -318,9 +360,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     int produced = 0;
     auto produce = [&](int u) {                                     // u-th ring use: K(u/2) if even, V(u/2) if odd
         const int st = u % n_stages;
-        const int ti = tbase + t_begin + (u >> 1);
-        const int row0 = pv.tile_row0[ti];
-        const int boxes = (pv.tile_len[ti] + kBoxRows - 1) / kBoxRows;
+        const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1);
+        const int row0 = tile.row0;
+        const int boxes = (tile.len + kBoxRows - 1) / kBoxRows;
         const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
         const uint32_t bar = smem_u32(&bars->kv_full[st][u & 1]);
         const uint32_t dst = ring_base + st * kTileBytes;
@@ -336,30 +378,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         for (; produced < 2; ++produced) produce(produced);        // first key and value tile; the rest follow below
     }
 
-    // query rows of this CTA into swizzled shared memory (zero rows beyond the valid ones); all
-    // loads of a thread are issued before the first store so their latencies overlap
-    {
-        uint4 val[8];
+    // query rows into swizzled shared memory (zero rows beyond the valid ones)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int idx = tid + i * kThreads;
-            const int chunk = idx & 15, r = idx >> 4;               // r: row within the CTA's row group
-            val[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (i < 4 * n_qt && r < rows_here) {
-                const int row = rg * rg_rows + r;
-                const int g = row / lq, j = row - g * lq;
-                const int h = kvh * group + g;
-                val[i] = __ldg(reinterpret_cast<const uint4*>(q + (((size_t)b * lq + j) * n_q_heads + h) * kD + chunk * 8));
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int idx = tid + i * kThreads;
-            const int chunk = idx & 15, r = idx >> 4;
-            if (i < 4 * n_qt) {
-                const int mt = r >> 7, rr = r & 127;
-                *reinterpret_cast<uint4*>(smem + (size_t)mt * kTileBytes + (chunk >> 3) * kHalfBytes + swz(rr, chunk & 7)) = val[i];
-            }
+    for (int i = 0; i < 8; ++i) {
+        const int idx = tid + i * kThreads;
+        const int chunk = idx & 15, r = idx >> 4;
+        if (i < 4 * n_qt) {
+            const int mt = r >> 7, rr = r & 127;
+            *reinterpret_cast<uint4*>(smem + (size_t)mt * kTileBytes + (chunk >> 3) * kHalfBytes + swz(rr, chunk & 7)) = qval[i];
         }
     }
     fence_proxy_async();
@@ -389,8 +415,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             auto issue_s = [&](int n) -> bool {
                 const int w = n & 1;
                 const int it = alternate ? n : (n >> 1);
-                const int ti = tbase + t_begin + it;
-                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
+                const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int stk = (2 * it) % n_stages;
                 const int kuse = (n_stages & 1) ? it / n_stages : it / (n_stages >> 1);
                 if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
@@ -410,8 +435,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             auto issue_pv = [&](int n) -> bool {
                 const int w = n & 1, j = n >> 1;
                 const int it = alternate ? n : j;
-                const int ti = tbase + t_begin + it;
-                const int n_keys = (pv.tile_len[ti] + 15) & ~15;
+                const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int uv = 2 * it + 1, stv = uv % n_stages;
                 const int vuse = (n_stages & 1) ? it / n_stages : uv / n_stages;   // value loads this stage has seen
                 if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
@@ -437,9 +461,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
         const int chunk = t & 7, rsub = t >> 3;
         for (int it = 0; it < n_it; ++it) {
-            const int ti = tbase + t_begin + it;
-            const int len = pv.tile_len[ti];
-            const float2* trig = pv.trig + (size_t)pv.tile_doc[ti] * (kD / 2);
+            const TileInfo tile = tile_info(s_meta, pv, ti0, it);
+            const int len = tile.len;
+            const float2* trig = pv.trig + (size_t)tile.doc * (kD / 2);
             const int u = 2 * it, st = u % n_stages;
             float2 cs[8];
             if (LAYOUT == CF_ROPE_HALF) {
@@ -509,8 +533,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             bool ok = true;
             for (int j = 0; j < n_items; ++j) {
                 const int it = alternate ? 2 * j + w : j;
-                const int ti = tbase + t_begin + it;
-                const int len = pv.tile_len[ti];
+                const int ti = ti0 + it;
+                const int len = tile_info(s_meta, pv, ti0, it).len;
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -691,7 +715,7 @@ int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const c
 }  // namespace
 
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
-    return g->dtype == CF_BF16 && g->head_dim == 128 && b->total_tokens > 0;
+    return g->dtype == CF_BF16 && g->head_dim == 128 && b->total_tokens > 0 && b->n_docs_total < (1 << 23);
 }
 
 int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span, const void* q,

@@ -3,6 +3,8 @@
 // Sec. 2.5), and what the hot kernels consume: per-document rotation tables (Eq. 2 angles of
 // the delta of Eq. 5) and the list of key tiles.  One thread block per request; everything
 // runs in stream order so a layer stack needs no host round trip between layers.
+#include <cmath>
+
 #include "cf_common.cuh"
 
 namespace cf {
@@ -12,11 +14,41 @@ static_assert(4 * kPlanThreads >= kMaxDocs, "the tile scan gives four ranks to e
 
 __device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// Rotary frequencies theta^(-2p/D), p < D/2 (Eq. 2), computed once on the host in fp64.
+struct InvFreq {
+    double f[64];
+};
+
+// cos and sin of an fp64 angle to about 2e-9 absolute, for |x| up to ~1e5 (positions times a
+// frequency <= 1): two-step Cody-Waite reduction by pi/2, then the Taylor polynomials of sin and
+// cos on [-pi/4, pi/4] (remainders x^11/11! < 2e-9 and x^12/12! < 2e-10).  The table entries are
+// rounded to fp32 afterwards, so this is as good as a correctly rounded fp64 routine at a fraction
+// of its fp64 instruction count.
+__device__ __forceinline__ void sincos_reduced(double x, double& sn, double& cs) {
+    const double n = rint(x * 0.63661977236758134308);               // 2/pi
+    double r = fma(-n, 1.57079632679489655800e+00, x);               // pi/2, high part
+    r = fma(-n, 6.12323399573676603587e-17, r);                      // pi/2, low part
+    const double r2 = r * r;
+    double ps = fma(r2, 2.75573192239858906526e-06, -1.98412698412698412698e-04);   // 1/9!, -1/7!
+    ps = fma(ps, r2, 8.33333333333333333333e-03);                    // 1/5!
+    ps = fma(ps, r2, -1.66666666666666666667e-01);                   // -1/3!
+    ps = fma(ps * r2, r, r);
+    double pc = fma(r2, -2.75573192239858906526e-07, 2.48015873015873015873e-05);   // -1/10!, 1/8!
+    pc = fma(pc, r2, -1.38888888888888888889e-03);                   // -1/6!
+    pc = fma(pc, r2, 4.16666666666666666667e-02);                    // 1/4!
+    pc = fma(pc, r2, -0.5);
+    pc = fma(pc, r2, 1.0);
+    const int q = (int)((long long)n & 3);                           // quadrant (two's complement: works for n < 0)
+    const double s0 = (q & 1) ? pc : ps, c0 = (q & 1) ? ps : pc;
+    sn = (q & 2) ? -s0 : s0;
+    cs = ((q + 1) & 2) ? -c0 : c0;
+}
+
 // mode 0: initialise from (order, kept_count); mode 1: prune by score, then rebuild.
 // Everything a later step needs from global memory is staged in shared memory at the start, so
 // the steps below do not each wait for a round trip of their own.
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restrict__ order,
+plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, const int* __restrict__ order,
             const int* __restrict__ kept_count_in, int query_start_arg,
             const float* __restrict__ score_accum, int keep, const int* __restrict__ keep_per_request,
             int strategy) {
@@ -27,7 +59,6 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
     __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
     __shared__ float s_score[kMaxDocs];
     __shared__ unsigned char s_flag[kMaxDocs];
-    __shared__ double s_inv_freq[64];
     __shared__ int s_longest, s_min_cursor, s_fail;
     __shared__ int s_warp_sum[kPlanThreads / 32];
 
@@ -77,8 +108,6 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
     int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
                                 : pv.query_start[b];
     int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
-    for (int p = tid; p < half; p += kPlanThreads)
-        s_inv_freq[p] = pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
     if (tid == 0) {
         s_longest = 0;
         s_min_cursor = 0x7fffffff;
@@ -167,7 +196,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
             raise_status(pv.status, CF_ERR_RANGE);
     }
 
-    // ---- key tiles: document-aligned runs of at most kTile rows -------------------------------
+    // ---- key tiles: runs of at most kTile rows that never straddle two documents -----------------
     // exclusive prefix sum of the per-rank tile counts: four consecutive ranks per thread
     int cnt[4], local = 0;
 #pragma unroll
@@ -220,10 +249,13 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
         pv.kept[doc0 + r] = id;
         pv.doc_tile_begin[i] = first;
         pv.doc_tile_count[i] = count;
+        // the document's rows are spread evenly over its tiles, in steps of 32 rows (160 rows make
+        // tiles of 96 and 64, not 128 and 32), so consecutive tiles cost about the same
+        const int step = count > 0 ? min(kTile, ((len + count - 1) / count + 31) & ~31) : kTile;
         for (int k = 0; k < count; ++k) {
             pv.tile_doc[first + k] = i;
-            pv.tile_row0[first + k] = row0 + k * kTile;
-            pv.tile_len[first + k] = min(kTile, len - k * kTile);
+            pv.tile_row0[first + k] = row0 + k * step;
+            pv.tile_len[first + k] = min(step, len - k * step);
         }
     }
 
@@ -233,7 +265,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
         const int id = s_ids[r];
         const double delta = (double)(s_dst[id] - s_src[id]);
         double sn, cs;
-        sincos(delta * s_inv_freq[p], &sn, &cs);
+        sincos_reduced(delta * inv_freq.f[p], sn, cs);
         pv.trig[(size_t)(doc0 + id) * half + p] = make_float2((float)cs, (float)sn);
     }
 }
@@ -241,7 +273,11 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, int mode, const int* __restr
 int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
                 const int* order, const int* kept_count, int query_start, const float* score_accum,
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream) {
-    plan_kernel<<<bv.n_requests, kPlanThreads, 0, stream>>>(gv, bv, pv, mode, order, kept_count,
+    if (gv.head_dim > 128) return CF_ERR_UNSUPPORTED;
+    InvFreq inv_freq;
+    for (int p = 0; p < gv.head_dim / 2; ++p)
+        inv_freq.f[p] = std::pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
+    plan_kernel<<<bv.n_requests, kPlanThreads, 0, stream>>>(gv, bv, pv, inv_freq, mode, order, kept_count,
                                                            query_start, score_accum, keep,
                                                            keep_per_request, strategy);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
