@@ -14,16 +14,18 @@ static_assert(4 * kPlanThreads >= kMaxDocs, "the tile scan gives four ranks to e
 
 __device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
-// Rotary frequencies theta^(-2p/D), p < D/2 (Eq. 2), computed once on the host in fp64.
+// Rotary frequencies theta^(-2p/D), p < D/2 (Eq. 2), computed once on the host: in fp64, and as
+// a fraction of a full turn in units of 2^-64 (frequency / 2 pi), which lets the device reduce
+// position * frequency modulo one turn in exact 64-bit integer arithmetic.
 struct InvFreq {
     double f[64];
+    unsigned long long turns[64];
 };
 
 // cos and sin of an fp64 angle to about 2e-9 absolute, for |x| up to ~1e5 (positions times a
 // frequency <= 1): two-step Cody-Waite reduction by pi/2, then the Taylor polynomials of sin and
-// cos on [-pi/4, pi/4] (remainders x^11/11! < 2e-9 and x^12/12! < 2e-10).  The table entries are
-// rounded to fp32 afterwards, so this is as good as a correctly rounded fp64 routine at a fraction
-// of its fp64 instruction count.
+// cos on [-pi/4, pi/4] (remainders x^11/11! < 2e-9 and x^12/12! < 2e-10).  Used for fp32 caches,
+// whose rotated keys are held to a few fp32 ulp.
 __device__ __forceinline__ void sincos_reduced(double x, double& sn, double& cs) {
     const double n = rint(x * 0.63661977236758134308);               // 2/pi
     double r = fma(-n, 1.57079632679489655800e+00, x);               // pi/2, high part
@@ -44,16 +46,63 @@ __device__ __forceinline__ void sincos_reduced(double x, double& sn, double& cs)
     cs = ((q + 1) & 2) ? -c0 : c0;
 }
 
+// cos and sin of delta positions at a frequency given in 2^-64 turns: the phase modulo one turn is
+// an exact wrapping 64-bit product, split into the nearest quarter turn and a remainder in
+// [-pi/4, pi/4) that fp32 evaluates to about 1e-7.  Used for bf16 caches (bf16 spacing is 4e-3).
+__device__ __forceinline__ void sincos_turns(int delta, unsigned long long turns, float& sn, float& cs) {
+    const unsigned long long phase = (unsigned long long)(long long)delta * turns;
+    const unsigned long long quarter = (phase + (1ull << 61)) >> 62;                 // nearest quarter turn, 0..3
+    const long long rem = (long long)(phase - (quarter << 62));                      // [-2^61, 2^61) of 2^-64 turns
+    const float r = (float)(int)(rem >> 37) * (0.78539816339744830962f / 16777216.0f);   // 2^24 steps per pi/4
+    float s0, c0;
+    sincosf(r, &s0, &c0);
+    const int q = (int)quarter;
+    const float s1 = (q & 1) ? c0 : s0, c1 = (q & 1) ? s0 : c0;
+    sn = (q & 2) ? -s1 : s1;
+    cs = ((q + 1) & 2) ? -c1 : c1;
+}
+
+// Exclusive prefix sum over 4 * kPlanThreads values, four consecutive ones per thread (v[k] has index
+// 4 * tid + k); returns the total.  Every thread of the block must call it.
+__device__ __forceinline__ int block_scan4(int (&v)[4], int* s_warp_sum) {
+    const int tid = threadIdx.x;
+    const int local = v[0] + v[1] + v[2] + v[3];
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((tid & 31) >= o) incl += up;
+    }
+    if ((tid & 31) == 31) s_warp_sum[tid >> 5] = incl;
+    __syncthreads();
+    int run = incl - local, total = 0;
+#pragma unroll
+    for (int w = 0; w < kPlanThreads / 32; ++w) {
+        const int sum = s_warp_sum[w];
+        if (w < (tid >> 5)) run += sum;
+        total += sum;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int x = v[k];
+        v[k] = run;
+        run += x;
+    }
+    return total;
+}
+
 // mode 0: initialise from (order, kept_count); mode 1: prune by score, then rebuild.
-// Everything a later step needs from global memory is staged in shared memory at the start, so
-// the steps below do not each wait for a round trip of their own.
+// Everything a later step needs from global memory is staged in shared memory at the start, and the
+// serial steps of the method (ranking, walking a window backwards from the query, numbering the
+// tiles) are written as counting and prefix sums over the whole block.
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, const int* __restrict__ order,
             const int* __restrict__ kept_count_in, int query_start_arg,
             const float* __restrict__ score_accum, int keep, const int* __restrict__ keep_per_request,
             int strategy) {
     __shared__ int s_ids[kMaxDocs];       // kept local ids by rank
-    __shared__ int s_tmp[kMaxDocs];       // new order, then the first tile of every rank
+    __shared__ int s_tmp[kMaxDocs];       // new order; running lengths of the windows; first tile of every rank
     __shared__ int s_row[kMaxDocs + 1];   // first store row of every document (by local id), and the end
     __shared__ int s_dst[kMaxDocs];       // start positions by local id
     __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
@@ -117,26 +166,35 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
 
     // ---- the kept list, in rank order -------------------------------------------------------
     if (mode != 0) {
-        // rank by counting: how many kept documents beat this one (ties: lower id wins)
-        for (int r = tid; r < n_old; r += kPlanThreads) {
-            const float sc = s_score[r];
-            const int id = s_ids[r];
+        // rank by counting: how many kept documents beat this one (ties: lower id wins); eight
+        // lanes share the count of one document
+        for (int r0 = 0; r0 < n_old; r0 += kPlanThreads / 8) {
+            const int r = r0 + (tid >> 3);
+            const float sc = r < n_old ? s_score[r] : 0.f;
+            const int id = r < n_old ? s_ids[r] : 0;
             int better = 0;
-            for (int o = 0; o < n_old; ++o) {
-                const float so = s_score[o];
-                better += (so > sc) || (so == sc && s_ids[o] < id);
+            if (r < n_old)
+                for (int o = tid & 7; o < n_old; o += 8) {
+                    const float so = s_score[o];
+                    better += (so > sc) || (so == sc && s_ids[o] < id);
+                }
+            better += __shfl_xor_sync(0xffffffffu, better, 1);
+            better += __shfl_xor_sync(0xffffffffu, better, 2);
+            better += __shfl_xor_sync(0xffffffffu, better, 4);
+            if (r < n_old && (tid & 7) == 0) {
+                s_flag[r] = better < keep_b;
+                if (strategy == CF_ALLOC_SORT && better < keep_b) s_tmp[better] = id;
             }
-            s_flag[r] = better < keep_b;
-            if (strategy == CF_ALLOC_SORT && better < keep_b) s_tmp[better] = id;
         }
         __syncthreads();
-        if (strategy != CF_ALLOC_SORT) {
-            for (int r = tid; r < n_old; r += kPlanThreads) {
-                if (!s_flag[r]) continue;
-                int before = 0;
-                for (int o = 0; o < r; ++o) before += s_flag[o];
-                s_tmp[before] = s_ids[r];
-            }
+        if (strategy != CF_ALLOC_SORT) {                  // survivors keep their order: slot = survivors before
+            int before[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) before[k] = (4 * tid + k < n_old) ? (int)s_flag[4 * tid + k] : 0;
+            block_scan4(before, s_warp_sum);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (4 * tid + k < n_old && s_flag[4 * tid + k]) s_tmp[before[k]] = s_ids[4 * tid + k];
         }
         __syncthreads();
         n_kept = keep_b;
@@ -179,58 +237,72 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
                 windows = (n_kept + per_window - 1) / per_window;
             }
         }
-        // one thread per window walks its ranks r = w, w + windows, ... backwards from the query
-        for (int w = tid; w < windows && w < n_kept; w += kPlanThreads) {
-            int cursor = query_start;
-            for (int r = w; r < n_kept; r += windows) {
-                const int id = s_ids[r];
-                cursor -= s_row[id + 1] - s_row[id];
-                s_dst[id] = cursor;
-                pv.dst_start[doc0 + id] = cursor;
-                pv.group[doc0 + id] = w;
+        // Window w holds the ranks w, w + windows, ... and is filled backwards from the query.  With
+        // the ranks listed window by window (index x), a document starts at the query start minus the
+        // lengths of its window up to and including itself: one prefix sum over x.
+        const int w_used = min(windows, n_kept);
+        const int small = n_kept / w_used, extra = n_kept - small * w_used;   // the first `extra` windows hold small + 1
+        int len4[4], rank4[4], first4[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int x = 4 * tid + k;
+            len4[k] = 0;
+            rank4[k] = -1;
+            first4[k] = 0;
+            if (x < n_kept) {
+                int w, slot;
+                if (x < extra * (small + 1)) {
+                    w = x / (small + 1);
+                    slot = x - w * (small + 1);
+                } else {
+                    const int y = x - extra * (small + 1);
+                    w = extra + y / small;
+                    slot = y - (w - extra) * small;
+                }
+                rank4[k] = slot * windows + w;
+                first4[k] = x - slot;                                       // index of the window's first rank
+                const int id = s_ids[rank4[k]];
+                len4[k] = s_row[id + 1] - s_row[id];
             }
-            atomicMin(&s_min_cursor, cursor);
         }
+        int before4[4] = {len4[0], len4[1], len4[2], len4[3]};
+        block_scan4(before4, s_warp_sum);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (rank4[k] >= 0) s_tmp[4 * tid + k] = before4[k];
+        __syncthreads();
+        int lowest = 0x7fffffff;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (rank4[k] >= 0) {
+                const int id = s_ids[rank4[k]];
+                const int start = query_start - (before4[k] - s_tmp[first4[k]] + len4[k]);
+                s_dst[id] = start;
+                pv.dst_start[doc0 + id] = start;
+                pv.group[doc0 + id] = rank4[k] % windows;
+                lowest = min(lowest, start);
+            }
+        atomicMin(&s_min_cursor, lowest);
         __syncthreads();
         if (tid == 0 && (s_min_cursor < bv.prefix_len || query_start + bv.tail_reserve > gv.pos_range))
             raise_status(pv.status, CF_ERR_RANGE);
     }
 
     // ---- key tiles: runs of at most kTile rows that never straddle two documents -----------------
-    // exclusive prefix sum of the per-rank tile counts: four consecutive ranks per thread
-    int cnt[4], local = 0;
+    int first_tile[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const int r = 4 * tid + k;
-        cnt[k] = r < n_kept ? (s_row[s_ids[r] + 1] - s_row[s_ids[r]] + kTile - 1) / kTile : 0;
-        local += cnt[k];
+        first_tile[k] = r < n_kept ? (s_row[s_ids[r] + 1] - s_row[s_ids[r]] + kTile - 1) / kTile : 0;
     }
-    int incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if ((tid & 31) >= o) incl += up;
-    }
-    if ((tid & 31) == 31) s_warp_sum[tid >> 5] = incl;
-    __syncthreads();
-    int run = incl - local, total = 0;
-    for (int w = 0; w < kPlanThreads / 32; ++w) {
-        if (w < (tid >> 5)) run += s_warp_sum[w];
-        total += s_warp_sum[w];
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int r = 4 * tid + k;
-        if (r < n_kept) s_tmp[r] = run;
-        run += cnt[k];
-    }
+    const int total = block_scan4(first_tile, s_warp_sum);
     const int base = tile_base(doc0, s_row[0]);
     if (tid == 0) {
-        if (base + total > pv.max_tiles) {    // cannot happen with a plan sized by cf_plan_layout_of
+        const bool fail = base + total > pv.max_tiles;   // cannot happen with a plan sized by cf_plan_layout_of
+        if (fail) {
             raise_status(pv.status, CF_ERR_WORKSPACE);
             s_fail = 1;
         }
-        const bool fail = base + total > pv.max_tiles;
         pv.n_tiles[b] = fail ? 0 : total;
         pv.kept_count[b] = fail ? 0 : n_kept;
         pv.tile_begin[b] = base;
@@ -239,12 +311,15 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     }
     __syncthreads();
     if (s_fail) return;
-    for (int r = tid; r < n_kept; r += kPlanThreads) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = 4 * tid + k;
+        if (r >= n_kept) continue;
         const int id = s_ids[r];
         const int i = doc0 + id;
         const int row0 = s_row[id];
         const int len = s_row[id + 1] - row0;
-        const int first = base + s_tmp[r];
+        const int first = base + first_tile[k];
         const int count = (len + kTile - 1) / kTile;
         pv.kept[doc0 + r] = id;
         pv.doc_tile_begin[i] = first;
@@ -252,21 +327,27 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         // the document's rows are spread evenly over its tiles, in steps of 32 rows (160 rows make
         // tiles of 96 and 64, not 128 and 32), so consecutive tiles cost about the same
         const int step = count > 0 ? min(kTile, ((len + count - 1) / count + 31) & ~31) : kTile;
-        for (int k = 0; k < count; ++k) {
-            pv.tile_doc[first + k] = i;
-            pv.tile_row0[first + k] = row0 + k * step;
-            pv.tile_len[first + k] = min(step, len - k * step);
+        for (int t = 0; t < count; ++t) {
+            pv.tile_doc[first + t] = i;
+            pv.tile_row0[first + t] = row0 + t * step;
+            pv.tile_len[first + t] = min(step, len - t * step);
         }
     }
 
-    // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D), angle in fp64 --------------
+    // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D) -------------------------------
     for (int idx = tid; idx < n_kept * half; idx += kPlanThreads) {
         const int r = idx / half, p = idx - r * half;
         const int id = s_ids[r];
-        const double delta = (double)(s_dst[id] - s_src[id]);
-        double sn, cs;
-        sincos_reduced(delta * inv_freq.f[p], sn, cs);
-        pv.trig[(size_t)(doc0 + id) * half + p] = make_float2((float)cs, (float)sn);
+        const int delta = s_dst[id] - s_src[id];
+        float2 entry;
+        if (gv.dtype == CF_BF16) {
+            sincos_turns(delta, inv_freq.turns[p], entry.y, entry.x);
+        } else {
+            double sn, cs;
+            sincos_reduced((double)delta * inv_freq.f[p], sn, cs);
+            entry = make_float2((float)cs, (float)sn);
+        }
+        pv.trig[(size_t)(doc0 + id) * half + p] = entry;
     }
 }
 
@@ -275,8 +356,11 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream) {
     if (gv.head_dim > 128) return CF_ERR_UNSUPPORTED;
     InvFreq inv_freq;
-    for (int p = 0; p < gv.head_dim / 2; ++p)
+    for (int p = 0; p < gv.head_dim / 2; ++p) {
         inv_freq.f[p] = std::pow(gv.rope_theta, -2.0 * (double)p / (double)gv.head_dim);
+        const long double turn = (long double)inv_freq.f[p] / (2.0L * 3.14159265358979323846264338327950288L);
+        inv_freq.turns[p] = (unsigned long long)ldexpl(turn, 64);          // < 2^62: theta > 1 keeps f <= 1
+    }
     plan_kernel<<<bv.n_requests, kPlanThreads, 0, stream>>>(gv, bv, pv, inv_freq, mode, order, kept_count,
                                                            query_start, score_accum, keep,
                                                            keep_per_request, strategy);
