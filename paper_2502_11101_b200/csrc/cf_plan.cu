@@ -47,15 +47,33 @@ __device__ __forceinline__ void sincos_reduced(double x, double& sn, double& cs)
 }
 
 // cos and sin of delta positions at a frequency given in 2^-64 turns: the phase modulo one turn is
-// an exact wrapping 64-bit product, split into the nearest quarter turn and a remainder in
-// [-pi/4, pi/4) that fp32 evaluates to about 1e-7.  Used for bf16 caches (bf16 spacing is 4e-3).
+// an exact wrapping 64-bit product, split into the nearest quarter turn and a remainder r in
+// [-pi/4, pi/4).  r is carried as a pair of floats (r_hi + r_lo, about 48 bits), and the Taylor
+// polynomials add their small terms to r_hi (sin) and to 1 (cos) last, so the results are within
+// about 7e-8 of the exact values -- fp32 tables for bf16 caches (bf16 spacing is 4e-3) without
+// any fp64 arithmetic.
 __device__ __forceinline__ void sincos_turns(int delta, unsigned long long turns, float& sn, float& cs) {
     const unsigned long long phase = (unsigned long long)(long long)delta * turns;
     const unsigned long long quarter = (phase + (1ull << 61)) >> 62;                 // nearest quarter turn, 0..3
     const long long rem = (long long)(phase - (quarter << 62));                      // [-2^61, 2^61) of 2^-64 turns
-    const float r = (float)(int)(rem >> 37) * (0.78539816339744830962f / 16777216.0f);   // 2^24 steps per pi/4
-    float s0, c0;
-    sincosf(r, &s0, &c0);
+    const float top = (float)(int)(rem >> 37);                                       // 25 signed bits, units of 2^-27 turn
+    const float low = (float)(int)((rem >> 13) & 0xFFFFFF);                          // the next 24 bits
+    constexpr double kStep = 6.283185307179586476925 / 134217728.0;                  // 2 pi / 2^27
+    constexpr float kStepHi = (float)kStep;
+    constexpr float kStepLo = (float)(kStep - (double)kStepHi);
+    constexpr float kStepLow = (float)(kStep / 16777216.0);
+    const float r_hi = top * kStepHi;
+    const float r_lo = fmaf(top, kStepLo, fmaf(top, kStepHi, -r_hi)) + low * kStepLow;
+    const float r2 = r_hi * r_hi;
+    float ps = fmaf(r2, 2.7557319e-6f, -1.9841270e-4f);                              // 1/9!, -1/7!
+    ps = fmaf(ps, r2, 8.3333333e-3f);                                                // 1/5!
+    ps = fmaf(ps, r2, -1.6666667e-1f);                                               // -1/3!
+    const float s0 = r_hi + fmaf(ps * r2, r_hi, r_lo);
+    float pc = fmaf(r2, -2.7557319e-7f, 2.4801587e-5f);                              // -1/10!, 1/8!
+    pc = fmaf(pc, r2, -1.3888889e-3f);                                               // -1/6!
+    pc = fmaf(pc, r2, 4.1666667e-2f);                                                // 1/4!
+    pc = fmaf(pc, r2, -0.5f);
+    const float c0 = 1.0f + fmaf(pc, r2, -(r_hi * r_lo));
     const int q = (int)quarter;
     const float s1 = (q & 1) ? c0 : s0, c1 = (q & 1) ? s0 : c0;
     sn = (q & 2) ? -s1 : s1;
