@@ -9,8 +9,8 @@
 
 namespace cf {
 
-constexpr int kPlanThreads = 256;
-static_assert(4 * kPlanThreads >= kMaxDocs, "the tile scan gives four ranks to every thread");
+constexpr int kPlanThreads = 1024;
+static_assert(kPlanThreads >= kMaxDocs, "every rank of a request has a thread of its own");
 
 __device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
@@ -80,40 +80,41 @@ __device__ __forceinline__ void sincos_turns(int delta, unsigned long long turns
     cs = ((q + 1) & 2) ? -c1 : c1;
 }
 
-// Exclusive prefix sum over 4 * kPlanThreads values, four consecutive ones per thread (v[k] has index
-// 4 * tid + k); returns the total.  Every thread of the block must call it.
-__device__ __forceinline__ int block_scan4(int (&v)[4], int* s_warp_sum) {
-    const int tid = threadIdx.x;
-    const int local = v[0] + v[1] + v[2] + v[3];
-    int incl = local;
+// Exclusive prefix sum of one value per thread over the block; *total receives the sum.  Every
+// thread of the block must call it.
+__device__ __forceinline__ int block_scan(int value, int* s_warp_sum, int* total) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int incl = value;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if ((tid & 31) >= o) incl += up;
+        if (lane >= o) incl += up;
     }
-    if ((tid & 31) == 31) s_warp_sum[tid >> 5] = incl;
+    if (lane == 31) s_warp_sum[warp] = incl;
     __syncthreads();
-    int run = incl - local, total = 0;
+    if (warp == 0) {                                     // scan of the 32 warp sums
+        const int mine = s_warp_sum[lane];
+        int acc = mine;
 #pragma unroll
-    for (int w = 0; w < kPlanThreads / 32; ++w) {
-        const int sum = s_warp_sum[w];
-        if (w < (tid >> 5)) run += sum;
-        total += sum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, acc, o);
+            if (lane >= o) acc += up;
+        }
+        s_warp_sum[lane] = acc - mine;                   // sum of the warps before this one
+        if (lane == 31) s_warp_sum[32] = acc;
     }
     __syncthreads();
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int x = v[k];
-        v[k] = run;
-        run += x;
-    }
-    return total;
+    const int before = s_warp_sum[warp] + incl - value;
+    *total = s_warp_sum[32];
+    __syncthreads();
+    return before;
 }
 
 // mode 0: initialise from (order, kept_count); mode 1: prune by score, then rebuild.
-// Everything a later step needs from global memory is staged in shared memory at the start, and the
+// Everything a later step needs from global memory is staged in shared memory at the start, the
 // serial steps of the method (ranking, walking a window backwards from the query, numbering the
-// tiles) are written as counting and prefix sums over the whole block.
+// tiles) are written as counting and prefix sums over the whole block, and the results leave for
+// global memory together at the end: no barrier in between has stores in flight to wait for.
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, const int* __restrict__ order,
             const int* __restrict__ kept_count_in, int query_start_arg,
@@ -123,11 +124,12 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     __shared__ int s_tmp[kMaxDocs];       // new order; running lengths of the windows; first tile of every rank
     __shared__ int s_row[kMaxDocs + 1];   // first store row of every document (by local id), and the end
     __shared__ int s_dst[kMaxDocs];       // start positions by local id
+    __shared__ int s_group[kMaxDocs];     // window index by local id
     __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
     __shared__ float s_score[kMaxDocs];
     __shared__ unsigned char s_flag[kMaxDocs];
-    __shared__ int s_longest, s_min_cursor, s_fail;
-    __shared__ int s_warp_sum[kPlanThreads / 32];
+    __shared__ int s_longest, s_min_cursor;
+    __shared__ int s_warp_sum[kPlanThreads / 32 + 1];
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
@@ -143,6 +145,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         return;
     }
     const int half = gv.head_dim / 2;
+    const int half_log2 = half == 64 ? 6 : 5;
 
     // ---- stage the inputs -------------------------------------------------------------------
     int n_old = 0, keep_b = 0, n_kept = 0;
@@ -171,6 +174,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     for (int i = tid; i < n_docs; i += kPlanThreads) {
         s_src[i] = bv.doc_src_start[doc0 + i];
         s_dst[i] = mode == 0 ? -1 : pv.dst_start[doc0 + i];
+        s_group[i] = mode == 0 ? -1 : pv.group[doc0 + i];
     }
     int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
                                 : pv.query_start[b];
@@ -178,7 +182,6 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     if (tid == 0) {
         s_longest = 0;
         s_min_cursor = 0x7fffffff;
-        s_fail = 0;
     }
     __syncthreads();
 
@@ -206,13 +209,10 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         }
         __syncthreads();
         if (strategy != CF_ALLOC_SORT) {                  // survivors keep their order: slot = survivors before
-            int before[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) before[k] = (4 * tid + k < n_old) ? (int)s_flag[4 * tid + k] : 0;
-            block_scan4(before, s_warp_sum);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (4 * tid + k < n_old && s_flag[4 * tid + k]) s_tmp[before[k]] = s_ids[4 * tid + k];
+            const int survives = tid < n_old ? (int)s_flag[tid] : 0;
+            int n_survive;
+            const int before = block_scan(survives, s_warp_sum, &n_survive);
+            if (survives) s_tmp[before] = s_ids[tid];
         }
         __syncthreads();
         n_kept = keep_b;
@@ -228,14 +228,6 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     __syncthreads();
     for (int r = tid; r < n_kept; r += kPlanThreads) s_flag[s_ids[r]] = 1;
     __syncthreads();
-    for (int i = tid; i < n_docs; i += kPlanThreads) {
-        pv.doc_tile_count[doc0 + i] = 0;
-        pv.doc_tile_begin[doc0 + i] = 0;
-        if (!s_flag[i]) {
-            pv.dst_start[doc0 + i] = -1;
-            pv.group[doc0 + i] = -1;
-        }
-    }
 
     // ---- positional allocation ----------------------------------------------------------------
     if (reallocate && n_kept > 0) {
@@ -260,46 +252,35 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         // lengths of its window up to and including itself: one prefix sum over x.
         const int w_used = min(windows, n_kept);
         const int small = n_kept / w_used, extra = n_kept - small * w_used;   // the first `extra` windows hold small + 1
-        int len4[4], rank4[4], first4[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int x = 4 * tid + k;
-            len4[k] = 0;
-            rank4[k] = -1;
-            first4[k] = 0;
-            if (x < n_kept) {
-                int w, slot;
-                if (x < extra * (small + 1)) {
-                    w = x / (small + 1);
-                    slot = x - w * (small + 1);
-                } else {
-                    const int y = x - extra * (small + 1);
-                    w = extra + y / small;
-                    slot = y - (w - extra) * small;
-                }
-                rank4[k] = slot * windows + w;
-                first4[k] = x - slot;                                       // index of the window's first rank
-                const int id = s_ids[rank4[k]];
-                len4[k] = s_row[id + 1] - s_row[id];
+        const int x = tid;
+        int len = 0, rank = -1, first = 0;
+        if (x < n_kept) {
+            int w, slot;
+            if (x < extra * (small + 1)) {
+                w = x / (small + 1);
+                slot = x - w * (small + 1);
+            } else {
+                const int y = x - extra * (small + 1);
+                w = extra + y / small;
+                slot = y - (w - extra) * small;
             }
+            rank = slot * windows + w;
+            first = x - slot;                                               // index of the window's first rank
+            const int id = s_ids[rank];
+            len = s_row[id + 1] - s_row[id];
         }
-        int before4[4] = {len4[0], len4[1], len4[2], len4[3]};
-        block_scan4(before4, s_warp_sum);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (rank4[k] >= 0) s_tmp[4 * tid + k] = before4[k];
+        int all_rows;
+        const int before = block_scan(len, s_warp_sum, &all_rows);
+        if (rank >= 0) s_tmp[x] = before;
         __syncthreads();
         int lowest = 0x7fffffff;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (rank4[k] >= 0) {
-                const int id = s_ids[rank4[k]];
-                const int start = query_start - (before4[k] - s_tmp[first4[k]] + len4[k]);
-                s_dst[id] = start;
-                pv.dst_start[doc0 + id] = start;
-                pv.group[doc0 + id] = rank4[k] % windows;
-                lowest = min(lowest, start);
-            }
+        if (rank >= 0) {
+            const int id = s_ids[rank];
+            const int start = query_start - (before - s_tmp[first] + len);
+            s_dst[id] = start;
+            s_group[id] = rank % windows;
+            lowest = start;
+        }
         atomicMin(&s_min_cursor, lowest);
         __syncthreads();
         if (tid == 0 && (s_min_cursor < bv.prefix_len || query_start + bv.tail_reserve > gv.pos_range))
@@ -307,38 +288,39 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     }
 
     // ---- key tiles: runs of at most kTile rows that never straddle two documents -----------------
-    int first_tile[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int r = 4 * tid + k;
-        first_tile[k] = r < n_kept ? (s_row[s_ids[r] + 1] - s_row[s_ids[r]] + kTile - 1) / kTile : 0;
-    }
-    const int total = block_scan4(first_tile, s_warp_sum);
+    const int my_tiles = tid < n_kept ? (s_row[s_ids[tid] + 1] - s_row[s_ids[tid]] + kTile - 1) / kTile : 0;
+    int total;
+    const int first_tile = block_scan(my_tiles, s_warp_sum, &total);
     const int base = tile_base(doc0, s_row[0]);
+    const bool fail = base + total > pv.max_tiles;       // cannot happen with a plan sized by cf_plan_layout_of
+
+    // ---- results to global memory ---------------------------------------------------------------
     if (tid == 0) {
-        const bool fail = base + total > pv.max_tiles;   // cannot happen with a plan sized by cf_plan_layout_of
-        if (fail) {
-            raise_status(pv.status, CF_ERR_WORKSPACE);
-            s_fail = 1;
-        }
+        if (fail) raise_status(pv.status, CF_ERR_WORKSPACE);
         pv.n_tiles[b] = fail ? 0 : total;
         pv.kept_count[b] = fail ? 0 : n_kept;
         pv.tile_begin[b] = base;
         pv.n_reuse[b] = windows;
         pv.query_start[b] = query_start;
     }
-    __syncthreads();
-    if (s_fail) return;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int r = 4 * tid + k;
-        if (r >= n_kept) continue;
+    if (fail) return;
+    for (int i = tid; i < n_docs; i += kPlanThreads) {
+        const bool kept = s_flag[i] != 0;
+        pv.dst_start[doc0 + i] = kept ? s_dst[i] : -1;
+        pv.group[doc0 + i] = kept ? s_group[i] : -1;
+        if (!kept) {
+            pv.doc_tile_count[doc0 + i] = 0;
+            pv.doc_tile_begin[doc0 + i] = 0;
+        }
+    }
+    if (tid < n_kept) {
+        const int r = tid;
         const int id = s_ids[r];
         const int i = doc0 + id;
         const int row0 = s_row[id];
         const int len = s_row[id + 1] - row0;
-        const int first = base + first_tile[k];
-        const int count = (len + kTile - 1) / kTile;
+        const int first = base + first_tile;
+        const int count = my_tiles;
         pv.kept[doc0 + r] = id;
         pv.doc_tile_begin[i] = first;
         pv.doc_tile_count[i] = count;
@@ -354,7 +336,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
 
     // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D) -------------------------------
     for (int idx = tid; idx < n_kept * half; idx += kPlanThreads) {
-        const int r = idx / half, p = idx - r * half;
+        const int r = idx >> half_log2, p = idx & (half - 1);            // half is 32 or 64
         const int id = s_ids[r];
         const int delta = s_dst[id] - s_src[id];
         float2 entry;
