@@ -41,8 +41,14 @@ constexpr int kThreads = 512;
 constexpr int kD = 128;
 constexpr int kHalfBytes = kTile * 128;            // one 64-column half of a 128-row tile, 128 B per row
 constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile, a Q tile or a P tile
-constexpr int kBoxRows = 32;                       // rows per TMA box
+constexpr int kBoxRows = 32;                       // TMA boxes are 32, 64, 96 or 128 rows high
 constexpr int kBoxBytes = kBoxRows * 128;
+
+// Tensor maps of the key store and of the value store, one per box height: a tile is fetched by
+// two bulk copies (one per 64-column half) whatever its length.
+struct StoreMaps {
+    CUtensorMap k[4], v[4];
+};
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
 constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
 constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512 + kMetaTiles * 8;   // tiles, alignment slack, barriers, tile list
@@ -263,7 +269,7 @@ __device__ __forceinline__ float chunk_exp(uint32_t (&v)[32], int valid, float s
 
 template <int LAYOUT>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
                float scale_log2, const __nv_bfloat16* __restrict__ q) {
     extern __shared__ unsigned char smem_raw[];
@@ -363,18 +369,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1);
         const int row0 = tile.row0;
         const int boxes = (tile.len + kBoxRows - 1) / kBoxRows;
-        const CUtensorMap* map = (u & 1) ? &map_v : &map_k;
+        const CUtensorMap* map = (u & 1) ? &maps.v[boxes - 1] : &maps.k[boxes - 1];
         const uint32_t bar = smem_u32(&bars->kv_full[st][u & 1]);
         const uint32_t dst = ring_base + st * kTileBytes;
         mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
-        for (int bx = 0; bx < boxes; ++bx) {
-            tma_load_4d(dst + bx * kBoxBytes, map, 0, kvh, row0 + bx * kBoxRows, layer, bar);
-            tma_load_4d(dst + kHalfBytes + bx * kBoxBytes, map, 64, kvh, row0 + bx * kBoxRows, layer, bar);
-        }
+        tma_load_4d(dst, map, 0, kvh, row0, layer, bar);
+        tma_load_4d(dst + kHalfBytes, map, 64, kvh, row0, layer, bar);
     };
     if (warp == 12 && lane == 0) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+        for (int i = 0; i < 4; ++i) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.k[i]) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.v[i]) : "memory");
+        }
         for (; produced < 2; ++produced) produce(produced);        // first key and value tile; the rest follow below
     }
 
@@ -696,7 +702,8 @@ EncodeTiledFn encode_fn() {
 
 // The store as a 4-D tensor (head_dim, kv heads, rows, layers); boxes of 64 x 1 x 32 x 1.  Rows past
 // the end of a layer read as zero, they never reach into the next layer.
-int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span) {
+int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span,
+                   int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return CF_ERR_CUDA;
     const cuuint64_t layer_bytes = span.n_layers > 1 ? (cuuint64_t)span.kv_stride * 2
@@ -704,7 +711,7 @@ int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const c
     const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, (cuuint64_t)b->total_tokens,
                                 (cuuint64_t)span.n_layers};
     const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)b->token_stride * 2, layer_bytes};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kBoxRows, 1};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
     const cuuint32_t elem[4] = {1, 1, 1, 1};
     CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -725,11 +732,13 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
     if ((long long)g->n_kv_heads * row_groups > 65535 || (long long)b->n_requests * span.n_layers > 65535 ||
         (ws.n_splits & 1) || (ws.rg_rows != 128 && ws.rg_rows != 256))
         return CF_ERR_INVALID_ARG;
-    CUtensorMap map_k, map_v;
-    int rc = make_store_map(&map_k, k, g, b, span);
-    if (rc != CF_OK) return rc;
-    rc = make_store_map(&map_v, v, g, b, span);
-    if (rc != CF_OK) return rc;
+    StoreMaps maps;
+    for (int i = 0; i < 4; ++i) {
+        int rc = make_store_map(&maps.k[i], k, g, b, span, (i + 1) * kBoxRows);
+        if (rc != CF_OK) return rc;
+        rc = make_store_map(&maps.v[i], v, g, b, span, (i + 1) * kBoxRows);
+        if (rc != CF_OK) return rc;
+    }
     dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
               (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
@@ -740,7 +749,7 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                 return CF_ERR_CUDA;
             configured[which] = true;
         }
-        kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_k, map_v, bv, pv, ws, span.q_stride, g->n_q_heads,
+        kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, bv, pv, ws, span.q_stride, g->n_q_heads,
                                                        g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q));
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
