@@ -95,6 +95,13 @@ __device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView
     return t;
 }
 
+// The ring has six stages (one query tile in shared memory) or five (two query tiles); dividing by
+// a literal keeps the index arithmetic of the hot loops to a few instructions.
+__device__ __forceinline__ int ring_mod(int x, bool six) { return six ? x % 6 : x % 5; }
+__device__ __forceinline__ int ring_div(int x, bool six) { return six ? x / 6 : x / 5; }
+// Loads of one kind (keys or values) a stage has received before the one of tile `it`.
+__device__ __forceinline__ int ring_uses(int it, bool six) { return six ? it / 3 : it / 5; }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -365,7 +372,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     // the producer starts streaming before the query tile is staged
     int produced = 0;
     auto produce = [&](int u) {                                     // u-th ring use: K(u/2) if even, V(u/2) if odd
-        const int st = u % n_stages;
+        const int st = ring_mod(u, alternate);
         const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1);
         const int row0 = tile.row0;
         const int boxes = (tile.len + kBoxRows - 1) / kBoxRows;
@@ -407,8 +414,8 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
         if (warp == 12 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
             for (int u = produced; u < 2 * n_it; ++u) {
-                const int st = u % n_stages;
-                if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), ((u / n_stages) - 1) & 1, abort_flag)) break;
+                const int st = ring_mod(u, alternate);
+                if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), (ring_div(u, alternate) - 1) & 1, abort_flag)) break;
                 produce(u);
             }
         } else if (warp == 13 && lane == 0) {
@@ -422,8 +429,8 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 const int w = n & 1;
                 const int it = alternate ? n : (n >> 1);
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
-                const int stk = (2 * it) % n_stages;
-                const int kuse = (n_stages & 1) ? it / n_stages : it / (n_stages >> 1);
+                const int stk = ring_mod(2 * it, alternate);
+                const int kuse = ring_uses(it, alternate);
                 if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t a0 = smem_desc(q_base + (alternate ? 0 : w) * kTileBytes, 16, 1024);
@@ -442,15 +449,18 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 const int w = n & 1, j = n >> 1;
                 const int it = alternate ? n : j;
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
-                const int uv = 2 * it + 1, stv = uv % n_stages;
-                const int vuse = (n_stages & 1) ? it / n_stages : uv / n_stages;   // value loads this stage has seen
+                const int stv = ring_mod(2 * it + 1, alternate);
+                const int vuse = ring_uses(it, alternate);                  // value loads this stage has seen
                 if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
                 if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
-                for (int kk = 0; kk < n_keys / 16; ++kk)            // 16 keys = 8 packed columns per instruction
-                    umma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o,
-                            (j > 0 || kk > 0));
+                const uint32_t o_tmem = tmem + 256 + w * 128, p_tmem = tmem + w * 128;
+                const int n_steps = n_keys >> 4;                    // 16 keys = 8 packed columns per instruction
+                umma_ts(o_tmem, p_tmem, b0, idesc_o, j > 0);
+#pragma unroll
+                for (int kk = 1; kk < kTile / 16; ++kk)
+                    if (kk < n_steps) umma_ts(o_tmem, p_tmem + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o, 1u);
                 umma_commit(smem_u32(&bars->o_done[w]));
                 if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 return true;
@@ -470,7 +480,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             const TileInfo tile = tile_info(s_meta, pv, ti0, it);
             const int len = tile.len;
             const float2* trig = pv.trig + (size_t)tile.doc * (kD / 2);
-            const int u = 2 * it, st = u % n_stages;
+            const int st = ring_mod(2 * it, alternate);
             float2 cs[8];
             if (LAYOUT == CF_ROPE_HALF) {
 #pragma unroll
@@ -482,7 +492,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                     cs[4 + e] = __ldg(trig + 32 + chunk * 4 + e);   // second half: dims 64 + chunk*8 ..
                 }
             }
-            const int kuse = (n_stages & 1) ? it / n_stages : u / n_stages;      // key loads this stage has seen
+            const int kuse = ring_uses(it, alternate);                        // key loads this stage has seen
             if (!mbar_wait(smem_u32(&bars->kv_full[st][0]), kuse & 1, abort_flag)) break;
             unsigned char* buf = smem + (ring_base - smem_base) + (size_t)st * kTileBytes;
 #pragma unroll 2
