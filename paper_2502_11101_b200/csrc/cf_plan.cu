@@ -125,6 +125,8 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     __shared__ int s_row[kMaxDocs + 1];   // first store row of every document (by local id), and the end
     __shared__ int s_dst[kMaxDocs];       // start positions by local id
     __shared__ int s_group[kMaxDocs];     // window index by local id
+    __shared__ int s_first[kMaxDocs];      // first tile by local id
+    __shared__ int s_cnt[kMaxDocs];       // tile count by local id
     __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
     __shared__ float s_score[kMaxDocs];
     __shared__ unsigned char s_flag[kMaxDocs];
@@ -304,34 +306,44 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         pv.query_start[b] = query_start;
     }
     if (fail) return;
+    // every array is written with consecutive threads on consecutive elements: per-document fields
+    // by document, the kept list by rank, the tile list by tile
+    if (tid < n_kept) {
+        s_tmp[tid] = first_tile;                             // first tile of rank tid (ascending)
+        s_score[tid] = __int_as_float(my_tiles);
+    }
+    __syncthreads();
+    if (tid < n_kept) {                                      // per-document view of the same numbers
+        const int id = s_ids[tid];
+        s_first[id] = first_tile;
+        s_cnt[id] = my_tiles;
+    }
+    __syncthreads();
     for (int i = tid; i < n_docs; i += kPlanThreads) {
         const bool kept = s_flag[i] != 0;
         pv.dst_start[doc0 + i] = kept ? s_dst[i] : -1;
         pv.group[doc0 + i] = kept ? s_group[i] : -1;
-        if (!kept) {
-            pv.doc_tile_count[doc0 + i] = 0;
-            pv.doc_tile_begin[doc0 + i] = 0;
-        }
+        pv.doc_tile_begin[doc0 + i] = kept ? base + s_first[i] : 0;
+        pv.doc_tile_count[doc0 + i] = kept ? s_cnt[i] : 0;
     }
-    if (tid < n_kept) {
-        const int r = tid;
-        const int id = s_ids[r];
-        const int i = doc0 + id;
+    if (tid < n_kept) pv.kept[doc0 + tid] = s_ids[tid];
+    for (int x = tid; x < total; x += kPlanThreads) {
+        int lo = 0, hi = n_kept;                             // last rank whose first tile is <= x
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_tmp[mid] <= x) lo = mid; else hi = mid;
+        }
+        const int id = s_ids[lo];
         const int row0 = s_row[id];
         const int len = s_row[id + 1] - row0;
-        const int first = base + first_tile;
-        const int count = my_tiles;
-        pv.kept[doc0 + r] = id;
-        pv.doc_tile_begin[i] = first;
-        pv.doc_tile_count[i] = count;
+        const int count = __float_as_int(s_score[lo]);
+        const int t = x - s_tmp[lo];
         // the document's rows are spread evenly over its tiles, in steps of 32 rows (160 rows make
         // tiles of 96 and 64, not 128 and 32), so consecutive tiles cost about the same
-        const int step = count > 0 ? min(kTile, ((len + count - 1) / count + 31) & ~31) : kTile;
-        for (int t = 0; t < count; ++t) {
-            pv.tile_doc[first + t] = i;
-            pv.tile_row0[first + t] = row0 + t * step;
-            pv.tile_len[first + t] = min(step, len - t * step);
-        }
+        const int step = min(kTile, ((len + count - 1) / count + 31) & ~31);
+        pv.tile_doc[base + x] = doc0 + id;
+        pv.tile_row0[base + x] = row0 + t * step;
+        pv.tile_len[base + x] = min(step, len - t * step);
     }
 
     // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D) -------------------------------
