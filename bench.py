@@ -311,6 +311,8 @@ def main():
     ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
     ap.add_argument("--per-layer", action="store_true",
                     help="one attention call per layer instead of one per run of layers between two pruning layers")
+    ap.add_argument("--skip-per-layer", action="store_true",
+                    help="do not also time the step with one attention call per layer")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
@@ -391,7 +393,7 @@ def main():
 
     # ---- the same step with one attention call per layer (what a running model can issue) ------
     per_layer = None
-    if wl.batch_layers and world == 1:
+    if wl.batch_layers and world == 1 and not args.skip_per_layer:
         main_graphs = graphs
         wl.batch_layers = False
         graphs = capture()
