@@ -32,6 +32,10 @@ if ROOT not in sys.path:
 from paper_2502_11101_b200 import workloads as W  # noqa: E402
 
 METRIC = "cached KV tokens/s through reposition+query-prefill attn"
+# DRAM bytes (read + write) of one attention-kernel launch, averaged over the four launches of a step of
+# workload 3 in the default configuration, from the ncu capture summarised in
+# profiles/attn_tc_kernel_workload3.md (102.7 MB per step).  Only valid for that kernel state and workload.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {("configs[2]", "layer-batched", "tcgen05"): 25.68e6}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 
@@ -447,7 +451,11 @@ def main():
     else:
         roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": gbs / peaks["hbm_gbs"]}
-    roofline.update({"traffic": None, "kernel": "fused re-position + query-prefill attention",
+    traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer",
+                   "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05")
+    traffic = None if args.layers else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
+    roofline.update({"traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write)",
+                     "algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()), "kernel": "fused re-position + query-prefill attention",
                      "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
                      "launches_timed": int(n), "hbm_gbs": gbs, "tflops": tfs,
                      "frac_of_applicable_roofline": max(t_hbm, t_tc) / dur_s})
