@@ -1,4 +1,5 @@
-"""Full-size runs in the launch configuration bench.py times (Session.run_stack), checked on sampled
+"""Full-size runs in the launch configurations bench.py times (Session.run_stack with one attention call
+per run of layers between two pruning layers, and with one call per layer), checked on sampled
 outputs the oracle computes one by one and on properties that hold at any size.
 
 Nothing the oracle consumes comes from the CUDA path: layer 1 attends every document in retrieval
@@ -14,7 +15,7 @@ from paper_2502_11101_b200.session import Session
 pytestmark = pytest.mark.gpu
 
 
-def _run_full(cfg, samples):
+def _run_full(cfg, samples, batch_layers):
     meta = W.make_meta(cfg, 0)
     dev = "cuda:0"
     q = W.make_q(meta, dev)
@@ -32,7 +33,7 @@ def _run_full(cfg, samples):
     out = torch.empty_like(q)
     lse = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), device=dev)
     scores = torch.empty((cfg.n_layers, meta.n_docs_total), device=dev)
-    sess.run_stack(q, k, v, cfg.schedule, oracle.ALLOC_ALIGN, out, lse, None, scores)
+    sess.run_stack(q, k, v, cfg.schedule, oracle.ALLOC_ALIGN, out, lse, None, scores, batch_layers=batch_layers)
     torch.cuda.synchronize()
     assert sess.status() == 0
     # ---- sampled outputs of layer 1 (all documents kept, retrieval order)
@@ -81,13 +82,17 @@ def _run_full(cfg, samples):
     return plan0
 
 
-def test_config4_full_size_sampled():
-    _run_full(W.CONFIGS[4], samples=[(0, 0), (1, 13), (3, 27)])
+@pytest.mark.parametrize("batch_layers", [True, False])
+def test_config4_full_size_sampled(batch_layers):
+    _run_full(W.CONFIGS[4], samples=[(0, 0), (1, 13), (3, 27)], batch_layers=batch_layers)
 
 
-def test_config5_four_layers_full_batch_sampled():
-    # the full 32-layer store is 90 GB; four layers keep the per-layer launch configuration (8 requests x
-    # 120 documents x 32 heads, six parallel windows) and hold 11 GB
-    cfg = W.scaled_config(W.CONFIGS[5], n_layers=4, schedule=((1, 60), (2, 30), (3, 15)))
-    plan0 = _run_full(cfg, samples=[(0, 0), (5, 17), (7, 31)])
+@pytest.mark.parametrize("batch_layers", [True, False])
+def test_config5_four_layers_full_batch_sampled(batch_layers):
+    # the full 32-layer store is 90 GB; four layers keep the launch configuration (8 requests x 120
+    # documents x 32 heads, six parallel windows) and hold 11 GB; the batched variant runs layers 1-2
+    # in one call
+    schedule = ((2, 60), (3, 30)) if batch_layers else ((1, 60), (2, 30), (3, 15))
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=4, schedule=schedule)
+    plan0 = _run_full(cfg, samples=[(0, 0), (5, 17), (7, 31)], batch_layers=batch_layers)
     assert all(int(x) == 6 for x in plan0["n_reuse"])
