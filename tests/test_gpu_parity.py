@@ -309,9 +309,10 @@ def test_degenerate_batches():
             cf.cf_set_attn_path(0)
         assert sess.status() == 0
         o = out.float().cpu().numpy()
-        # one-token document: the softmax has a single term, the output is that value row
+        # one-token document: the softmax has a single term, the output is that value row (to the
+        # tolerance of attention outputs: the one weight is a bf16 number near 1, not exactly 1)
         for h in range(hq):
-            assert np.allclose(o[0, :, h], v[0, h // 2].float().cpu().numpy(), atol=1e-2)
+            assert np.allclose(o[0, :, h], v[0, h // 2].float().cpu().numpy(), atol=1e-2, rtol=2e-2)
         assert np.all(o[1] == 0.0) and np.all(np.isneginf(lse[1].cpu().numpy()))   # nothing to attend
         s = sess.doc_scores.cpu().numpy()
         assert abs(s[0] - 1.0) < 1e-4 and abs(s[1] + s[2] - 1.0) < 1e-3
