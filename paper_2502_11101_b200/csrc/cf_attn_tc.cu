@@ -50,9 +50,8 @@ struct StoreMaps {
     CUtensorMap k[4], v[4];
 };
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
-constexpr int kMetaTiles = 64;                     // key tiles of a CTA whose description is staged in shared memory
-constexpr int kXchgBytes = 2048;                   // mailbox of the two warpgroups when they share a key tile
-constexpr int kSmemBytes = kSmemTiles * kTileBytes + 512 + kMetaTiles * 8 + kXchgBytes;   // tiles, barriers, tile list, mailbox
+constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
+constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512 + kMetaTiles * 8;   // tiles, alignment slack, barriers, tile list
 constexpr int kMaxStages = 6;
 constexpr int kRotateThreads = 192;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
@@ -66,11 +65,9 @@ struct Barriers {
     unsigned long long kv_full[kMaxStages][2];   // [stage][0 = keys, 1 = values]
     unsigned long long kv_empty[kMaxStages];
     unsigned long long k_ready[kMaxStages];
-    unsigned long long s_full[3];                // per S accumulator: two (one per warpgroup) or three (shared tile)
-    unsigned long long p_ready[3];
+    unsigned long long s_full[2];
+    unsigned long long p_ready[2];
     unsigned long long o_done[2];
-    unsigned long long pair_bar[4];              // shared tile: warp q of warpgroup 0 meets warp q of warpgroup 1
-    unsigned long long epi_bar;                  // shared tile: both warpgroups before the partial O leaves
     unsigned int tmem_base;
     volatile int abort_flag;
 };
@@ -282,13 +279,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
                float scale_log2, const __nv_bfloat16* __restrict__ q) {
-    extern __shared__ __align__(1024) unsigned char smem_raw[];    // 128-byte-swizzled tiles repeat every 1024 bytes
-    unsigned char* smem = smem_raw;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
-    if (smem_base & 1023u) {                                        // the alignment was not honoured: refuse to run
-        if (threadIdx.x == 0) atomicCAS(pv.status, 0, CF_ERR_CUDA);
-        return;
-    }
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -316,7 +309,6 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     const uint32_t ring_base = q_base + n_qt * kTileBytes;
     Barriers* bars = reinterpret_cast<Barriers*>(smem + kSmemTiles * kTileBytes);
     int2* s_meta = reinterpret_cast<int2*>(smem + kSmemTiles * kTileBytes + 512);
-    unsigned char* xchg = smem + kSmemTiles * kTileBytes + 512 + kMetaTiles * 8;
     volatile int* abort_flag = &bars->abort_flag;
 
     const int tbase = pv.tile_begin[b];
@@ -331,7 +323,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     // rows that will carry no data in one of the two parts: mark them neutral (m = -inf)
     for (int r = tid; r < rows_here; r += kThreads) {
         if (n_it <= 0) ws.part_m[slot0 + r] = -INFINITY;
-        ws.part_m[slot0 + rows_total + r] = -INFINITY;              // the CTA delivers one part; its twin stays empty
+        if (n_it <= 0 || !alternate || n_it < 2) ws.part_m[slot0 + rows_total + r] = -INFINITY;
     }
     if (n_it <= 0) return;
     const int ti0 = tbase + t_begin;                                // first tile of this CTA in the plan's list
@@ -362,16 +354,12 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             mbar_init(smem_u32(&bars->kv_empty[s]), 1);
             mbar_init(smem_u32(&bars->k_ready[s]), kRotateThreads);
         }
-        for (int w = 0; w < 3; ++w) {
-            // threads of warps that own rows: of one warpgroup, or of both when they share the tile
-            const int active = alternate ? 2 * 32 * ((rows_t0 + 31) / 32) : 32 * (((w ? rows_t1 : rows_t0) + 31) / 32);
+        for (int w = 0; w < 2; ++w) {
+            const int active = 32 * (((w ? rows_t1 : rows_t0) + 31) / 32);   // threads of warps that own rows
             mbar_init(smem_u32(&bars->s_full[w]), 1);
-            mbar_init(smem_u32(&bars->p_ready[w]), max(active, 1));
+            mbar_init(smem_u32(&bars->p_ready[w]), active);
+            mbar_init(smem_u32(&bars->o_done[w]), 1);
         }
-        mbar_init(smem_u32(&bars->o_done[0]), 1);
-        mbar_init(smem_u32(&bars->o_done[1]), 1);
-        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&bars->pair_bar[i]), 64);
-        mbar_init(smem_u32(&bars->epi_bar), 2 * 32 * ((rows_t0 + 31) / 32));
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -432,17 +420,13 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             }
         } else if (warp == 13 && lane == 0) {
             // -------------------------------------------------------------- MMA issue
-            // Side by side: sequence entry n is warpgroup w = n & 1 on key tile n >> 1, with S and O
-            // accumulators of its own (S_w, O_w); issue order S(0) S(1), then PV(n) followed by S(n + 2).
-            // Shared tile: entry n is key tile n on S accumulator n mod 3 and the one O accumulator;
-            // issue order S(0) S(1) S(2), then PV(n) followed by S(n + 3), so the QK^T of the next
-            // tiles runs while the warpgroups exponentiate.  In both, the QK^T that reuses an S
-            // accumulator follows, in the pipe, the PV that read the P aliased onto it.
+            // Sequence entry n: warpgroup w = n & 1, its item j = n >> 1, key tile = n (alternating)
+            // or j (side by side).  Issue order: S(0) S(1), then PV(n) followed by S(n + 2): the
+            // next QK^T of a warpgroup follows its own PV in the pipe, so S may overwrite the P it aliases.
             const uint32_t idesc_o = instr_desc(kD, true);
             const int n_seq = alternate ? n_it : 2 * n_it;
-            const int ahead = alternate ? 3 : 2;
             auto issue_s = [&](int n) -> bool {
-                const int w = alternate ? n % 3 : (n & 1);          // S accumulator
+                const int w = n & 1;
                 const int it = alternate ? n : (n >> 1);
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int stk = ring_mod(2 * it, alternate);
@@ -458,13 +442,12 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                     umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
                 umma_commit(smem_u32(&bars->s_full[w]));
-                if (alternate || (n & 1)) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
                 return true;
             };
             auto issue_pv = [&](int n) -> bool {
-                const int w = alternate ? n % 3 : (n & 1);          // S accumulator that holds P
-                const int j = alternate ? n / 3 : (n >> 1);         // earlier uses of that accumulator
-                const int it = alternate ? n : (n >> 1);
+                const int w = n & 1, j = n >> 1;
+                const int it = alternate ? n : j;
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int stv = ring_mod(2 * it + 1, alternate);
                 const int vuse = ring_uses(it, alternate);                  // value loads this stage has seen
@@ -472,21 +455,21 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
-                const uint32_t o_tmem = alternate ? tmem + 384 : tmem + 256 + w * 128, p_tmem = tmem + w * 128;
+                const uint32_t o_tmem = tmem + 256 + w * 128, p_tmem = tmem + w * 128;
                 const int n_steps = n_keys >> 4;                    // 16 keys = 8 packed columns per instruction
-                umma_ts(o_tmem, p_tmem, b0, idesc_o, it > 0);
+                umma_ts(o_tmem, p_tmem, b0, idesc_o, j > 0);
 #pragma unroll
                 for (int kk = 1; kk < kTile / 16; ++kk)
                     if (kk < n_steps) umma_ts(o_tmem, p_tmem + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o, 1u);
-                umma_commit(smem_u32(&bars->o_done[alternate ? 0 : w]));
-                if (alternate || (n & 1)) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
+                umma_commit(smem_u32(&bars->o_done[w]));
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 return true;
             };
-            bool ok = true;
-            for (int n = 0; n < ahead && n < n_seq && ok; ++n) ok = issue_s(n);
+            bool ok = issue_s(0);
+            if (ok && n_seq > 1) ok = issue_s(1);
             for (int n = 0; n < n_seq && ok; ++n) {
                 ok = issue_pv(n);
-                if (ok && n + ahead < n_seq) ok = issue_s(n + ahead);
+                if (ok && n + 2 < n_seq) ok = issue_s(n + 2);
             }
         }
     } else if (warp >= 8) {
@@ -546,162 +529,6 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             }
             fence_proxy_async();
             mbar_arrive(smem_u32(&bars->k_ready[st]));
-        }
-    } else if (alternate) {
-        // ------------------------------------------------------------------ softmax on a shared tile
-        // At most 128 query rows: both warpgroups work on the same key tile, thread r of each on
-        // row r, warpgroup 0 on the first 32-key chunks of the tile and warpgroup 1 on the rest.
-        // A thread loads its (at most two) chunks of S into registers, the two threads of a row
-        // agree on the row's reference maximum through a shared-memory mailbox (values rounded up
-        // to bf16 so that both compute with the identical number), and only then is P written --
-        // by then every S value of the tile sits in registers, so P may overwrite any S column.
-        const int w = warp >> 2;                                    // warpgroup
-        const int wq = warp & 3;                                    // warp within it = TMEM lane quarter
-        const int r = tid & 127;                                    // row = TMEM lane
-        const bool warp_active = wq * 32 < rows_here;
-        if (warp_active) {
-            const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-            const uint32_t o_addr = tmem + lane_addr + 384 + w * 64;                   // this thread's half of the O row
-            const bool row_valid = r < rows_here;
-            const size_t tile_row = (size_t)kvh * rows + rg * rg_rows + r;
-            float* tile_lse2 = ws.tile_lse2 + (size_t)layer * ws.max_tiles * rows_total;
-            __nv_bfloat16* xmax = reinterpret_cast<__nv_bfloat16*>(xchg);             // [2][2][128] half-tile maxima
-            float* xsum = reinterpret_cast<float*>(xchg + 1024);                      // [2][128] sums of warpgroup 1
-            const uint32_t pair_bar = smem_u32(&bars->pair_bar[wq]);
-            const uint32_t o_done = smem_u32(&bars->o_done[0]);
-            int pair_phase = 0, o_seen = 0;                         // o_seen: completed PVs this thread has observed
-            float m_ref = -INFINITY, l_half = 0.f, prev_sum = 0.f, prev_m = 0.f;
-            bool ok = true;
-            auto meet = [&]() -> bool {                             // the two warps that share these 32 rows
-                mbar_arrive(pair_bar);
-                const bool done = mbar_wait(pair_bar, pair_phase, abort_flag);
-                pair_phase ^= 1;
-                return done;
-            };
-            auto see_pv = [&](int count) -> bool {                  // observe the completion of PV(0..count-1), in order
-                while (o_seen < count) {
-                    if (!mbar_wait(o_done, o_seen & 1, abort_flag)) return false;
-                    ++o_seen;
-                }
-                tc_fence_after();
-                return true;
-            };
-            for (int t = 0; t < n_it && ok; ++t) {
-                const int buf = t % 3;
-                const int len = tile_info(s_meta, pv, ti0, t).len;
-                const int chunks = (len + 31) >> 5;                 // 1..4
-                const int c0 = (chunks + 1) >> 1;                   // chunks of warpgroup 0
-                const int c_begin = w ? c0 : 0, n_c = w ? chunks - c0 : c0;
-                const uint32_t s_addr = tmem + lane_addr + buf * 128;
-                ok = mbar_wait(smem_u32(&bars->s_full[buf]), (t / 3) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t va[32], vb[32];
-                if (n_c > 0) tmem_ld32_async(s_addr + c_begin * 32, va);
-                if (n_c > 1) tmem_ld32_async(s_addr + (c_begin + 1) * 32, vb);
-                tmem_ld_wait(va);
-                tmem_ld_wait(vb);
-                const int valid_a = len - c_begin * 32, valid_b = valid_a - 32;
-                float hmax = -INFINITY;
-                if (n_c > 0) hmax = valid_a >= 32 ? chunk_max<false>(va, 32) : chunk_max<true>(va, valid_a);
-                if (n_c > 1) hmax = fmaxf(hmax, valid_b >= 32 ? chunk_max<false>(vb, 32) : chunk_max<true>(vb, valid_b));
-                const __nv_bfloat16 mine = __float2bfloat16_ru(hmax * scale_log2);    // -inf stays -inf
-                xmax[((t & 1) * 2 + w) * 128 + r] = mine;
-                ok = meet();
-                if (!ok) break;
-                const float cmax = fmaxf(__bfloat162float(mine), __bfloat162float(xmax[((t & 1) * 2 + (w ^ 1)) * 128 + r]));
-                if (w == 0 && t > 0 && row_valid)                   // the previous tile's mass, now that both halves are known
-                    tile_lse2[(size_t)(ti0 + t - 1) * rows_total + tile_row] = prev_m + log2f(prev_sum + xsum[((t - 1) & 1) * 128 + r]);
-                const bool move = cmax > m_ref + kRescaleThreshold;                  // first tile: m_ref = -inf
-                if (__any_sync(0xffffffffu, move)) {
-                    float alpha = 1.f;
-                    if (move) {
-                        alpha = fast_exp2(m_ref - cmax);            // 0 when nothing is accumulated yet
-                        m_ref = cmax;
-                    }
-                    if (t > 0) {                                    // O holds PV(0..t-1): wait for the last of them
-                        ok = see_pv(t);
-                        if (!ok) break;
-                        for (int cc = 0; cc < 4; ++cc) {
-                            uint32_t o[16];
-                            tmem_ld16(o_addr + cc * 16, o);
-#pragma unroll
-                            for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                            tmem_st16(o_addr + cc * 16, o);
-                        }
-                    }
-                    l_half *= alpha;
-                }
-                float tile_sum = 0.f;
-                if (n_c > 0) {
-                    tile_sum += valid_a >= 32 ? chunk_exp<false>(va, 32, scale_log2, -m_ref) : chunk_exp<true>(va, valid_a, scale_log2, -m_ref);
-                    tmem_st16_async(s_addr + c_begin * 16, va);
-                }
-                if (n_c > 1) {
-                    tile_sum += valid_b >= 32 ? chunk_exp<false>(vb, 32, scale_log2, -m_ref) : chunk_exp<true>(vb, valid_b, scale_log2, -m_ref);
-                    tmem_st16_async(s_addr + (c_begin + 1) * 16, vb);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                // PV(t-1) was issued a softmax ago; observing it here keeps this thread within one
-                // phase of the barrier (PV(t) cannot complete before this thread's arrival below)
-                if (t > 0) {
-                    ok = see_pv(t);
-                    if (!ok) break;
-                }
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars->p_ready[buf]));
-                l_half += tile_sum;
-                if (w) {
-                    xsum[(t & 1) * 128 + r] = tile_sum;
-                } else {
-                    prev_sum = tile_sum;
-                    prev_m = m_ref;
-                }
-            }
-            if (ok) {
-                if (w) xsum[(n_it & 1) * 128 + r] = l_half;         // the slot of tile n_it - 2, read long ago
-                ok = meet();
-            }
-            if (ok && w == 0 && row_valid) {
-                tile_lse2[(size_t)(ti0 + n_it - 1) * rows_total + tile_row] = prev_m + log2f(prev_sum + xsum[((n_it - 1) & 1) * 128 + r]);
-                ws.part_m[slot0 + r] = m_ref;
-                ws.part_l[slot0 + r] = l_half + xsum[(n_it & 1) * 128 + r];
-            }
-            if (ok) ok = see_pv(n_it);
-            if (ok) {
-                // Partial O row: this thread's 64 columns go to shared memory (the query tile, which no
-                // MMA reads any more), then full 256-byte rows leave with coalesced stores.
-                unsigned char* stage = smem;
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(o_addr + c * 32, o);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {                   // 8 dims = one 16-byte chunk
-                        const int chunk = w * 8 + c * 4 + i;
-                        *reinterpret_cast<uint4*>(stage + r * 256 + ((chunk ^ (r & 15)) << 4)) =
-                            make_uint4(pack_bf16(__uint_as_float(o[8 * i]), __uint_as_float(o[8 * i + 1])),
-                                       pack_bf16(__uint_as_float(o[8 * i + 2]), __uint_as_float(o[8 * i + 3])),
-                                       pack_bf16(__uint_as_float(o[8 * i + 4]), __uint_as_float(o[8 * i + 5])),
-                                       pack_bf16(__uint_as_float(o[8 * i + 6]), __uint_as_float(o[8 * i + 7])));
-                    }
-                }
-                mbar_arrive(smem_u32(&bars->epi_bar));
-                ok = mbar_wait(smem_u32(&bars->epi_bar), 0, abort_flag);
-                if (ok) {
-                    const int row0 = wq * 32 + w * 16;              // this warp's 16 rows
-                    const int rows_left = rows_here - row0;
-                    unsigned char* dst = reinterpret_cast<unsigned char*>(ws.part_o) + (slot0 + row0) * (size_t)(kD * 2);
-#pragma unroll 4
-                    for (int i = 0; i < 8; ++i) {                   // two rows per step, 16 lanes each
-                        const int rr = 2 * i + (lane >> 4), chunk = lane & 15;
-                        if (rr < rows_left) {
-                            const int srow = row0 + rr;
-                            const uint4 val = *reinterpret_cast<const uint4*>(stage + srow * 256 + ((chunk ^ (srow & 15)) << 4));
-                            *reinterpret_cast<uint4*>(dst + (size_t)rr * (kD * 2) + chunk * 16) = val;
-                        }
-                    }
-                }
-            }
         }
     } else {
         // ------------------------------------------------------------------ softmax, one row per thread
