@@ -347,19 +347,24 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     }
 
     // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D) -------------------------------
-    for (int idx = tid; idx < n_kept * half; idx += kPlanThreads) {
-        const int r = idx >> half_log2, p = idx & (half - 1);            // half is 32 or 64
-        const int id = s_ids[r];
-        const int delta = s_dst[id] - s_src[id];
-        float2 entry;
-        if (gv.dtype == CF_BF16) {
-            sincos_turns(delta, inv_freq.turns[p], entry.y, entry.x);
-        } else {
-            double sn, cs;
-            sincos_reduced((double)delta * inv_freq.f[p], sn, cs);
-            entry = make_float2((float)cs, (float)sn);
+    // thread = (slice p, every (kPlanThreads / half)-th rank): the frequency is read once per thread
+    {
+        const int p = tid & (half - 1);
+        const unsigned long long turns = inv_freq.turns[p];
+        const double freq = inv_freq.f[p];
+        for (int r = tid >> half_log2; r < n_kept; r += kPlanThreads >> half_log2) {
+            const int id = s_ids[r];
+            const int delta = s_dst[id] - s_src[id];
+            float2 entry;
+            if (gv.dtype == CF_BF16) {
+                sincos_turns(delta, turns, entry.y, entry.x);
+            } else {
+                double sn, cs;
+                sincos_reduced((double)delta * freq, sn, cs);
+                entry = make_float2((float)cs, (float)sn);
+            }
+            pv.trig[(size_t)(doc0 + id) * half + p] = entry;
         }
-        pv.trig[(size_t)(doc0 + id) * half + p] = entry;
     }
 }
 
