@@ -81,3 +81,20 @@ def test_schedule_matches_oracle_and_printed_example(lib, golden):
     assert [k for _, k in sched] == [35, 30, 25, 20, 15, 10, 5]
     for L, n, k, kf in [(28, 4, 50, 5), (32, 4, 120, 15), (3, 4, 10, 2), (28, 7, 33, 4)]:
         assert cf.cf_schedule_linear(L, n, k, kf) == oracle.prune_schedule_linear(L, n, k, kf)
+
+
+def test_workspace_size_of_layer_batched_calls(lib):
+    """Host arithmetic only: the descriptor's device pointers are never dereferenced by these calls."""
+    geom = cf.make_geom(12, 2, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256                                            # any non-null address
+    batch = cf.cf_batch(1, 50, 48, 0, 48, 0, 0, 0, 8000, 2 * 128, fake, fake, fake)
+    one = cf.cf_attn_workspace_bytes(geom, batch)
+    assert one > 0 and one == cf.cf_attn_workspace_bytes_layers(geom, batch, 1)
+    for n_layers in (2, 8, cf.CF_MAX_LAYERS_PER_CALL):
+        need = cf.cf_attn_workspace_bytes_layers(geom, batch, n_layers)
+        assert need > 0 and need % 256 == 0
+        # per layer: the merged log-sum-exp of every row and one value per (tile slot, row)
+        rows, tile_slots = 12 * 48, 50 + 8000 // 128 + 1
+        assert need >= n_layers * 4 * (rows + tile_slots * rows)
+    assert cf.cf_attn_workspace_bytes_layers(geom, batch, 0) == 0
+    assert cf.cf_attn_workspace_bytes_layers(geom, batch, cf.CF_MAX_LAYERS_PER_CALL + 1) == 0
