@@ -13,12 +13,6 @@ import torch
 from . import binding as B
 
 
-def _share_memory(a: torch.Tensor, b: torch.Tensor) -> bool:
-    """True unless the storages of `a` and `b` are disjoint address ranges."""
-    sa, sb = a.untyped_storage(), b.untyped_storage()
-    return not (sa.data_ptr() + sa.nbytes() <= sb.data_ptr() or sb.data_ptr() + sb.nbytes() <= sa.data_ptr())
-
-
 class Session:
     def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: torch.dtype, pos_range: int,
                  rope_theta: float, q_len: int, doc_len: np.ndarray, req_doc_begin: np.ndarray,
@@ -47,7 +41,6 @@ class Session:
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()) if self.n_requests else 0)
         self.workspace = torch.empty(256, dtype=torch.uint8, device=self.device)
         self.reserve_workspace(1)
-        self._side = None           # second stream for work that is independent of the layer loop (run_stack)
         self.doc_scores = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
         self.score_accum = torch.zeros(self.n_docs_total, dtype=torch.float32, device=self.device)
 
@@ -119,28 +112,9 @@ class Session:
         lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores.
 
         With `batch_layers` the layers between two pruning layers go to the library in one call
-        (possible here because every layer's query states are given up front).
-
-        Phase 2 only needs the plan as the last pruning layer left it, so when `k_final` is a buffer
-        of its own it is issued right after that pruning step on a second stream and runs beside the
-        remaining layers; the calling stream waits for it before this method returns."""
+        (possible here because every layer's query states are given up front)."""
         sched = dict(schedule)
         n_layers = q.shape[0]
-        last_prune = max((l for l in sched if l <= n_layers), default=0)
-        main = torch.cuda.current_stream(self.device)
-        overlap = k_final is not None and 0 < last_prune < n_layers and not _share_memory(k, k_final)
-        forked = False
-
-        def phase2_beside(layer_done: int) -> bool:
-            if not overlap or layer_done != last_prune:
-                return False
-            if self._side is None:
-                self._side = torch.cuda.Stream(device=self.device)
-            self._side.wait_stream(main)
-            with torch.cuda.stream(self._side):
-                self.reposition(k, k_final, n_layers, k.stride(0))
-            return True
-
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))
         self.init()
         if batch_layers:
@@ -153,7 +127,6 @@ class Session:
                                        None if layer_scores is None else layer_scores[lo:hi])
                 if last in sched:
                     self.prune(sched[last], strategy)
-                    forked = phase2_beside(last) or forked
                 first = last
         else:
             for layer in range(1, n_layers + 1):
@@ -163,8 +136,5 @@ class Session:
                     layer_scores[i].copy_(self.doc_scores)
                 if layer in sched:
                     self.prune(sched[layer], strategy)
-                    forked = phase2_beside(layer) or forked
-        if forked:
-            main.wait_stream(self._side)
-        elif k_final is not None:
+        if k_final is not None:
             self.reposition(k, k_final, n_layers, k.stride(0))
