@@ -330,3 +330,10 @@ def test_degenerate_batches():
     torch.cuda.synchronize()
     assert sess.status() == 0 and sess.read_plan()["order"] == [[], [], []]
     assert np.all(out.float().cpu().numpy() == 0.0) and np.all(sess.doc_scores.cpu().numpy() == 0.0)
+
+
+def test_store_smaller_than_one_tile():
+    """A store of five rows in all: every bulk copy reaches past the end of the store."""
+    cfg = W.WorkloadConfig("five-rows", 2, 4, 2, 128, "bf16", 1e4, 4096, 1, 5, 5, 3, 1, 1, ())
+    for batch_layers in (False, True):
+        harness.run_and_compare(cfg, 0, oracle.ALLOC_ALIGN, min_margin=0.0, batch_layers=batch_layers)
