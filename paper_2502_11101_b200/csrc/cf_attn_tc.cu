@@ -16,13 +16,10 @@
 // the combine kernel.  Warp roles (512 threads):
 //   warps 0-3    softmax warpgroup 0 (thread = query row = TMEM lane)
 //   warps 4-7    softmax warpgroup 1
-//   warps 8-11, 14  key rotation in shared memory
-//   warp 12      TMA producer (one lane)
-//   warp 13      TMEM allocation; one lane issues the MMAs of warpgroup 0
-//   warp 15      one lane issues the MMAs of warpgroup 1
-// Each warpgroup has an MMA-issuing thread of its own (PV of a tile, then the QK^T of its next
-// tile), so neither waits behind the other's instructions and one warpgroup's exponentials
-// overlap the other's tensor-core work.
+//   warps 8-11, 14, 15  key rotation in shared memory
+//   warp 12      TMA producer (one lane)     warp 13  TMEM allocation and MMA issue (one lane)
+// The MMA warp interleaves the two warpgroups (PV of one, then the next QK^T of the same one), so
+// one warpgroup's exponentials overlap the other's tensor-core work.
 // The softmax is single-pass: the reference maximum of a row only moves when a 32-key chunk exceeds
 // it by more than 2^8, in which case O, the sums and the P columns already written are rescaled
 // (rare after the first chunk); any reference within the exponent range is exact enough because
@@ -56,7 +53,7 @@ constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 r
 constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
 constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512 + kMetaTiles * 8;   // tiles, alignment slack, barriers, tile list
 constexpr int kMaxStages = 6;
-constexpr int kRotateThreads = 160;
+constexpr int kRotateThreads = 192;
 constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
 constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference maximum moves only
                                                    // when a tile exceeds it by more than 2^8
@@ -354,7 +351,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars->kv_full[s][0]), 1);
             mbar_init(smem_u32(&bars->kv_full[s][1]), 1);
-            mbar_init(smem_u32(&bars->kv_empty[s]), alternate ? 1 : 2);   // MMA issuers that read the stage
+            mbar_init(smem_u32(&bars->kv_empty[s]), 1);
             mbar_init(smem_u32(&bars->k_ready[s]), kRotateThreads);
         }
         for (int w = 0; w < 2; ++w) {
@@ -413,7 +410,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     // Work of warpgroup w: item j uses key tile kt(w, j) and query tile qt(w).
     //   side by side (two row tiles): kt = j,          n_items = n_it
     //   alternating  (one row tile):  kt = 2 j + w,    n_items = ceil((n_it - w) / 2)
-    if (warp == 12 || warp == 13 || warp == 15) {
+    if (warp == 12 || warp == 13) {
         if (warp == 12 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
             for (int u = produced; u < 2 * n_it; ++u) {
@@ -421,17 +418,16 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (u >= n_stages && !mbar_wait(smem_u32(&bars->kv_empty[st]), (ring_div(u, alternate) - 1) & 1, abort_flag)) break;
                 produce(u);
             }
-        } else if (warp != 12 && lane == 0) {
-            // -------------------------------------------------------------- MMA issue for warpgroup w
-            // Item j of warpgroup w is key tile 2 j + w (alternating) or j (side by side).  Issue
-            // order: S(0), then PV(j) followed by S(j + 1): the next QK^T follows the PV in the pipe,
-            // so it may overwrite the P that PV reads (P is aliased onto S).
-            const int w = warp == 13 ? 0 : 1;
-            const int n_items = alternate ? (n_it - w + 1) / 2 : n_it;
+        } else if (warp == 13 && lane == 0) {
+            // -------------------------------------------------------------- MMA issue
+            // Sequence entry n: warpgroup w = n & 1, its item j = n >> 1, key tile = n (alternating)
+            // or j (side by side).  Issue order: S(0) S(1), then PV(n) followed by S(n + 2): the
+            // next QK^T of a warpgroup follows its own PV in the pipe, so S may overwrite the P it aliases.
             const uint32_t idesc_o = instr_desc(kD, true);
-            const uint32_t s_tmem = tmem + w * 128, o_tmem = tmem + 256 + w * 128;
-            auto issue_s = [&](int j) -> bool {
-                const int it = alternate ? 2 * j + w : j;
+            const int n_seq = alternate ? n_it : 2 * n_it;
+            auto issue_s = [&](int n) -> bool {
+                const int w = n & 1;
+                const int it = alternate ? n : (n >> 1);
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int stk = ring_mod(2 * it, alternate);
                 const int kuse = ring_uses(it, alternate);
@@ -443,14 +439,15 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {                    // 16 dims per instruction
                     const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-                    umma(s_tmem, a0 + off, b0 + off, idesc_s, kk > 0);
+                    umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
                 umma_commit(smem_u32(&bars->s_full[w]));
-                umma_commit(smem_u32(&bars->kv_empty[stk]));        // this reader is done with the keys
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
                 return true;
             };
-            auto issue_pv = [&](int j) -> bool {
-                const int it = alternate ? 2 * j + w : j;
+            auto issue_pv = [&](int n) -> bool {
+                const int w = n & 1, j = n >> 1;
+                const int it = alternate ? n : j;
                 const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
                 const int stv = ring_mod(2 * it + 1, alternate);
                 const int vuse = ring_uses(it, alternate);                  // value loads this stage has seen
@@ -458,24 +455,26 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
+                const uint32_t o_tmem = tmem + 256 + w * 128, p_tmem = tmem + w * 128;
                 const int n_steps = n_keys >> 4;                    // 16 keys = 8 packed columns per instruction
-                umma_ts(o_tmem, s_tmem, b0, idesc_o, j > 0);
+                umma_ts(o_tmem, p_tmem, b0, idesc_o, j > 0);
 #pragma unroll
                 for (int kk = 1; kk < kTile / 16; ++kk)
-                    if (kk < n_steps) umma_ts(o_tmem, s_tmem + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o, 1u);
+                    if (kk < n_steps) umma_ts(o_tmem, p_tmem + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o, 1u);
                 umma_commit(smem_u32(&bars->o_done[w]));
-                umma_commit(smem_u32(&bars->kv_empty[stv]));        // this reader is done with the values
+                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
                 return true;
             };
-            bool ok = n_items > 0 && issue_s(0);
-            for (int j = 0; j < n_items && ok; ++j) {
-                ok = issue_pv(j);
-                if (ok && j + 1 < n_items) ok = issue_s(j + 1);
+            bool ok = issue_s(0);
+            if (ok && n_seq > 1) ok = issue_s(1);
+            for (int n = 0; n < n_seq && ok; ++n) {
+                ok = issue_pv(n);
+                if (ok && n + 2 < n_seq) ok = issue_s(n + 2);
             }
         }
     } else if (warp >= 8) {
         // ------------------------------------------------------------------ key rotation (Eq. 5)
-        const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..159 (warps 8-11, 14)
+        const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
         const int chunk = t & 7, rsub = t >> 3;
         for (int it = 0; it < n_it; ++it) {
             const TileInfo tile = tile_info(s_meta, pv, ti0, it);
