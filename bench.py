@@ -320,11 +320,21 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
+    ap.add_argument("--schedule", default="config", choices=["config", "linear"],
+                    help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
+                         "a constant number of documents, down to 5)")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
     if args.layers:
         cfg = W.scaled_config(cfg, n_layers=args.layers,
                               schedule=tuple(s for s in cfg.schedule if s[0] <= args.layers))
+    if args.schedule == "linear":
+        # App. C, integers only: prune after layers 4, 8, ...; floor((k - k_finish) / prunes) documents each
+        # time, the remainder at the last pruning layer
+        prunes = cfg.n_layers // 4
+        step_docs = (cfg.n_docs - 5) // max(prunes, 1)
+        cfg = W.scaled_config(cfg, schedule=tuple((4 * j, 5 if j == prunes else cfg.n_docs - j * step_docs)
+                                                  for j in range(1, prunes + 1)))
     rank, world, local = dist_env()
 
     if args.impl == "reference":
@@ -453,7 +463,7 @@ def main():
                     "frac": gbs / peaks["hbm_gbs"]}
     traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer",
                    "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05")
-    traffic = None if args.layers else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
+    traffic = None if (args.layers or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
     roofline.update({"traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write)",
                      "algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()), "kernel": "fused re-position + query-prefill attention",
                      "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
@@ -519,7 +529,7 @@ def main():
             "config": {"workload": f"configs[{args.workload - 1}] {cfg.name}", "n_layers": cfg.n_layers,
                        "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                        "docs_per_request": cfg.n_docs, "requests": cfg.batch, "q_len": cfg.q_len,
-                       "schedule": [list(s) for s in cfg.schedule], "strategy": "align",
+                       "schedule": [list(s) for s in cfg.schedule], "schedule_kind": args.schedule, "strategy": "align",
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
                              f"{slot_mb:.0f} MB) cycled between steps",

@@ -337,3 +337,23 @@ def test_store_smaller_than_one_tile():
     cfg = W.WorkloadConfig("five-rows", 2, 4, 2, 128, "bf16", 1e4, 4096, 1, 5, 5, 3, 1, 1, ())
     for batch_layers in (False, True):
         harness.run_and_compare(cfg, 0, oracle.ALLOC_ALIGN, min_margin=0.0, batch_layers=batch_layers)
+
+
+@pytest.mark.parametrize("heads", [(32, 32), (12, 2)])
+def test_single_query_row(heads):
+    """q_len = 1 (the shape of a decoding step over the kept caches): one row per head."""
+    cfg = W.WorkloadConfig("one-row", 2, heads[0], heads[1], 128, "bf16", 1e4, 4096, 8, 100, 200, 1, 2, 2, ((1, 4),))
+    for batch_layers in (False, True):
+        harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3,
+                                batch_layers=batch_layers)
+
+
+def test_linear_pruning_schedule_of_the_paper():
+    """App. C: prune every n = 4 layers by a constant amount down to k_finish = 5 (schedule from the library)."""
+    import paper_2502_11101_b200 as cf
+    base = W.CONFIGS[3]
+    schedule = tuple(cf.cf_schedule_linear(base.n_layers, 4, base.n_docs, 5))
+    assert schedule == tuple(oracle.prune_schedule_linear(base.n_layers, 4, base.n_docs, 5)) and len(schedule) == 7
+    cfg = W.scaled_config(base, schedule=schedule)
+    harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3,
+                            batch_layers=True)
