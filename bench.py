@@ -62,7 +62,7 @@ class ClockSampler:
         self.thread = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -343,7 +343,7 @@ def main():
         run_reference(args, cfg, rank)
         return
 
-    args.steps = 300 if args.steps is None else args.steps
+    args.steps = 3000 if args.steps is None else args.steps      # about half a second: several clock samples
     args.warmup = 10 if args.warmup is None else max(3, args.warmup)
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     torch.cuda.set_device(local)
