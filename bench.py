@@ -320,6 +320,7 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
+    ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
     ap.add_argument("--schedule", default="config", choices=["config", "linear"],
                     help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
                          "a constant number of documents, down to 5)")
@@ -328,6 +329,8 @@ def main():
     if args.layers:
         cfg = W.scaled_config(cfg, n_layers=args.layers,
                               schedule=tuple(s for s in cfg.schedule if s[0] <= args.layers))
+    if args.q_len:
+        cfg = W.scaled_config(cfg, q_len=args.q_len)
     if args.schedule == "linear":
         # App. C, integers only: prune after layers 4, 8, ...; floor((k - k_finish) / prunes) documents each
         # time, the remainder at the last pruning layer
@@ -463,7 +466,7 @@ def main():
                     "frac": gbs / peaks["hbm_gbs"]}
     traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer",
                    "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05")
-    traffic = None if (args.layers or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
+    traffic = None if (args.layers or args.q_len or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
     roofline.update({"traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write)",
                      "algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()), "kernel": "fused re-position + query-prefill attention",
                      "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
