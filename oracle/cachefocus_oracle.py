@@ -208,6 +208,43 @@ def query_prefill_attn(q: np.ndarray, k_rot: np.ndarray, v_store: np.ndarray,
 
 
 # ----------------------------------------------------------------------------- pruning
+def query_self_block(q: np.ndarray, k_self: np.ndarray, v_self: np.ndarray,
+                     scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 1 for the query tokens over their own keys and values, with the causal mask the footnote
+    to Eq. 1 refers to: query row j sees the query tokens 0..j.
+
+    q[Lq, Hq, D]; k_self, v_self[Lq, Hkv, D] (keys encoded at the query's positions).
+    Returns out[Lq, Hq, D] and lse[Hq, Lq] of this block alone."""
+    q = np.asarray(q, dtype=np.float64)
+    k_self = np.asarray(k_self, dtype=np.float64)
+    v_self = np.asarray(v_self, dtype=np.float64)
+    lq, hq, d = q.shape
+    g = hq // k_self.shape[1]
+    if scale is None or scale == 0.0:
+        scale = 1.0 / math.sqrt(d)
+    out = np.zeros((lq, hq, d))
+    lse = np.zeros((hq, lq))
+    for h in range(hq):
+        kvh = h // g
+        for j in range(lq):
+            s = (k_self[:j + 1, kvh, :] @ q[j, h, :]) * scale
+            m = s.max()
+            e = np.exp(s - m)
+            out[j, h, :] = (e / e.sum()) @ v_self[:j + 1, kvh, :]
+            lse[h, j] = m + math.log(e.sum())
+    return out, lse
+
+
+def merge_softmax_blocks(out_a: np.ndarray, lse_a: np.ndarray, out_b: np.ndarray, lse_b: np.ndarray
+                         ) -> Tuple[np.ndarray, np.ndarray]:
+    """Softmax attention over the union of two disjoint key sets from the results over each:
+    the outputs are averaged with weights exp(lse) (out[Lq, Hq, D], lse[Hq, Lq])."""
+    lse = np.logaddexp(lse_a, lse_b)
+    wa = np.exp(lse_a - lse).T[:, :, None]
+    wb = np.exp(lse_b - lse).T[:, :, None]
+    return wa * out_a + wb * out_b, lse
+
+
 def prune_topk(score_accum: Sequence[float], order: Sequence[int], keep: int, strategy: int
                ) -> List[int]:
     """Algorithm 2, pruning step: among the documents in `order` keep the `keep` with the

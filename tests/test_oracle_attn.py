@@ -219,3 +219,64 @@ def test_stack_follows_algorithm2(strategy):
         at_prune = res["layers"][2]["score_accum"]
         assert [at_prune[i] for i in order] == sorted([at_prune[i] for i in order], reverse=True)
         assert len(final) == 2
+
+
+def test_self_block_and_merge_equal_textbook_causal_attention():
+    """Documents in one window (N_reuse = 1) followed by the query: attention of the query rows over
+    the re-positioned caches, merged with the causal query-self block, is ordinary causal attention
+    over the whole sequence with every key encoded directly at its final position (library routine)."""
+    import torch
+    rng = np.random.default_rng(5)
+    hq, hkv, d, lq, theta = 4, 2, 16, 6, 1e4
+    doc_len = [5, 9, 3]
+    offsets = np.concatenate([[0], np.cumsum(doc_len)])
+    total = int(offsets[-1])
+    raw_k = rng.standard_normal((total, hkv, d))
+    v_docs = rng.standard_normal((total, hkv, d))
+    raw_q = rng.standard_normal((lq, hq, d))
+    raw_kq = rng.standard_normal((lq, hkv, d))
+    v_q = rng.standard_normal((lq, hkv, d))
+    src = [0, 0, 0]
+    def at(x, first):                                              # encode token t of x at position first + t
+        return oracle.rope_rotate(x, (first + np.arange(x.shape[0]))[:, None] * np.ones((1, x.shape[1])), theta)
+    k_store = np.concatenate([at(raw_k[offsets[i]:offsets[i + 1]], src[i]) for i in range(3)])
+    order = [2, 0, 1]
+    dst, _, n_reuse, qs = oracle.allocate_positions(doc_len, order, 64, n_reuse=1, query_start=40)
+    assert n_reuse == 1
+    k_rot = oracle.reposition_keys(k_store, offsets, src, dst, order, theta)
+    q = at(raw_q, qs)
+    k_self = at(raw_kq, qs)
+    o_docs, lse_docs, _, _ = oracle.query_prefill_attn(q, k_rot, v_docs, offsets, order, 3)
+    o_self, lse_self = oracle.query_self_block(q, k_self, v_q)
+    o_full, lse_full = oracle.merge_softmax_blocks(o_docs, lse_docs, o_self, lse_self)
+    # the same thing as one sequence: documents sorted by position, then the query tokens
+    by_pos = sorted(range(3), key=lambda i: dst[i])
+    keys = np.concatenate([at(raw_k[offsets[i]:offsets[i + 1]], dst[i]) for i in by_pos] + [k_self])
+    vals = np.concatenate([v_docs[offsets[i]:offsets[i + 1]] for i in by_pos] + [v_q])
+    n = keys.shape[0]
+    q_all = np.zeros((n, hq, d))
+    q_all[n - lq:] = q
+    g = hq // hkv
+    qt = torch.from_numpy(q_all).permute(1, 0, 2)                      # [Hq, n, D]
+    kt = torch.from_numpy(keys).permute(1, 0, 2).repeat_interleave(g, dim=0)
+    vt = torch.from_numpy(vals).permute(1, 0, 2).repeat_interleave(g, dim=0)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True).permute(1, 0, 2).numpy()
+    assert np.allclose(o_full, ref[n - lq:], atol=1e-12)
+    # the merged denominator is the denominator over the union
+    s = np.einsum("jhd,thd->hjt", q, np.repeat(keys, g, axis=1)) / np.sqrt(d)
+    mask = np.arange(n)[None, :] <= (n - lq + np.arange(lq))[:, None]
+    lse_ref = np.log(np.where(mask[None], np.exp(s), 0.0).sum(axis=2))
+    assert np.allclose(lse_full, lse_ref, atol=1e-12)
+
+
+def test_merge_of_two_halves_is_attention_over_the_whole():
+    rng = np.random.default_rng(6)
+    lq, hq, d, t = 3, 2, 8, 10
+    q = rng.standard_normal((lq, hq, d))
+    k = rng.standard_normal((t, hq, d))
+    v = rng.standard_normal((t, hq, d))
+    whole = oracle.query_prefill_attn(q, k, v, [0, t], [0], 1)
+    a = oracle.query_prefill_attn(q, k[:4], v[:4], [0, 4], [0], 1)
+    b = oracle.query_prefill_attn(q, k[4:], v[4:], [0, 6], [0], 1)
+    out, lse = oracle.merge_softmax_blocks(a[0], a[1], b[0], b[1])
+    assert np.allclose(out, whole[0], atol=1e-13) and np.allclose(lse, whole[1], atol=1e-13)
