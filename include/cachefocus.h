@@ -225,6 +225,26 @@ int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, con
                                  float* lse, float* doc_scores, float* score_accum,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* The whole attention of the query tokens in layer_l (Algorithm 2): over the kept documents' caches
+ * as in cf_query_prefill_attn_layers, and over the query tokens themselves under the causal mask
+ * that the footnote to Eq. 1 refers to (query row j sees query tokens 0..j), merged into one softmax.
+ *   k_self, v_self  device, keys and values of the query tokens, keys already encoded at
+ *                   query_start + j: layer i at + i * self_layer_stride elements, each layer
+ *                   [n_requests][q_len][n_kv_heads][head_dim]; q_len <= 128
+ *   out, lse        cover both key sets (lse = log of the joint denominator)
+ *   doc_scores, score_accum  as in cf_query_prefill_attn: the documents' shares of the mass that falls
+ *                   on the documents (they still sum to 1 per request), so pruning decisions do not
+ *                   depend on whether the caller merges the query-self block here or elsewhere
+ *   workspace       at least cf_attn_workspace_bytes_full(geom, batch, n_layers) bytes */
+size_t cf_attn_workspace_bytes_full(const cf_geom* geom, const cf_batch* batch, int32_t n_layers);
+int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                               int32_t n_layers, const void* q, int64_t q_layer_stride,
+                               const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                               const void* k_self, const void* v_self, int64_t self_layer_stride,
+                               float softmax_scale, void* out, int64_t out_layer_stride,
+                               float* lse, float* doc_scores, float* score_accum,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same computation as cf_query_prefill_attn for callers that cannot allocate device memory
  * (the paper has no counterpart; this is a property of the library, not of the method).
  * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host

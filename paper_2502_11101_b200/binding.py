@@ -23,7 +23,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
-           "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
+           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -84,13 +85,18 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes_layers.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_layers.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64,
                                                  vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.cf_attn_workspace_bytes_full.restype = ctypes.c_size_t
+    lib.cf_attn_workspace_bytes_full.argtypes = [gp, bp, i32]
+    lib.cf_query_prefill_attn_full.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, vp, vp, i64, ctypes.c_float,
+                                               vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_query_prefill_attn_static.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
     lib.cf_profile_end.argtypes = [vp, i32, vp]
     for name in EXPORTS:
-        if name not in ("cf_error_string", "cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers"):
+        if name not in ("cf_error_string", "cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers",
+                        "cf_attn_workspace_bytes_full"):
             getattr(lib, name).restype = ctypes.c_int
     _LIB = lib
     return lib
@@ -231,6 +237,32 @@ def cf_query_prefill_attn_layers(geom: cf_geom, batch: cf_batch, plan: torch.Ten
         _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn_layers")
+
+
+def cf_attn_workspace_bytes_full(geom: cf_geom, batch: cf_batch, n_layers: int) -> int:
+    return int(load_library().cf_attn_workspace_bytes_full(ctypes.byref(geom), ctypes.byref(batch), n_layers))
+
+
+def cf_query_prefill_attn_full(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,
+                               k_cache: torch.Tensor, v_cache: torch.Tensor, k_self: torch.Tensor,
+                               v_self: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor,
+                               lse: Optional[torch.Tensor] = None, doc_scores: Optional[torch.Tensor] = None,
+                               score_accum: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                               stream=None) -> None:
+    """cf_query_prefill_attn_layers plus the causal block of the query tokens over themselves:
+    `k_self`, `v_self` [n_layers, B, Lq, Hkv, D] (dimension 0 may be strided)."""
+    n_layers = q.shape[0]
+    assert k_cache.shape[0] == n_layers and v_cache.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k_self.shape[0] == n_layers and v_self.shape[0] == n_layers
+    assert k_cache.stride(0) == v_cache.stride(0) and k_self.stride(0) == v_self.stride(0)
+    for t in (lse, doc_scores):
+        assert t is None or (t.shape[0] == n_layers and t.is_contiguous())
+    rc = load_library().cf_query_prefill_attn_full(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), n_layers, q.data_ptr(), q.stride(0),
+        k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(0), k_self.data_ptr(), v_self.data_ptr(),
+        k_self.stride(0), softmax_scale, out.data_ptr(), out.stride(0), _ptr(lse), _ptr(doc_scores),
+        _ptr(score_accum), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn_full")
 
 
 def cf_query_prefill_attn_static(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,

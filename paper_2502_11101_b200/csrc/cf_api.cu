@@ -165,7 +165,7 @@ int choose_splits(const cf_geom* g, const cf_batch* b, int n_layers) {
     return 2 * (int)std::max<long long>(s, 1);
 }
 
-size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers,
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers, bool with_self,
                              AttnWorkspace* ws, void* base_ptr) {
     const size_t rows = (size_t)g->n_q_heads * b->q_len;
     const size_t nlb = (size_t)b->n_requests * (size_t)n_layers;
@@ -182,6 +182,12 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
     size_t l = take(nlb * n_splits * rows);
     size_t t = take((size_t)n_layers * max_tiles * rows);
     size_t r = take(nlb * rows);
+    size_t so = 0, sm = 0, sl = 0;
+    if (with_self) {                                  // behind everything else: the rest of the layout does not move
+        so = take(nlb * rows * g->head_dim);
+        sm = take(nlb * rows);
+        sl = take(nlb * rows);
+    }
     if (ws) {
         ws->part_o = reinterpret_cast<float*>(base + o);
         ws->part_m = reinterpret_cast<float*>(base + m);
@@ -193,6 +199,9 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->n_layers = n_layers;
         ws->max_tiles = (int)max_tiles;
         ws->rg_rows = choose_row_group(g, b);
+        ws->self_o = with_self ? reinterpret_cast<float*>(base + so) : nullptr;
+        ws->self_m = with_self ? reinterpret_cast<float*>(base + sm) : nullptr;
+        ws->self_l = with_self ? reinterpret_cast<float*>(base + sl) : nullptr;
     }
     return off;
 }
@@ -214,7 +223,8 @@ static int check_plan(const cf_geom* geom, const cf_batch* batch, const void* pl
 }
 
 int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan, const LayerSpan& span,
-                    const void* q, const void* k_cache, const void* v_cache, float softmax_scale,
+                    const void* q, const void* k_cache, const void* v_cache, const void* k_self,
+                    const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t s) {
     int rc = check_plan(geom, batch, plan);
@@ -236,12 +246,23 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
             (span.out_stride * esize) % 16 || (span.kv_stride * esize) % 16)
             return CF_ERR_INVALID_ARG;
     }
+    const bool with_self = k_self != nullptr || v_self != nullptr;
+    if (with_self) {
+        const long long layer_rows = (long long)batch->n_requests * batch->q_len * geom->n_kv_heads * geom->head_dim;
+        if (!k_self || !v_self || reinterpret_cast<uintptr_t>(k_self) % 16 || reinterpret_cast<uintptr_t>(v_self) % 16 ||
+            (span.n_layers > 1 && self_stride < layer_rows))
+            return CF_ERR_INVALID_ARG;
+    }
     const int n_splits = choose_splits(geom, batch, span.n_layers);
     AttnWorkspace ws;
-    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, &ws, workspace);
+    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, with_self, &ws, workspace);
     if (workspace_bytes < need) return CF_ERR_WORKSPACE;
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    if (with_self) {
+        rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, scale * kLog2e, ws, s);
+        if (rc != CF_OK) return rc;
+    }
     const bool timed = g_prof_used < g_prof_capacity;
     if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
     if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch)) {
@@ -395,7 +416,12 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
 
 size_t cf_attn_workspace_bytes_layers(const cf_geom* geom, const cf_batch* batch, int32_t n_layers) {
     if (!batch || validate(geom, batch) != CF_OK || n_layers <= 0 || n_layers > CF_MAX_LAYERS_PER_CALL) return 0;
-    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, n_layers), n_layers, nullptr, nullptr);
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, n_layers), n_layers, false, nullptr, nullptr);
+}
+
+size_t cf_attn_workspace_bytes_full(const cf_geom* geom, const cf_batch* batch, int32_t n_layers) {
+    if (!batch || validate(geom, batch) != CF_OK || n_layers <= 0 || n_layers > CF_MAX_LAYERS_PER_CALL) return 0;
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, n_layers), n_layers, true, nullptr, nullptr);
 }
 
 size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch) {
@@ -442,8 +468,8 @@ int cf_query_prefill_attn(const cf_geom* geom, const cf_batch* batch, const void
                           float* score_accum, void* workspace, size_t workspace_bytes,
                           void* stream) {
     const LayerSpan span = {1, 0, 0, 0};
-    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
-                           score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, nullptr, nullptr, 0, softmax_scale, out, lse,
+                           doc_scores, score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan,
@@ -454,8 +480,23 @@ int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, con
                                  void* workspace, size_t workspace_bytes, void* stream) {
     if (q_layer_stride < 0 || kv_layer_stride < 0 || out_layer_stride < 0) return CF_ERR_INVALID_ARG;
     const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
-    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
-                           score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, nullptr, nullptr, 0, softmax_scale, out, lse,
+                           doc_scores, score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                               int32_t n_layers, const void* q, int64_t q_layer_stride,
+                               const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                               const void* k_self, const void* v_self, int64_t self_layer_stride,
+                               float softmax_scale, void* out, int64_t out_layer_stride,
+                               float* lse, float* doc_scores, float* score_accum,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    if (q_layer_stride < 0 || kv_layer_stride < 0 || out_layer_stride < 0 || self_layer_stride < 0 || !k_self || !v_self)
+        return CF_ERR_INVALID_ARG;
+    const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, k_self, v_self, self_layer_stride,
+                           softmax_scale, out, lse, doc_scores, score_accum, workspace, workspace_bytes,
+                           static_cast<cudaStream_t>(stream));
 }
 
 int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,

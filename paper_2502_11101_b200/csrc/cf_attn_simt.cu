@@ -250,14 +250,27 @@ combine_kernel(AttnWorkspace ws, int n_requests, long long n_rows_all, long long
                 for (int i = 0; i < V; ++i) acc[i] = fmaf(x[u][i], wp[u], acc[i]);
             }
     }
-    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+    // the documents' share of the row: what the document scores are measured against
+    const float docs_lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
+    float m_all = m_max, l_all = l_sum;
+    if (ws.self_m) {                                                   // the query-self block joins as one more part
+        const size_t srow = (size_t)lb * rows_total + rg;
+        const float ms = ws.self_m[srow], ls = ws.self_l[srow];
+        float xs[V];
+        load_part<V>(ws.self_o + srow * D + lane * V, xs);
+        m_all = fmaxf(m_max, ms);
+        const float wd = l_sum > 0.f ? exp2f(m_max - m_all) : 0.f, wsf = exp2f(ms - m_all);
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = fmaf(xs[i], wsf, acc[i] * wd);
+        l_all = fmaf(ls, wsf, l_sum * wd);
+    }
+    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] *= inv;
     store_row<V>(out + (size_t)layer * out_layer_stride + (((size_t)b * lq + j) * n_q_heads + h) * D + lane * V, acc);
     if (lane == 0) {
-        const float lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
-        ws.row_lse2[(size_t)lb * rows_total + rg] = lse2;
-        if (lse) lse[(size_t)lb * rows_total + rg] = lse2 * kLn2;
+        ws.row_lse2[(size_t)lb * rows_total + rg] = docs_lse2;
+        if (lse) lse[(size_t)lb * rows_total + rg] = (l_all > 0.f ? m_all + log2f(l_all) : -INFINITY) * kLn2;
     }
 }
 

@@ -77,8 +77,12 @@ struct AttnWorkspace {
     int n_layers;
     int max_tiles;     // tile slots per layer in tile_lse2
     int rg_rows;       // query rows per CTA of the tensor-core kernel: 256 (two row tiles) or 128
+    // the query-self block of a call that has one (null otherwise): one more part, always fp32
+    float* self_o;     // [L*B][Hq*Lq][D]
+    float* self_m;     // [L*B][Hq*Lq]
+    float* self_l;     // [L*B][Hq*Lq]
 };
-size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers,
+size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers, bool with_self,
                              AttnWorkspace* ws, void* base);
 
 // Where the layers of a call sit (element strides between consecutive layers).
@@ -103,9 +107,13 @@ bool attn_tc_supported(const cf_geom* g, const cf_batch* b);
 int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
                    const AttnWorkspace& ws, void* out, float* lse, float* doc_scores,
                    float* score_accum, cudaStream_t stream);
-// Shared body of the attention entry points.
+int launch_self_block(const cf_geom* g, const cf_batch* b, const LayerSpan& span, long long self_stride,
+                      const void* q, const void* k_self, const void* v_self, float scale_log2,
+                      const AttnWorkspace& ws, cudaStream_t stream);
+// Shared body of the attention entry points (k_self = v_self = null: cached documents only).
 int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan, const LayerSpan& span,
-                    const void* q, const void* k_cache, const void* v_cache, float softmax_scale,
+                    const void* q, const void* k_cache, const void* v_cache, const void* k_self,
+                    const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t stream);
 

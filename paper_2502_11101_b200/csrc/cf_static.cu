@@ -42,14 +42,14 @@ extern "C" int cf_query_prefill_attn_static(const cf_geom* geom, const cf_batch*
     if (!batch || !plan) return CF_ERR_INVALID_ARG;
     int rc = validate(geom, batch);
     if (rc != CF_OK) return rc;
-    if (attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), 1, nullptr, nullptr) >
+    if (attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), 1, false, nullptr, nullptr) >
         (size_t)CF_STATIC_WORKSPACE_BYTES)
         return CF_ERR_WORKSPACE;            // this batch needs more scratch than the library carries
     void* scratch = nullptr;
     rc = static_scratch_address(&scratch);
     if (rc != CF_OK) return rc;
     const LayerSpan span = {1, 0, 0, 0};
-    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, softmax_scale, out, lse, doc_scores,
-                           score_accum, scratch, (size_t)CF_STATIC_WORKSPACE_BYTES,
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, nullptr, nullptr, 0, softmax_scale, out, lse,
+                           doc_scores, score_accum, scratch, (size_t)CF_STATIC_WORKSPACE_BYTES,
                            static_cast<cudaStream_t>(stream));
 }

@@ -54,10 +54,11 @@ class Session:
             worst = max(worst, int(tiles[:kept_per_request].sum()))
         self.batch.tiles_hint = worst
 
-    def reserve_workspace(self, n_layers: int) -> None:
+    def reserve_workspace(self, n_layers: int, with_self: bool = False) -> None:
         """Grow the attention workspace to what a call over `n_layers` layers needs with the current
         live-document hint (allocation happens here, never inside a library call)."""
-        need = B.cf_attn_workspace_bytes_layers(self.geom, self.batch, n_layers)
+        need = (B.cf_attn_workspace_bytes_full if with_self else B.cf_attn_workspace_bytes_layers)(
+            self.geom, self.batch, n_layers)
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
 
@@ -73,10 +74,16 @@ class Session:
 
     def attend_layers(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                       lse: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
-                      softmax_scale: float = 0.0) -> None:
+                      softmax_scale: float = 0.0, k_self: Optional[torch.Tensor] = None,
+                      v_self: Optional[torch.Tensor] = None) -> None:
         """Consecutive layers that attend the same kept documents, in one library call: q, out
-        [m, B, Lq, Hq, D]; k, v [m, T, Hkv, D]; lse [m, B, Hq, Lq]; layer_scores [m, n_docs_total]."""
-        self.reserve_workspace(q.shape[0])
+        [m, B, Lq, Hq, D]; k, v [m, T, Hkv, D]; lse [m, B, Hq, Lq]; layer_scores [m, n_docs_total].
+        With `k_self`, `v_self` [m, B, Lq, Hkv, D] the causal query-self block is merged in."""
+        self.reserve_workspace(q.shape[0], k_self is not None)
+        if k_self is not None:
+            B.cf_query_prefill_attn_full(self.geom, self.batch, self.plan, q, k, v, k_self, v_self, out, self.workspace,
+                                         lse, layer_scores, self.score_accum, softmax_scale)
+            return
         B.cf_query_prefill_attn_layers(self.geom, self.batch, self.plan, q, k, v, out, self.workspace, lse,
                                        layer_scores, self.score_accum, softmax_scale)
 
@@ -107,12 +114,14 @@ class Session:
     def run_stack(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, schedule: Sequence[Tuple[int, int]],
                   strategy: int, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
                   k_final: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
-                  batch_layers: bool = False) -> None:
+                  batch_layers: bool = False, k_self: Optional[torch.Tensor] = None,
+                  v_self: Optional[torch.Tensor] = None) -> None:
         """Algorithm 2, Phases 1 and 2, as library calls: q, out [L, B, Lq, Hq, D]; k, v [L, T, Hkv, D];
         lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores.
 
         With `batch_layers` the layers between two pruning layers go to the library in one call
-        (possible here because every layer's query states are given up front)."""
+        (possible here because every layer's query states are given up front).  With `k_self`,
+        `v_self` [L, B, Lq, Hkv, D] every layer also attends the query tokens themselves (causal)."""
         sched = dict(schedule)
         n_layers = q.shape[0]
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))
@@ -124,16 +133,24 @@ class Session:
                 for lo in range(first, last, B.CF_MAX_LAYERS_PER_CALL):
                     hi = min(last, lo + B.CF_MAX_LAYERS_PER_CALL)
                     self.attend_layers(q[lo:hi], k[lo:hi], v[lo:hi], out[lo:hi], None if lse is None else lse[lo:hi],
-                                       None if layer_scores is None else layer_scores[lo:hi])
+                                       None if layer_scores is None else layer_scores[lo:hi],
+                                       k_self=None if k_self is None else k_self[lo:hi],
+                                       v_self=None if v_self is None else v_self[lo:hi])
                 if last in sched:
                     self.prune(sched[last], strategy)
                 first = last
         else:
             for layer in range(1, n_layers + 1):
                 i = layer - 1
-                self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
-                if layer_scores is not None:
-                    layer_scores[i].copy_(self.doc_scores)
+                if k_self is None:
+                    self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
+                    if layer_scores is not None:
+                        layer_scores[i].copy_(self.doc_scores)
+                else:
+                    self.attend_layers(q[i:i + 1], k[i:i + 1], v[i:i + 1], out[i:i + 1],
+                                       None if lse is None else lse[i:i + 1],
+                                       None if layer_scores is None else layer_scores[i:i + 1],
+                                       k_self=k_self[i:i + 1], v_self=v_self[i:i + 1])
                 if layer in sched:
                     self.prune(sched[layer], strategy)
         if k_final is not None:

@@ -37,6 +37,8 @@ TENSOR_Q = 1
 TENSOR_K = 2
 TENSOR_V = 3
 TENSOR_META = 4
+TENSOR_K_SELF = 5
+TENSOR_V_SELF = 6
 
 
 def _signed(x: int) -> int:
@@ -239,6 +241,17 @@ def make_kv(meta: WorkloadMeta, device: torch.device | str = "cpu",
     v = torch.empty(shape, dtype=cfg.torch_dtype, device=device)
     for n, layer in enumerate(layers):
         fill_kv_layer(meta, layer, k[n], v[n])
+    return k, v
+
+
+def make_kv_self(meta: WorkloadMeta, device: torch.device | str = "cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """Key and value states of the query tokens themselves, [n_layers, batch, q_len, n_kv_heads,
+    head_dim] in the storage type; like the query states they count as already position-encoded."""
+    cfg = meta.cfg
+    shape = (cfg.n_layers, cfg.batch, cfg.q_len, cfg.n_kv_heads, cfg.head_dim)
+    count = int(np.prod(shape))
+    k = hashed_normal(meta.seed, TENSOR_K_SELF, 0, count, device).view(shape).to(cfg.torch_dtype)
+    v = hashed_normal(meta.seed, TENSOR_V_SELF, 0, count, device).view(shape).to(cfg.torch_dtype)
     return k, v
 
 

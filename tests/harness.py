@@ -71,8 +71,19 @@ def cut_margins(meta: W.WorkloadMeta, ref: List[Dict], strategy: int, schedule=N
     return float(worst)
 
 
+def add_self_block(meta: W.WorkloadMeta, ref: List[Dict], q: torch.Tensor, k_self: torch.Tensor,
+                   v_self: torch.Tensor) -> None:
+    """Replace every layer's output and log-sum-exp of the oracle run by the merge with the causal
+    query-self block (document scores are defined on the documents alone and stay)."""
+    qd, ks, vs = q.double().cpu().numpy(), k_self.double().cpu().numpy(), v_self.double().cpu().numpy()
+    for b in range(meta.cfg.batch):
+        for l, rec in enumerate(ref[b]["layers"]):
+            o_self, lse_self = oracle.query_self_block(qd[l, b], ks[l, b], vs[l, b])
+            rec["out"], rec["lse"] = oracle.merge_softmax_blocks(rec["out"], rec["lse"], o_self, lse_self)
+
+
 def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, device="cuda:0", n_reuse: int = 0,
-              with_final: bool = True, batch_layers: bool = False):
+              with_final: bool = True, batch_layers: bool = False, k_self=None, v_self=None):
     from paper_2502_11101_b200.session import Session
     cfg = meta.cfg
     sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
@@ -85,7 +96,9 @@ def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, devic
     scores = torch.full((n_layers, meta.n_docs_total), float("nan"), device=device)
     k_final = kg.clone() if with_final else None
     sched = cfg.schedule if schedule is None else schedule
-    sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores, batch_layers=batch_layers)
+    sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores, batch_layers=batch_layers,
+                   k_self=None if k_self is None else k_self.to(device),
+                   v_self=None if v_self is None else v_self.to(device))
     torch.cuda.synchronize()
     status = sess.status()
     return {"out": out.float().cpu().numpy(), "lse": lse.cpu().numpy(), "scores": scores.cpu().numpy(),
@@ -156,14 +169,20 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
 
 
 def run_and_compare(cfg: W.WorkloadConfig, seed: int, strategy: int, device="cuda:0", n_reuse: int = 0,
-                    min_margin: float = 2e-3, doc_len_override=None, batch_layers: bool = False) -> Dict[str, float]:
+                    min_margin: float = 2e-3, doc_len_override=None, batch_layers: bool = False,
+                    self_block: bool = False) -> Dict[str, float]:
     meta = W.make_meta(cfg, seed, doc_len_override)
     q = W.make_q(meta)
     k, v = W.make_kv(meta)
     ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse)
     margin = cut_margins(meta, ref, strategy)
     assert margin >= min_margin, f"workload rejected: decisive score gap {margin:.2e} below {min_margin:.0e}"
-    got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse, batch_layers=batch_layers)
+    k_self = v_self = None
+    if self_block:
+        k_self, v_self = W.make_kv_self(meta)
+        add_self_block(meta, ref, q, k_self, v_self)
+    got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse, batch_layers=batch_layers,
+                    k_self=k_self, v_self=v_self)
     report = compare(meta, ref, got, k)
     report["margin"] = margin
     return report

@@ -357,3 +357,27 @@ def test_linear_pruning_schedule_of_the_paper():
     cfg = W.scaled_config(base, schedule=schedule)
     harness.run_and_compare(cfg, _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3), oracle.ALLOC_ALIGN, min_margin=1e-3,
                             batch_layers=True)
+
+
+@pytest.mark.parametrize("which", ["config3", "config2-mha", "config4-reduced", "ragged-f32-d64", "config1-f32"])
+def test_query_self_block_merged_in(which):
+    """cf_query_prefill_attn_full: the causal block of the query tokens over themselves joins the softmax."""
+    if which == "config3":
+        cfg = W.scaled_config(W.CONFIGS[3], n_layers=6, schedule=((2, 25), (4, 12)))
+    elif which == "config2-mha":
+        cfg = W.CONFIGS[2]
+    elif which == "config4-reduced":
+        cfg = W.scaled_config(W.CONFIGS[4], n_layers=3, batch=2, schedule=((2, 50),))
+    elif which == "config1-f32":
+        cfg = W.CONFIGS[1]
+    else:
+        lens = [1, 63, 64, 65, 127, 128, 129, 200, 300, 17, 256, 31]
+        cfg = W.WorkloadConfig("ragged", 3, 8, 2, 64, "f32", 1e4, 4096, len(lens), 1, 300, 5, 1, 2, ((2, 7),))
+        for batch_layers in (False, True):
+            harness.run_and_compare(cfg, 1, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=1e-3,
+                                    batch_layers=batch_layers, self_block=True)
+        return
+    seed = _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3)
+    for batch_layers in (False, True):
+        harness.run_and_compare(cfg, seed, oracle.ALLOC_ALIGN, min_margin=1e-3, batch_layers=batch_layers,
+                                self_block=True)
