@@ -119,7 +119,7 @@ class GpuWorkload:
     """A ring of resident input sets (distinct seeds) so that consecutive steps never find their
     inputs in L2, plus the session and output buffers of the library."""
 
-    def __init__(self, cfg, seed, device, ring, batch_layers=True):
+    def __init__(self, cfg, seed, device, ring, batch_layers=True, self_block=False):
         from paper_2502_11101_b200.session import Session
         self.cfg, self.device = cfg, device
         self.batch_layers = batch_layers
@@ -129,6 +129,7 @@ class GpuWorkload:
                             cfg.rope_theta, cfg.q_len, m.doc_len, m.req_doc_begin, m.doc_src_start,
                             tail_reserve=cfg.q_len, device=device)
         self.slots = []
+        self.self_kv = []
         for r in range(ring):
             # same documents (lengths, relevance), fresh tensor contents per slot
             mr = W.make_meta(cfg, seed + 1000 * r, doc_len_override=m.doc_len) if r else m
@@ -136,6 +137,7 @@ class GpuWorkload:
             q = W.make_q(mr, device)
             k, v = W.make_kv(mr, device)
             self.slots.append((q, k, v))
+            self.self_kv.append(W.make_kv_self(mr, device) if self_block else (None, None))
         q0 = self.slots[0][0]
         self.out = torch.empty_like(q0)
         self.lse = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), device=device)
@@ -143,8 +145,9 @@ class GpuWorkload:
 
     def step(self, slot):
         q, k, v = self.slots[slot % len(self.slots)]
+        k_self, v_self = self.self_kv[slot % len(self.slots)]
         self.sess.run_stack(q, k, v, self.cfg.schedule, STRATEGY_ALIGN, self.out, self.lse, self.k_final,
-                            batch_layers=self.batch_layers)
+                            batch_layers=self.batch_layers, k_self=k_self, v_self=v_self)
 
     def calls(self):
         """(first, last) layer ranges of the attention calls of one step."""
@@ -179,8 +182,10 @@ class GpuWorkload:
 
     def launches_per_step(self):
         cfg = self.cfg
-        # plan init + per attention call (attention, merge, scores) + prune/plan kernels + final re-positioning
-        return 1 + 3 * len(self.calls()) + len(cfg.schedule) + 1
+        # plan init + per attention call (attention, merge, scores; the query-self block if asked for) +
+        # prune/plan kernels + final re-positioning
+        per_call = 4 if self.self_kv[0][0] is not None else 3
+        return 1 + per_call * len(self.calls()) + len(cfg.schedule) + 1
 
 
 def time_steps(fn, steps, warmup, world):
@@ -321,6 +326,8 @@ def main():
     ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
     ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
     ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
+    ap.add_argument("--self-block", action="store_true",
+                    help="variant: every layer also attends the query tokens themselves (cf_query_prefill_attn_full)")
     ap.add_argument("--schedule", default="config", choices=["config", "linear"],
                     help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
                          "a constant number of documents, down to 5)")
@@ -365,7 +372,8 @@ def main():
         cf.cf_set_attn_path(1)
     peaks = load_peaks()
 
-    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer)
+    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
+                     self_block=args.self_block)
     kept, survivors = wl.kept_per_layer()
     per_layer_tokens = token_layers(cfg, wl.meta, kept)
     tokens_per_step = sum(per_layer_tokens)
@@ -466,7 +474,7 @@ def main():
                     "frac": gbs / peaks["hbm_gbs"]}
     traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer",
                    "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05")
-    traffic = None if (args.layers or args.q_len or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
+    traffic = None if (args.layers or args.q_len or args.self_block or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
     roofline.update({"traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write)",
                      "algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()), "kernel": "fused re-position + query-prefill attention",
                      "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
@@ -475,13 +483,14 @@ def main():
 
     # ---- end to end: query and cache store start in pinned host memory every step --------------
     q0, k0, v0 = wl.slots[0]
-    host = [t.cpu().pin_memory() for t in (q0, k0, v0)]
+    resident = [q0, k0, v0] + [t for t in wl.self_kv[0] if t is not None]
+    host = [t.cpu().pin_memory() for t in resident]
     out_h = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
     acc_h = torch.empty(wl.sess.score_accum.shape, dtype=torch.float32).pin_memory()
     kept_h = torch.empty(wl.sess.n_docs_total, dtype=torch.int32).pin_memory()
 
     def e2e_step(_):
-        for src, dst in zip(host, (q0, k0, v0)):
+        for src, dst in zip(host, resident):
             dst.copy_(src, non_blocking=True)
         wl.step(0)
         out_h.copy_(wl.out, non_blocking=True)
@@ -510,7 +519,7 @@ def main():
                  "are inputs of the step)") if wl.batch_layers else "one attention call per layer"
     repo = None
     if world == 1 and not args.skip_reposition:
-        del wl, graphs, host, q0, k0, v0
+        del wl, graphs, host, q0, k0, v0, resident
         torch.cuda.empty_cache()
         repo = reposition_roofline(device, peaks)
 
@@ -533,6 +542,7 @@ def main():
                        "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                        "docs_per_request": cfg.n_docs, "requests": cfg.batch, "q_len": cfg.q_len,
                        "schedule": [list(s) for s in cfg.schedule], "schedule_kind": args.schedule, "strategy": "align",
+                       "query_self_block": bool(args.self_block),
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
                              f"{slot_mb:.0f} MB) cycled between steps",
