@@ -35,10 +35,16 @@ self_block_kernel(AttnWorkspace ws, LayerSpan span, long long self_stride, int n
     k_self += (size_t)layer * self_stride + (size_t)b * lq * n_kv_heads * D;
     v_self += (size_t)layer * self_stride + (size_t)b * lq * n_kv_heads * D;
 
-    for (int idx = tid; idx < lq * D; idx += kSelfThreads) {
-        const int t = idx / D, d = idx - t * D;
-        Ks[(size_t)t * kPitch + d] = k_self[((size_t)t * n_kv_heads + kvh) * D + d];
-        Vs[(size_t)t * D + d] = v_self[((size_t)t * n_kv_heads + kvh) * D + d];
+    // 16-byte loads; the padded key rows are only 4-byte aligned, so they are stored word by word
+    constexpr int kVec = 16 / (int)sizeof(T), kWords = 4;           // elements and 32-bit words per vector
+    for (int idx = tid; idx < lq * (D / kVec); idx += kSelfThreads) {
+        const int t = idx / (D / kVec), c = idx - t * (D / kVec);
+        const size_t src = ((size_t)t * n_kv_heads + kvh) * D + c * kVec;
+        const uint4 kq = *reinterpret_cast<const uint4*>(k_self + src);
+        const uint4 vq = *reinterpret_cast<const uint4*>(v_self + src);
+        uint32_t* kd = reinterpret_cast<uint32_t*>(Ks + (size_t)t * kPitch + c * kVec);
+        kd[0] = kq.x; kd[1] = kq.y; kd[kWords - 2] = kq.z; kd[kWords - 1] = kq.w;
+        *reinterpret_cast<uint4*>(Vs + (size_t)t * D + c * kVec) = vq;
     }
     __syncthreads();
 
@@ -59,10 +65,14 @@ self_block_kernel(AttnWorkspace ws, LayerSpan span, long long self_stride, int n
             const int t = lane + 32 * c;
             s[c] = -INFINITY;
             if (t <= j) {
-                float acc = 0.f;
+                float acc0 = 0.f, acc1 = 0.f;
                 const T* kr = Ks + (size_t)t * kPitch;
-                for (int d = 0; d < D; ++d) acc = fmaf(qrow[d], to_float(kr[d]), acc);
-                s[c] = acc * scale_log2;
+#pragma unroll 8
+                for (int d = 0; d < D; d += 2) {
+                    acc0 = fmaf(qrow[d], to_float(kr[d]), acc0);
+                    acc1 = fmaf(qrow[d + 1], to_float(kr[d + 1]), acc1);
+                }
+                s[c] = (acc0 + acc1) * scale_log2;
             }
             m = fmaxf(m, s[c]);
         }
