@@ -202,6 +202,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->self_o = with_self ? reinterpret_cast<float*>(base + so) : nullptr;
         ws->self_m = with_self ? reinterpret_cast<float*>(base + sm) : nullptr;
         ws->self_l = with_self ? reinterpret_cast<float*>(base + sl) : nullptr;
+        ws->self_mode = 0;
     }
     return off;
 }
@@ -259,15 +260,19 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     if (workspace_bytes < need) return CF_ERR_WORKSPACE;
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
-    if (with_self) {
+    const bool tensor_core = g_attn_path.load() == 0 && attn_tc_supported(geom, batch);
+    if (with_self && batch->q_len > CF_TILE_TOKENS) return CF_ERR_UNSUPPORTED;
+    if (with_self && !tensor_core) {                  // the CUDA-core path computes the block as a part of its own
+        ws.self_mode = 1;
         rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, scale * kLog2e, ws, s);
         if (rc != CF_OK) return rc;
     }
     const bool timed = g_prof_used < g_prof_capacity;
     if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
-    if (g_attn_path.load() == 0 && attn_tc_supported(geom, batch)) {
+    if (tensor_core) {
         ws.part_bf16 = 1;
-        rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
+        ws.self_mode = with_self ? 2 : 0;             // the block rides along as one more key tile
+        rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, k_self, v_self, self_stride, scale * kLog2e, ws, s);
     } else
         rc = launch_attn_simt(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
     if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);

@@ -251,9 +251,20 @@ combine_kernel(AttnWorkspace ws, int n_requests, long long n_rows_all, long long
             }
     }
     // the documents' share of the row: what the document scores are measured against
-    const float docs_lse2 = l_sum > 0.f ? m_max + log2f(l_sum) : -INFINITY;
+    float docs_l = l_sum;
+    if (ws.self_mode == 2) {
+        // the block was the last key tile of one part: that part counts with its sum over documents alone
+        const size_t srow = (size_t)lb * rows_total + rg;
+        const int sp = __float_as_int(ws.self_m[srow]);
+        const float ld = ws.self_l[srow];
+        const float l0 = sp == lane ? ld : l[0], l1 = sp == lane + 32 ? ld : l[1];
+        docs_l = fmaf(l1, w[1], l0 * w[0]);                             // same tree as l_sum, no subtraction
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) docs_l += __shfl_xor_sync(0xffffffffu, docs_l, o);
+    }
+    const float docs_lse2 = docs_l > 0.f ? m_max + log2f(docs_l) : -INFINITY;
     float m_all = m_max, l_all = l_sum;
-    if (ws.self_m) {                                                   // the query-self block joins as one more part
+    if (ws.self_mode == 1) {                                           // the query-self block joins as one more part
         const size_t srow = (size_t)lb * rows_total + rg;
         const float ms = ws.self_m[srow], ls = ws.self_l[srow];
         float xs[V];

@@ -48,6 +48,7 @@ constexpr int kBoxBytes = kBoxRows * 128;
 // two bulk copies (one per 64-column half) whatever its length.
 struct StoreMaps {
     CUtensorMap k[4], v[4];
+    CUtensorMap ks[4], vs[4];      // keys and values of the query tokens themselves (calls with a query-self block)
 };
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
 constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
@@ -80,9 +81,16 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 struct TileInfo {
     int row0, len, doc;
 };
-__device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView& pv, int ti0, int it) {
+// The query-self block, when the CTA has it, is its last tile: document -1, rows of the query's own
+// key/value tensors.
+__device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView& pv, int ti0, int it, int self_it = -1,
+                                              int self_row0 = 0, int self_len = 0) {
     TileInfo t;
-    if (it < kMetaTiles) {
+    if (it == self_it) {
+        t.row0 = self_row0;
+        t.len = self_len;
+        t.doc = -1;
+    } else if (it < kMetaTiles) {
         const int2 m = s_meta[it];
         t.row0 = m.x;
         t.len = m.y & 0xff;
@@ -278,7 +286,7 @@ template <int LAYOUT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
-               float scale_log2, const __nv_bfloat16* __restrict__ q) {
+               float scale_log2, const __nv_bfloat16* __restrict__ q, int with_self) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -316,7 +324,11 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     const int n_pairs = n_parts >> 1;
     const int t_begin = (int)((long long)n_tiles * pair / n_pairs);
     const int t_end = (int)((long long)n_tiles * (pair + 1) / n_pairs);
-    const int n_it = t_end - t_begin;                               // key tiles of this CTA
+    // the CTA of the last pair of parts also takes the query-self block, as one more tile after its documents'
+    const bool has_self = with_self && pair == n_pairs - 1;
+    const int n_it = t_end - t_begin + (has_self ? 1 : 0);          // key tiles of this CTA
+    const int self_it = has_self ? n_it - 1 : -1;
+    const int self_row0 = b * lq;
     // first workspace row of this CTA in part 2*pair
     const size_t slot0 = ((size_t)lb * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * rg_rows;
 
@@ -327,7 +339,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     }
     if (n_it <= 0) return;
     const int ti0 = tbase + t_begin;                                // first tile of this CTA in the plan's list
-    if (tid < min(n_it, kMetaTiles)) {
+    if (tid < min(n_it, kMetaTiles) && tid != self_it) {
         const int len = pv.tile_len[ti0 + tid], doc = pv.tile_doc[ti0 + tid];
         s_meta[tid] = make_int2(pv.tile_row0[ti0 + tid], (len & 0xff) | (doc << 8));   // len 1..128 -> 0x80 at most
     }
@@ -373,10 +385,11 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     int produced = 0;
     auto produce = [&](int u) {                                     // u-th ring use: K(u/2) if even, V(u/2) if odd
         const int st = ring_mod(u, alternate);
-        const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1);
+        const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1, self_it, self_row0, lq);
         const int row0 = tile.row0;
         const int boxes = (tile.len + kBoxRows - 1) / kBoxRows;
-        const CUtensorMap* map = (u & 1) ? &maps.v[boxes - 1] : &maps.k[boxes - 1];
+        const CUtensorMap* map = tile.doc < 0 ? ((u & 1) ? &maps.vs[boxes - 1] : &maps.ks[boxes - 1])
+                                              : ((u & 1) ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
         const uint32_t bar = smem_u32(&bars->kv_full[st][u & 1]);
         const uint32_t dst = ring_base + st * kTileBytes;
         mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
@@ -428,7 +441,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             auto issue_s = [&](int n) -> bool {
                 const int w = n & 1;
                 const int it = alternate ? n : (n >> 1);
-                const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
+                const int n_keys = (tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len + 15) & ~15;
                 const int stk = ring_mod(2 * it, alternate);
                 const int kuse = ring_uses(it, alternate);
                 if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
@@ -448,7 +461,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             auto issue_pv = [&](int n) -> bool {
                 const int w = n & 1, j = n >> 1;
                 const int it = alternate ? n : j;
-                const int n_keys = (tile_info(s_meta, pv, ti0, it).len + 15) & ~15;
+                const int n_keys = (tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len + 15) & ~15;
                 const int stv = ring_mod(2 * it + 1, alternate);
                 const int vuse = ring_uses(it, alternate);                  // value loads this stage has seen
                 if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
@@ -477,12 +490,15 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
         const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
         const int chunk = t & 7, rsub = t >> 3;
         for (int it = 0; it < n_it; ++it) {
-            const TileInfo tile = tile_info(s_meta, pv, ti0, it);
+            const TileInfo tile = tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq);
             const int len = tile.len;
-            const float2* trig = pv.trig + (size_t)tile.doc * (kD / 2);
+            const float2* trig = pv.trig + (size_t)max(tile.doc, 0) * (kD / 2);
             const int st = ring_mod(2 * it, alternate);
             float2 cs[8];
-            if (LAYOUT == CF_ROPE_HALF) {
+            if (tile.doc < 0) {                                     // the query's own keys are already in place
+#pragma unroll
+                for (int e = 0; e < 8; ++e) cs[e] = make_float2(1.f, 0.f);
+            } else if (LAYOUT == CF_ROPE_HALF) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) cs[e] = __ldg(trig + chunk * 8 + e);
             } else {
@@ -545,12 +561,16 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             const bool row_valid = row_in_group < rows_here;
             const size_t tile_row = (size_t)kvh * rows + rg * rg_rows + row_in_group;
             float* tile_lse2 = ws.tile_lse2 + (size_t)layer * ws.max_tiles * rows_total;
-            float m_ref = -INFINITY, l_run = 0.f;
+            float m_ref = -INFINITY, l_run = 0.f, l_docs = 0.f;
+            const int q_index = (rg * rg_rows + row_in_group) % lq;     // position of this row's token in the query
             bool ok = true;
             for (int j = 0; j < n_items; ++j) {
                 const int it = alternate ? 2 * j + w : j;
                 const int ti = ti0 + it;
-                const int len = tile_info(s_meta, pv, ti0, it).len;
+                const int len = tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len;
+                // keys this row may see: the whole tile of a document, the query tokens 0..q_index of the
+                // query-self block (causal mask, footnote to Eq. 1)
+                const int vis = it == self_it ? min(len, q_index + 1) : len;
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -608,22 +628,26 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 tmem_ld32_async(s_addr, va);
                 tmem_ld_wait(va);
                 for (int c = 0; c < n_chunks; c += 2) {
-                    prepare(va, len - c * 32, c);
+                    prepare(va, vis - c * 32, c);
                     if (c + 1 < n_chunks) tmem_ld32_async(s_addr + (c + 1) * 32, vb);
-                    finish(va, len - c * 32, c);
+                    finish(va, vis - c * 32, c);
                     if (c + 1 < n_chunks) {
                         tmem_ld_wait(vb);
-                        prepare(vb, len - c * 32 - 32, c + 1);
+                        prepare(vb, vis - c * 32 - 32, c + 1);
                         if (c + 2 < n_chunks) tmem_ld32_async(s_addr + (c + 2) * 32, va);
-                        finish(vb, len - c * 32 - 32, c + 1);
+                        finish(vb, vis - c * 32 - 32, c + 1);
                         if (c + 2 < n_chunks) tmem_ld_wait(va);
                     }
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars->p_ready[w]));
+                if (it == self_it) {
+                    l_docs = l_run;                                 // the documents' share of this part's sum (the block is the last tile)
+                } else if (row_valid) {
+                    tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
+                }
                 l_run += tile_sum;
-                if (row_valid) tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
             }
             if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (n_items - 1) & 1, abort_flag);
             if (ok) {
@@ -666,6 +690,12 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (row_valid) {
                     ws.part_m[slot] = m_ref;
                     ws.part_l[slot] = l_run;
+                    if (has_self && (alternate ? 2 * (n_items - 1) + w : n_items - 1) == self_it) {
+                        // which part of this row holds the block, and that part's sum over documents alone
+                        const size_t srow = (size_t)lb * rows_total + tile_row;
+                        ws.self_m[srow] = __int_as_float(2 * pair + (alternate ? w : 0));
+                        ws.self_l[srow] = l_docs;
+                    }
                 }
             }
         }
@@ -729,6 +759,25 @@ int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const c
     return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
 }
 
+// Keys or values of the query tokens, [layers][requests][q_len][kv heads][head_dim], as a 4-D tensor
+// (head_dim, kv heads, requests * q_len rows, layers).
+int make_self_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span,
+                  long long self_stride, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return CF_ERR_CUDA;
+    const cuuint64_t rows = (cuuint64_t)b->n_requests * (cuuint64_t)b->q_len;
+    const cuuint64_t row_bytes = (cuuint64_t)g->n_kv_heads * kD * 2;
+    const cuuint64_t layer_bytes = span.n_layers > 1 ? (cuuint64_t)self_stride * 2 : rows * row_bytes;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, rows, (cuuint64_t)span.n_layers};
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, row_bytes, layer_bytes};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
+}
+
 }  // namespace
 
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
@@ -736,7 +785,8 @@ bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
 }
 
 int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span, const void* q,
-                   const void* k, const void* v, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
+                   const void* k, const void* v, const void* k_self, const void* v_self, long long self_stride,
+                   float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_groups = (rows + ws.rg_rows - 1) / ws.rg_rows;
     if ((long long)g->n_kv_heads * row_groups > 65535 || (long long)b->n_requests * span.n_layers > 65535 ||
@@ -748,7 +798,17 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
         if (rc != CF_OK) return rc;
         rc = make_store_map(&maps.v[i], v, g, b, span, (i + 1) * kBoxRows);
         if (rc != CF_OK) return rc;
+        if (k_self) {
+            rc = make_self_map(&maps.ks[i], k_self, g, b, span, self_stride, (i + 1) * kBoxRows);
+            if (rc != CF_OK) return rc;
+            rc = make_self_map(&maps.vs[i], v_self, g, b, span, self_stride, (i + 1) * kBoxRows);
+            if (rc != CF_OK) return rc;
+        } else {
+            maps.ks[i] = maps.k[i];
+            maps.vs[i] = maps.v[i];
+        }
     }
+    if (k_self && b->q_len > kTile) return CF_ERR_UNSUPPORTED;   // the query-self block is one key tile
     dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
               (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
@@ -760,7 +820,8 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
             configured[which] = true;
         }
         kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, bv, pv, ws, span.q_stride, g->n_q_heads,
-                                                       g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q));
+                                                       g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q),
+                                                       k_self ? 1 : 0);
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
     if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);

@@ -77,10 +77,14 @@ struct AttnWorkspace {
     int n_layers;
     int max_tiles;     // tile slots per layer in tile_lse2
     int rg_rows;       // query rows per CTA of the tensor-core kernel: 256 (two row tiles) or 128
-    // the query-self block of a call that has one (null otherwise): one more part, always fp32
+    // The query-self block of a call that has one.  self_mode 1 (CUDA-core path): it is one more part,
+    // (self_m, self_l, self_o) like (part_m, part_l, part_o) in fp32.  self_mode 2 (tensor-core path):
+    // it is the last key tile of one of the parts; self_m holds that part's index (an int) and self_l
+    // the part's sum over the documents alone.  self_mode 0: none.
     float* self_o;     // [L*B][Hq*Lq][D]
     float* self_m;     // [L*B][Hq*Lq]
     float* self_l;     // [L*B][Hq*Lq]
+    int self_mode;
 };
 size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers, bool with_self,
                              AttnWorkspace* ws, void* base);
@@ -101,8 +105,8 @@ int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, co
                      const void* q, const void* k, const void* v, float scale_log2,
                      const AttnWorkspace& ws, cudaStream_t stream);
 int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
-                   const void* q, const void* k, const void* v, float scale_log2,
-                   const AttnWorkspace& ws, cudaStream_t stream);
+                   const void* q, const void* k, const void* v, const void* k_self, const void* v_self,
+                   long long self_stride, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream);
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b);
 int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
                    const AttnWorkspace& ws, void* out, float* lse, float* doc_scores,
