@@ -251,7 +251,7 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     if (with_self) {
         const long long layer_rows = (long long)batch->n_requests * batch->q_len * geom->n_kv_heads * geom->head_dim;
         if (!k_self || !v_self || reinterpret_cast<uintptr_t>(k_self) % 16 || reinterpret_cast<uintptr_t>(v_self) % 16 ||
-            (span.n_layers > 1 && self_stride < layer_rows))
+            (span.n_layers > 1 && (self_stride < layer_rows || (self_stride * esize) % 16)))
             return CF_ERR_INVALID_ARG;
     }
     const int n_splits = choose_splits(geom, batch, span.n_layers);

@@ -14,6 +14,13 @@ constexpr int kSelfThreads = 256;
 constexpr int kSelfRows = 32;          // query rows per block: four per warp
 constexpr int kSelfMaxLq = 128;
 
+// Bytes of the padded key rows in shared memory, rounded up so that the value rows behind them can be
+// written with 16-byte stores.
+template <typename T, int D>
+__host__ __device__ constexpr size_t self_keys_bytes(int lq) {
+    return ((size_t)lq * (D + 2) * sizeof(T) + 15) / 16 * 16;
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kSelfThreads)
 self_block_kernel(AttnWorkspace ws, LayerSpan span, long long self_stride, int n_requests, int n_q_heads,
@@ -22,7 +29,7 @@ self_block_kernel(AttnWorkspace ws, LayerSpan span, long long self_stride, int n
     extern __shared__ __align__(16) unsigned char self_smem[];
     constexpr int kPitch = D + 2;                                   // odd number of 32-bit words per key row: no bank conflicts
     T* Ks = reinterpret_cast<T*>(self_smem);                        // [lq][kPitch]
-    T* Vs = Ks + (size_t)lq * kPitch;                               // [lq][D]
+    T* Vs = reinterpret_cast<T*>(self_smem + self_keys_bytes<T, D>(lq));   // [lq][D], 16-byte aligned
     float* Qs = reinterpret_cast<float*>(Vs + (size_t)lq * D);      // [warps][D]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int group = n_q_heads / n_kv_heads;
@@ -117,12 +124,13 @@ int launch_self_typed(const cf_geom* g, const cf_batch* b, const LayerSpan& span
                       const void* q, const void* k_self, const void* v_self, float scale_log2,
                       const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
-    const size_t smem = (size_t)b->q_len * (D + 2) * sizeof(T) + (size_t)b->q_len * D * sizeof(T) +
+    const size_t smem = self_keys_bytes<T, D>(b->q_len) + (size_t)b->q_len * D * sizeof(T) +
                         (size_t)(kSelfThreads / 32) * D * sizeof(float);
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(self_block_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)((size_t)kSelfMaxLq * (2 * D + 2) * sizeof(T) + (kSelfThreads / 32) * D * sizeof(float))) != cudaSuccess)
+                                 (int)(self_keys_bytes<T, D>(kSelfMaxLq) + (size_t)kSelfMaxLq * D * sizeof(T) +
+                                       (kSelfThreads / 32) * D * sizeof(float))) != cudaSuccess)
             return CF_ERR_CUDA;
         configured = true;
     }
