@@ -123,6 +123,7 @@ class GpuWorkload:
         from paper_2502_11101_b200.session import Session
         self.cfg, self.device = cfg, device
         self.batch_layers = batch_layers
+        self.self_kernel = False            # set by main(): the query-self block runs as a kernel of its own
         self.meta = W.make_meta(cfg, seed)
         m = self.meta
         self.sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range,
@@ -184,7 +185,8 @@ class GpuWorkload:
         cfg = self.cfg
         # plan init + per attention call (attention, merge, scores; the query-self block if asked for) +
         # prune/plan kernels + final re-positioning
-        per_call = 4 if self.self_kv[0][0] is not None else 3
+        # (on the tensor-core path the block is a key tile of the attention kernel, not a launch)
+        per_call = 4 if self.self_kernel else 3
         return 1 + per_call * len(self.calls()) + len(cfg.schedule) + 1
 
 
@@ -374,6 +376,7 @@ def main():
 
     wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
                      self_block=args.self_block)
+    wl.self_kernel = args.self_block and (args.force_simt or not _tc_used(cf, wl))
     kept, survivors = wl.kept_per_layer()
     per_layer_tokens = token_layers(cfg, wl.meta, kept)
     tokens_per_step = sum(per_layer_tokens)
