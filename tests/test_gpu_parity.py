@@ -381,3 +381,26 @@ def test_query_self_block_merged_in(which):
     for batch_layers in (False, True):
         harness.run_and_compare(cfg, seed, oracle.ALLOC_ALIGN, min_margin=1e-3, batch_layers=batch_layers,
                                 self_block=True)
+
+
+def test_query_self_block_argument_errors():
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[2], n_docs=4, n_planted=1, q_len=130)      # more query tokens than one key tile
+    meta = W.make_meta(cfg, 0)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+    q, (k, v), (ks, vs) = W.make_q(meta).cuda(), [t.cuda() for t in W.make_kv(meta)], [t.cuda() for t in W.make_kv_self(meta)]
+    out = torch.empty_like(q)
+    sess.init()
+    for path in (0, 1):
+        cf.cf_set_attn_path(path)
+        try:
+            with pytest.raises(cf.CacheFocusError) as e:
+                sess.attend_layers(q, k, v, out, k_self=ks, v_self=vs)
+            assert e.value.code == cf.CF_ERR_UNSUPPORTED
+        finally:
+            cf.cf_set_attn_path(0)
+    sess.attend_layers(q, k, v, out)                                            # without the block the batch is fine
+    torch.cuda.synchronize()
+    assert sess.status() == 0
