@@ -34,8 +34,8 @@ from paper_2502_11101_b200 import workloads as W  # noqa: E402
 METRIC = "cached KV tokens/s through reposition+query-prefill attn"
 # DRAM bytes (read + write) of one attention-kernel launch, averaged over the four launches of a step of
 # workload 3 in the default configuration, from the ncu capture summarised in
-# profiles/attn_tc_kernel_workload3.md (102.7 MB per step).  Only valid for that kernel state and workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {("configs[2]", "layer-batched", "tcgen05"): 25.68e6}
+# profiles/attn_tc_kernel_workload3.md (102.8 MB per step).  Only valid for that kernel state and workload.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {("configs[2]", "layer-batched", "tcgen05"): 25.70e6}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 
