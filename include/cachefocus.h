@@ -175,6 +175,21 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
                        int32_t n_layers, int64_t layer_stride, const void* k_in, void* k_out,
                        void* stream);
 
+/* Algorithm 2, Phase 2, assembled (C_final): for every layer and request, the re-positioned keys
+ * (Eq. 5) and the values of the surviving documents, packed in rank order (rank 0 first), followed by
+ * the query tokens' own keys and values (C_Q^l, unchanged).
+ *   k_cache, v_cache  the store, n_layers layers, layer_stride elements apart (as cf_reposition_keys)
+ *   k_self, v_self    [n_layers][n_requests][q_len][n_kv_heads][head_dim], self_layer_stride apart
+ *   k_out, v_out      device [n_layers][n_requests][out_rows][n_kv_heads][head_dim], dense; request b
+ *                     receives final_rows[b] rows per layer, rows beyond stay untouched
+ *   final_rows        device int32 [n_requests]: tokens of the survivors + q_len
+ * A request whose rows do not fit out_rows is not written and CF_ERR_WORKSPACE is recorded in the
+ * plan's status word. */
+int cf_assemble_final_cache(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                            int32_t n_layers, int64_t layer_stride, const void* k_cache, const void* v_cache,
+                            int64_t self_layer_stride, const void* k_self, const void* v_self,
+                            int32_t out_rows, void* k_out, void* v_out, int32_t* final_rows, void* stream);
+
 /* Scratch needed by cf_query_prefill_attn for this batch (bytes; 256-byte aligned buffer).
  * Grows with batch->tiles_hint: ask with the largest hint that will be used. */
 size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch);

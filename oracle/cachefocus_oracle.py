@@ -245,6 +245,22 @@ def merge_softmax_blocks(out_a: np.ndarray, lse_a: np.ndarray, out_b: np.ndarray
     return wa * out_a + wb * out_b, lse
 
 
+def assemble_final_cache(k_rot: np.ndarray, v_store: np.ndarray, doc_offsets: Sequence[int],
+                         order: Sequence[int], k_self: np.ndarray, v_self: np.ndarray, doc_base: int = 0
+                         ) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 2, Phase 2 for one layer of one request: the re-positioned keys and the values of the
+    surviving documents in rank order, then the query tokens' own keys and values (C_Q, unchanged).
+    k_rot, v_store[T, Hkv, D]; k_self, v_self[Lq, Hkv, D].  Returns (K_final, V_final)."""
+    ks, vs = [], []
+    for i in order:
+        lo, hi = int(doc_offsets[doc_base + i]), int(doc_offsets[doc_base + i + 1])
+        ks.append(np.asarray(k_rot, dtype=np.float64)[lo:hi])
+        vs.append(np.asarray(v_store, dtype=np.float64)[lo:hi])
+    ks.append(np.asarray(k_self, dtype=np.float64))
+    vs.append(np.asarray(v_self, dtype=np.float64))
+    return np.concatenate(ks), np.concatenate(vs)
+
+
 def prune_topk(score_accum: Sequence[float], order: Sequence[int], keep: int, strategy: int
                ) -> List[int]:
     """Algorithm 2, pruning step: among the documents in `order` keep the `keep` with the

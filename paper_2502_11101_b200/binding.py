@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
-           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -85,6 +85,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes_layers.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_layers.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64,
                                                  vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.cf_assemble_final_cache.argtypes = [gp, bp, vp, i32, i64, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cf_attn_workspace_bytes_full.restype = ctypes.c_size_t
     lib.cf_attn_workspace_bytes_full.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_full.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, vp, vp, i64, ctypes.c_float,
@@ -237,6 +238,20 @@ def cf_query_prefill_attn_layers(geom: cf_geom, batch: cf_batch, plan: torch.Ten
         _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn_layers")
+
+
+def cf_assemble_final_cache(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, k_cache: torch.Tensor,
+                            v_cache: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor, k_out: torch.Tensor,
+                            v_out: torch.Tensor, final_rows: torch.Tensor, stream=None) -> None:
+    """k_cache, v_cache [L, T, Hkv, D]; k_self, v_self [L, B, Lq, Hkv, D]; k_out, v_out [L, B, out_rows, Hkv, D]
+    (contiguous); final_rows int32 [B]."""
+    assert k_out.is_contiguous() and v_out.is_contiguous() and k_out.shape == v_out.shape
+    assert final_rows.dtype == torch.int32 and k_cache.stride(0) == v_cache.stride(0)
+    rc = load_library().cf_assemble_final_cache(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), k_cache.shape[0], k_cache.stride(0),
+        k_cache.data_ptr(), v_cache.data_ptr(), k_self.stride(0), k_self.data_ptr(), v_self.data_ptr(),
+        k_out.shape[2], k_out.data_ptr(), v_out.data_ptr(), final_rows.data_ptr(), _stream(stream))
+    _check(rc, "cf_assemble_final_cache")
 
 
 def cf_attn_workspace_bytes_full(geom: cf_geom, batch: cf_batch, n_layers: int) -> int:

@@ -419,6 +419,28 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
                              static_cast<cudaStream_t>(stream));
 }
 
+int cf_assemble_final_cache(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                            int32_t n_layers, int64_t layer_stride, const void* k_cache, const void* v_cache,
+                            int64_t self_layer_stride, const void* k_self, const void* v_self,
+                            int32_t out_rows, void* k_out, void* v_out, int32_t* final_rows, void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (!k_cache || !v_cache || !k_self || !v_self || !k_out || !v_out || !final_rows || n_layers <= 0 ||
+        out_rows <= 0)
+        return CF_ERR_INVALID_ARG;
+    const int esize = geom->dtype == CF_BF16 ? 2 : 4;
+    const void* ptrs[6] = {k_cache, v_cache, k_self, v_self, k_out, v_out};
+    for (const void* p : ptrs)
+        if (reinterpret_cast<uintptr_t>(p) % 16) return CF_ERR_INVALID_ARG;
+    if ((layer_stride * esize) % 16 || (self_layer_stride * esize) % 16) return CF_ERR_INVALID_ARG;
+    if (n_layers > 1 && (layer_stride < batch->total_tokens * batch->token_stride ||
+                         self_layer_stride < (int64_t)batch->n_requests * batch->q_len * geom->n_kv_heads * geom->head_dim))
+        return CF_ERR_INVALID_ARG;
+    PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
+    return launch_assemble(geom, batch, pv, n_layers, layer_stride, self_layer_stride, out_rows, k_cache, v_cache,
+                           k_self, v_self, k_out, v_out, final_rows, static_cast<cudaStream_t>(stream));
+}
+
 size_t cf_attn_workspace_bytes_layers(const cf_geom* geom, const cf_batch* batch, int32_t n_layers) {
     if (!batch || validate(geom, batch) != CF_OK || n_layers <= 0 || n_layers > CF_MAX_LAYERS_PER_CALL) return 0;
     return attn_workspace_layout(geom, batch, choose_splits(geom, batch, n_layers), n_layers, false, nullptr, nullptr);

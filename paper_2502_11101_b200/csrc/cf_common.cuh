@@ -101,6 +101,9 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream);
 int launch_reposition(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers,
                       long long layer_stride, const void* k_in, void* k_out, cudaStream_t stream);
+int launch_assemble(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers, long long layer_stride,
+                    long long self_stride, int out_rows, const void* k_in, const void* v_in, const void* k_self,
+                    const void* v_self, void* k_out, void* v_out, int* final_rows, cudaStream_t stream);
 int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
                      const void* q, const void* k, const void* v, float scale_log2,
                      const AttnWorkspace& ws, cudaStream_t stream);

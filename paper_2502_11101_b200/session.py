@@ -94,6 +94,11 @@ class Session:
     def reposition(self, k_in: torch.Tensor, k_out: torch.Tensor, n_layers: int = 1, layer_stride: int = 0) -> None:
         B.cf_reposition_keys(self.geom, self.batch, self.plan, k_in, k_out, n_layers, layer_stride)
 
+    def assemble(self, k: torch.Tensor, v: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor,
+                 k_out: torch.Tensor, v_out: torch.Tensor, final_rows: torch.Tensor) -> None:
+        """Phase 2 with the final caches packed per request: survivors in rank order, then the query rows."""
+        B.cf_assemble_final_cache(self.geom, self.batch, self.plan, k, v, k_self, v_self, k_out, v_out, final_rows)
+
     def status(self) -> int:
         return B.cf_plan_status(self.geom, self.batch, self.plan)
 

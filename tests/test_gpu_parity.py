@@ -404,3 +404,52 @@ def test_query_self_block_argument_errors():
     sess.attend_layers(q, k, v, out)                                            # without the block the batch is fine
     torch.cuda.synchronize()
     assert sess.status() == 0
+
+
+@pytest.mark.parametrize("dtype,head_dim", [("bf16", 128), ("f32", 64)])
+def test_assembled_final_cache(dtype, head_dim):
+    """cf_assemble_final_cache: survivors' re-positioned keys and values in rank order, then the query rows."""
+    from paper_2502_11101_b200.session import Session
+    cfg = W.WorkloadConfig("assemble", 3, 8, 2, head_dim, dtype, 1e4, 4096, 9, 20, 150, 6, 2, 2, ((1, 5), (2, 3)))
+    seed = _pick_seed(cfg, oracle.ALLOC_SORT, 1e-3)
+    meta = W.make_meta(cfg, seed)
+    q = W.make_q(meta)
+    k, v = W.make_kv(meta)
+    k_self, v_self = W.make_kv_self(meta)
+    ref = harness.oracle_stack(meta, q, k, v, oracle.ALLOC_SORT)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta, cfg.q_len,
+                   meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+    qg, kg, vg, ksg, vsg = [t.cuda() for t in (q, k, v, k_self, v_self)]
+    out = torch.empty_like(qg)
+    sess.run_stack(qg, kg, vg, cfg.schedule, oracle.ALLOC_SORT, out)
+    out_rows = 3 * 150 + cfg.q_len + 7
+    sentinel = 12345.0
+    k_out = torch.full((cfg.n_layers, cfg.batch, out_rows, cfg.n_kv_heads, head_dim), sentinel, dtype=cfg.torch_dtype, device="cuda")
+    v_out = torch.full_like(k_out, sentinel)
+    final_rows = torch.full((cfg.batch,), -1, dtype=torch.int32, device="cuda")
+    sess.assemble(kg, vg, ksg, vsg, k_out, v_out, final_rows)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    kf_got, vf_got = k_out.float().cpu().numpy(), v_out.float().cpu().numpy()
+    for b in range(cfg.batch):
+        lo = int(meta.req_doc_begin[b])
+        order = ref[b]["order"]
+        assert sess.read_plan()["order"][b] == order
+        for l in range(cfg.n_layers):
+            kf, vf = oracle.assemble_final_cache(ref[b]["k_final"][l], v[l].double().numpy(), meta.doc_offsets, order,
+                                                 k_self[l, b].double().numpy(), v_self[l, b].double().numpy(), doc_base=lo)
+            n = kf.shape[0]
+            assert int(final_rows[b]) == n
+            n_docs_rows = n - cfg.q_len
+            err = np.abs(kf_got[l, b, :n_docs_rows] - kf[:n_docs_rows]) / harness.rotated_key_tolerance(kf[:n_docs_rows], dtype)
+            assert err.max() <= 1.0
+            assert np.array_equal(kf_got[l, b, n_docs_rows:n], kf[n_docs_rows:])          # the query rows are copies
+            assert np.array_equal(vf_got[l, b, :n], vf)                                   # values are copies
+            assert np.all(kf_got[l, b, n:] == sentinel) and np.all(vf_got[l, b, n:] == sentinel)
+    # a buffer that is too small is reported, not overrun
+    small_k = torch.full((cfg.n_layers, cfg.batch, 10, cfg.n_kv_heads, head_dim), sentinel, dtype=cfg.torch_dtype, device="cuda")
+    small_v = torch.full_like(small_k, sentinel)
+    sess.assemble(kg, vg, ksg, vsg, small_k, small_v, final_rows)
+    torch.cuda.synchronize()
+    import paper_2502_11101_b200 as cf
+    assert sess.status() == cf.CF_ERR_WORKSPACE

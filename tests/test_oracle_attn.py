@@ -280,3 +280,26 @@ def test_merge_of_two_halves_is_attention_over_the_whole():
     b = oracle.query_prefill_attn(q, k[4:], v[4:], [0, 6], [0], 1)
     out, lse = oracle.merge_softmax_blocks(a[0], a[1], b[0], b[1])
     assert np.allclose(out, whole[0], atol=1e-13) and np.allclose(lse, whole[1], atol=1e-13)
+
+
+def test_assembled_final_cache_holds_the_pieces_in_order():
+    rng = np.random.default_rng(7)
+    hkv, d, lq = 2, 8, 3
+    doc_len = [4, 2, 5]
+    offsets = np.concatenate([[0], np.cumsum(doc_len)])
+    k_rot = rng.standard_normal((11, hkv, d))
+    v = rng.standard_normal((11, hkv, d))
+    k_self = rng.standard_normal((lq, hkv, d))
+    v_self = rng.standard_normal((lq, hkv, d))
+    order = [2, 0]                                                   # document 1 was pruned
+    kf, vf = oracle.assemble_final_cache(k_rot, v, offsets, order, k_self, v_self)
+    assert kf.shape == (5 + 4 + lq, hkv, d)
+    assert np.array_equal(kf[:5], k_rot[6:11]) and np.array_equal(kf[5:9], k_rot[0:4]) and np.array_equal(kf[9:], k_self)
+    assert np.array_equal(vf[:5], v[6:11]) and np.array_equal(vf[5:9], v[0:4]) and np.array_equal(vf[9:], v_self)
+    # a later token attending the assembled cache = the survivors' caches and the query block, merged
+    q_new = rng.standard_normal((1, 4, d))
+    whole = oracle.query_prefill_attn(q_new, kf, vf, [0, kf.shape[0]], [0], 1)
+    docs = oracle.query_prefill_attn(q_new, k_rot, v, offsets, order, 3)
+    tail = oracle.query_prefill_attn(q_new, k_self, v_self, [0, lq], [0], 1)
+    out, lse = oracle.merge_softmax_blocks(docs[0], docs[1], tail[0], tail[1])
+    assert np.allclose(out, whole[0], atol=1e-13) and np.allclose(lse, whole[1], atol=1e-13)
