@@ -423,7 +423,7 @@ def test_assembled_final_cache(dtype, head_dim):
     out = torch.empty_like(qg)
     sess.run_stack(qg, kg, vg, cfg.schedule, oracle.ALLOC_SORT, out)
     out_rows = 3 * 150 + cfg.q_len + 7
-    sentinel = 12345.0
+    sentinel = 12288.0                                               # exact in bf16
     k_out = torch.full((cfg.n_layers, cfg.batch, out_rows, cfg.n_kv_heads, head_dim), sentinel, dtype=cfg.torch_dtype, device="cuda")
     v_out = torch.full_like(k_out, sentinel)
     final_rows = torch.full((cfg.batch,), -1, dtype=torch.int32, device="cuda")
