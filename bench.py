@@ -247,6 +247,43 @@ def reposition_roofline(device, peaks, layers=8, iters=5):
             "peak_source": peaks["source"]}
 
 
+def assemble_roofline(device, peaks, layers=2, iters=5):
+    """cf_assemble_final_cache (Phase 2 with the final caches packed per request) over a store shaped
+    like the largest configuration, every document kept: K and V are read once and written once."""
+    from paper_2502_11101_b200.session import Session
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=layers)
+    meta = W.make_meta(cfg, 0)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len,
+                   device=device)
+    k, v = W.make_kv(meta, device)
+    k_self, v_self = W.make_kv_self(meta, device)
+    out_rows = int(max(meta.doc_offsets[meta.req_doc_begin[b + 1]] - meta.doc_offsets[meta.req_doc_begin[b]]
+                       for b in range(cfg.batch))) + cfg.q_len
+    k_out = torch.empty((layers, cfg.batch, out_rows, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device=device)
+    v_out = torch.empty_like(k_out)
+    final_rows = torch.zeros(cfg.batch, dtype=torch.int32, device=device)
+    sess.set_live_docs(cfg.n_docs)
+    sess.init()
+    for _ in range(2):
+        sess.assemble(k, v, k_self, v_self, k_out, v_out, final_rows)
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(iters):
+        sess.assemble(k, v, k_self, v_self, k_out, v_out, final_rows)
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / iters
+    assert sess.status() == 0
+    moved = int(final_rows.sum().item()) * layers * cfg.n_kv_heads * cfg.head_dim * 2      # rows x row bytes
+    nbytes = 4 * moved                                                                    # K and V, read and written
+    gbs = nbytes / ms / 1e6
+    return {"kernel": "cf_assemble_final_cache", "workload": f"configs[4]-shaped store, {layers} of 32 layers, every document kept",
+            "bound": "hbm", "bytes_per_launch": nbytes, "ms_per_launch": ms, "achieved": gbs, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
+
+
 def whole_job(ms, tokens_per_step, steps, world, device):
     """Whole-job numbers of a replica run: every rank processed `tokens_per_step` tokens per step in `ms`
     milliseconds for `steps` steps; the job's time is the slowest rank's, its work the sum over ranks.
@@ -520,11 +557,13 @@ def main():
     launch_mode = "cuda graph per ring slot" if graphs is not None else "eager"
     call_mode = ("one attention call per run of layers between two pruning layers (every layer's query states "
                  "are inputs of the step)") if wl.batch_layers else "one attention call per layer"
-    repo = None
+    repo = assemble = None
     if world == 1 and not args.skip_reposition:
         del wl, graphs, host, q0, k0, v0, resident
         torch.cuda.empty_cache()
         repo = reposition_roofline(device, peaks)
+        torch.cuda.empty_cache()
+        assemble = assemble_roofline(device, peaks)
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -554,7 +593,8 @@ def main():
                        "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "cpu_baseline": cpu}
+            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble,
+            "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
