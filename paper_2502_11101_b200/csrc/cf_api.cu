@@ -385,7 +385,8 @@ int cf_plan_init(const cf_geom* geom, const cf_batch* batch, const int32_t* orde
         return CF_ERR_RANGE;
     PlanView pv = make_plan_view(geom, batch, plan);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(pv.status, 0, 16, s) != cudaSuccess) return CF_ERR_CUDA;
+    rc = launch_clear_status(pv, s);
+    if (rc != CF_OK) return rc;
     return launch_plan(make_geom_view(geom), make_batch_view(batch), pv, 0, order, kept_count,
                        query_start, nullptr, 0, nullptr, CF_ALLOC_ALIGN, s);
 }

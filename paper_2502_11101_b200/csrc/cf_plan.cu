@@ -368,6 +368,17 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     }
 }
 
+// Clears the status words of a plan (a one-thread kernel: a kernel node after a kernel node costs
+// less than a memset node between two kernels).
+__global__ void clear_status_kernel(int* status) {
+    status[0] = status[1] = status[2] = status[3] = 0;
+}
+
+int launch_clear_status(const PlanView& pv, cudaStream_t stream) {
+    clear_status_kernel<<<1, 1, 0, stream>>>(pv.status);
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
+
 int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
                 const int* order, const int* kept_count, int query_start, const float* score_accum,
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream) {

@@ -66,8 +66,7 @@ reposition_kernel(BatchView bv, PlanView pv, int n_kv_heads, long long layer_str
 
     const int b = blockIdx.z;
     const int layer = blockIdx.y;
-    const int doc0 = bv.req_doc_begin[b];
-    const int base = tile_base(doc0, bv.doc_offsets[doc0]);
+    const int base = pv.tile_begin[b];                              // = tile_base of the request, one load instead of two
     const int n_tiles = pv.n_tiles[b];
     const T* src = k_in + (long long)layer * layer_stride;
     T* dst = k_out + (long long)layer * layer_stride;
@@ -142,8 +141,7 @@ assemble_kernel(BatchView bv, PlanView pv, int n_kv_heads, long long layer_strid
     constexpr int kVecPerHead = D / E;
     __shared__ int s_red[kRepoThreads / 32];
     const int b = blockIdx.z, layer = blockIdx.y;
-    const int doc0 = bv.req_doc_begin[b];
-    const int base = tile_base(doc0, bv.doc_offsets[doc0]);
+    const int base = pv.tile_begin[b];                              // = tile_base of the request, one load instead of two
     const int n_tiles = pv.n_tiles[b];
     const int ti = blockIdx.x;
     if (ti > n_tiles) return;
