@@ -453,3 +453,34 @@ def test_assembled_final_cache(dtype, head_dim):
     torch.cuda.synchronize()
     import paper_2502_11101_b200 as cf
     assert sess.status() == cf.CF_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("group,q_len", [(8, 32), (7, 37), (3, 43), (8, 64), (5, 77)])
+def test_row_counts_around_the_row_tile_boundaries(group, q_len):
+    """256, 259, 129, 512 and 385 query rows per kv head: full row groups, a three-row remainder, one
+    row over a tile, two full groups, an odd number of row tiles."""
+    lens = [129, 64, 192, 1, 128]
+    cfg = W.WorkloadConfig("row-tiles", 2, 2 * group, 2, 128, "bf16", 1e4, 8192, len(lens), 1, 300, q_len, 1, 1, ())
+    for batch_layers, self_block in ((False, False), (True, True)):
+        harness.run_and_compare(cfg, 3, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=0.0,
+                                batch_layers=batch_layers, self_block=self_block)
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_random_shapes(case):
+    """Seeded random geometries around the tile boundaries of the tensor-core kernel (row counts next to
+    128 and 256, one- to three-tile documents, several requests), without pruning so that no score gap
+    can decide a result; random call granularity and query-self block."""
+    rng = np.random.default_rng(1000 + case)
+    n_kv = int(rng.choice([1, 2, 4]))
+    group = int(rng.choice([1, 2, 3, 5, 7, 8]))
+    q_len = int(rng.choice([1, 3, 16, 18, 19, 26, 32, 37, 43, 64]))
+    n_docs = int(rng.integers(1, 7))
+    batch = int(rng.integers(1, 4))
+    n_layers = int(rng.integers(1, 4))
+    lens = [int(x) for x in rng.choice([1, 31, 32, 33, 95, 96, 97, 127, 128, 129, 191, 192, 193, 257, 300],
+                                       size=n_docs * batch)]
+    cfg = W.WorkloadConfig(f"random-{case}", n_layers, n_kv * group, n_kv, 128, "bf16", 1e4, 8192, n_docs, 1, 300,
+                           q_len, batch, 1, ())
+    harness.run_and_compare(cfg, case, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=0.0,
+                            batch_layers=bool(rng.integers(0, 2)), self_block=bool(rng.integers(0, 2)))
