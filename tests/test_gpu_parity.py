@@ -484,3 +484,48 @@ def test_random_shapes(case):
                            q_len, batch, 1, ())
     harness.run_and_compare(cfg, case, oracle.ALLOC_ALIGN, doc_len_override=lens, min_margin=0.0,
                             batch_layers=bool(rng.integers(0, 2)), self_block=bool(rng.integers(0, 2)))
+
+
+def test_query_self_block_when_a_request_has_no_documents():
+    """With nothing cached to attend, the layer's attention is the causal query-self block alone."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    lens = np.array([40, 130], dtype=np.int32)                       # request 0: none; request 1: two documents
+    req = np.array([0, 0, 2], dtype=np.int32)
+    hq, hkv, d, lq = 4, 2, 128, 7
+    gen = torch.Generator().manual_seed(1)
+    q = torch.randn((1, 2, lq, hq, d), generator=gen).bfloat16().cuda()
+    k = torch.randn((1, 170, hkv, d), generator=gen).bfloat16().cuda()
+    v = torch.randn((1, 170, hkv, d), generator=gen).bfloat16().cuda()
+    ks = torch.randn((1, 2, lq, hkv, d), generator=gen).bfloat16().cuda()
+    vs = torch.randn((1, 2, lq, hkv, d), generator=gen).bfloat16().cuda()
+    for path in (0, 1):
+        cf.cf_set_attn_path(path)
+        try:
+            sess = Session(hq, hkv, d, torch.bfloat16, 4096, 1e4, lq, lens, req, np.zeros(2, dtype=np.int32), tail_reserve=lq)
+            sess.init()
+            out = torch.full_like(q, float("nan"))
+            lse = torch.full((1, 2, hq, lq), float("nan"), device="cuda")
+            scores = torch.full((1, 2), float("nan"), device="cuda")
+            sess.attend_layers(q, k, v, out, lse, scores, k_self=ks, v_self=vs)
+            torch.cuda.synchronize()
+        finally:
+            cf.cf_set_attn_path(0)
+        assert sess.status() == 0
+        o_self, lse_self = oracle.query_self_block(q[0, 0].double().cpu().numpy(), ks[0, 0].double().cpu().numpy(),
+                                                   vs[0, 0].double().cpu().numpy())
+        got = out[0, 0].float().cpu().numpy()
+        assert np.all(np.abs(got - o_self) <= 1e-2 + 2e-2 * np.abs(o_self))
+        assert np.all(np.abs(lse[0, 0].cpu().numpy() - lse_self) <= 1e-2)
+        # request 1: documents and the block, merged
+        dst, _, _, _ = oracle.allocate_positions(lens, [0, 1], 4096, 0, lq)
+        kr = oracle.reposition_keys(k[0].double().cpu().numpy(), [0, 40, 170], [0, 0], dst, [0, 1], 1e4)
+        o_d, lse_d, _, s_ref = oracle.query_prefill_attn(q[0, 1].double().cpu().numpy(), kr, v[0].double().cpu().numpy(),
+                                                         [0, 40, 170], [0, 1], 2)
+        o_s, lse_s = oracle.query_self_block(q[0, 1].double().cpu().numpy(), ks[0, 1].double().cpu().numpy(),
+                                             vs[0, 1].double().cpu().numpy())
+        o_ref, lse_ref = oracle.merge_softmax_blocks(o_d, lse_d, o_s, lse_s)
+        got = out[0, 1].float().cpu().numpy()
+        assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
+        assert np.all(np.abs(lse[0, 1].cpu().numpy() - lse_ref) <= 1e-2)
+        assert np.allclose(scores[0].cpu().numpy(), s_ref, rtol=2e-2, atol=1e-3)
