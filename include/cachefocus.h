@@ -175,6 +175,17 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
                        int32_t n_layers, int64_t layer_stride, const void* k_in, void* k_out,
                        void* stream);
 
+/* Attention over the union of two disjoint key sets from the attention over each (Eq. 1 is a softmax,
+ * so two results combine through their log-sum-exp): for instance the kept documents and a pinned
+ * segment such as the shared prefix cache C_prefix of Algorithm 2, which is attended by a call of its
+ * own (a batch whose only "document" is the prefix, cached and kept at the same positions, so its
+ * delta is 0; it is in no kept list, hence never pruned, and the documents' scores are untouched).
+ *   out_a, out_b, out  device [n_blocks][q_len][n_q_heads][head_dim], storage type (out may be out_a or out_b)
+ *   lse_a, lse_b, lse  device float [n_blocks][n_q_heads][q_len], natural log; lse may be NULL
+ *   n_blocks           layers x requests covered by the buffers */
+int cf_merge_attn(const cf_geom* geom, int32_t n_blocks, int32_t q_len, const void* out_a, const float* lse_a,
+                  const void* out_b, const float* lse_b, void* out, float* lse, void* stream);
+
 /* Algorithm 2, Phase 2, assembled (C_final): for every layer and request, the re-positioned keys
  * (Eq. 5) and the values of the surviving documents, packed in rank order (rank 0 first), followed by
  * the query tokens' own keys and values (C_Q^l, unchanged).

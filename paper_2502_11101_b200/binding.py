@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
-           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
 
 
 class cf_geom(ctypes.Structure):
@@ -86,6 +86,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_query_prefill_attn_layers.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64,
                                                  vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_assemble_final_cache.argtypes = [gp, bp, vp, i32, i64, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
+    lib.cf_merge_attn.argtypes = [gp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.cf_attn_workspace_bytes_full.restype = ctypes.c_size_t
     lib.cf_attn_workspace_bytes_full.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_full.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, vp, vp, i64, ctypes.c_float,
@@ -252,6 +253,18 @@ def cf_assemble_final_cache(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, 
         k_cache.data_ptr(), v_cache.data_ptr(), k_self.stride(0), k_self.data_ptr(), v_self.data_ptr(),
         k_out.shape[2], k_out.data_ptr(), v_out.data_ptr(), final_rows.data_ptr(), _stream(stream))
     _check(rc, "cf_assemble_final_cache")
+
+
+def cf_merge_attn(geom: cf_geom, out_a: torch.Tensor, lse_a: torch.Tensor, out_b: torch.Tensor, lse_b: torch.Tensor,
+                  out: torch.Tensor, lse: Optional[torch.Tensor] = None, stream=None) -> None:
+    """out_* [..., Lq, Hq, D] and lse_* [..., Hq, Lq] with the same leading dimensions, all contiguous."""
+    for t in (out_a, out_b, out, lse_a, lse_b):
+        assert t.is_contiguous()
+    q_len = out_a.shape[-3]
+    n_blocks = out_a.numel() // (q_len * out_a.shape[-2] * out_a.shape[-1])
+    rc = load_library().cf_merge_attn(ctypes.byref(geom), n_blocks, q_len, out_a.data_ptr(), lse_a.data_ptr(),
+                                      out_b.data_ptr(), lse_b.data_ptr(), out.data_ptr(), _ptr(lse), _stream(stream))
+    _check(rc, "cf_merge_attn")
 
 
 def cf_attn_workspace_bytes_full(geom: cf_geom, batch: cf_batch, n_layers: int) -> int:

@@ -420,6 +420,16 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
                              static_cast<cudaStream_t>(stream));
 }
 
+int cf_merge_attn(const cf_geom* geom, int32_t n_blocks, int32_t q_len, const void* out_a, const float* lse_a,
+                  const void* out_b, const float* lse_b, void* out, float* lse, void* stream) {
+    int rc = validate(geom, nullptr);
+    if (rc != CF_OK) return rc;
+    if (n_blocks <= 0 || q_len <= 0 || !out_a || !lse_a || !out_b || !lse_b || !out) return CF_ERR_INVALID_ARG;
+    const long long n_rows = (long long)n_blocks * q_len * geom->n_q_heads;
+    return launch_merge_attn(geom, n_rows, q_len, out_a, lse_a, out_b, lse_b, out, lse,
+                             static_cast<cudaStream_t>(stream));
+}
+
 int cf_assemble_final_cache(const cf_geom* geom, const cf_batch* batch, const void* plan,
                             int32_t n_layers, int64_t layer_stride, const void* k_cache, const void* v_cache,
                             int64_t self_layer_stride, const void* k_self, const void* v_self,

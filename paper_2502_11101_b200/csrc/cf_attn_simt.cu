@@ -3,6 +3,7 @@
 // kernel serves the geometries the tensor-core kernel does not cover (fp32 storage, head_dim
 // 64) and is the second implementation the tensor-core kernel is checked against.
 #include <algorithm>
+#include <type_traits>
 
 #include "cf_common.cuh"
 
@@ -346,6 +347,52 @@ score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float*
         }
         if (score_accum) score_accum[doc] = acc;
     }
+}
+
+// Softmax attention over the union of two disjoint key sets from the results over each set:
+// one warp per (block, query token, head); weights 2^(lse - max) so nothing overflows.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+merge_attn_kernel(long long n_rows, int n_q_heads, int lq, const T* __restrict__ out_a, const float* __restrict__ lse_a,
+                  const T* __restrict__ out_b, const float* __restrict__ lse_b, T* __restrict__ out,
+                  float* __restrict__ lse) {
+    constexpr int V = D / 32;
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // index into out: (block, token, head)
+    if (row >= n_rows) return;
+    const long long blk = row / ((long long)lq * n_q_heads);
+    const int rem = (int)(row - blk * lq * n_q_heads);
+    const int j = rem / n_q_heads, h = rem - j * n_q_heads;
+    const long long li = (blk * n_q_heads + h) * lq + j;                      // index into lse: (block, head, token)
+    const float la = lse_a[li], lb = lse_b[li];
+    const float m = fmaxf(la, lb);
+    const float wa = la > -INFINITY ? expf(la - m) : 0.f, wb = lb > -INFINITY ? expf(lb - m) : 0.f;
+    const float inv = wa + wb > 0.f ? 1.f / (wa + wb) : 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        const long long e = row * D + lane * V + i;
+        out[e] = from_float<T>((to_float(out_a[e]) * wa + to_float(out_b[e]) * wb) * inv);
+    }
+    if (lane == 0 && lse) lse[li] = wa + wb > 0.f ? m + logf(wa + wb) : -INFINITY;
+}
+
+int launch_merge_attn(const cf_geom* g, long long n_rows, int q_len, const void* out_a, const float* lse_a,
+                      const void* out_b, const float* lse_b, void* out, float* lse, cudaStream_t stream) {
+    const long long blocks = (n_rows + 7) / 8;
+    if (blocks <= 0 || blocks > 0x7fffffffLL) return CF_ERR_INVALID_ARG;
+    auto run = [&](auto kernel, auto* typed) {
+        using T = std::remove_pointer_t<decltype(typed)>;
+        kernel<<<(unsigned)blocks, 256, 0, stream>>>(n_rows, g->n_q_heads, q_len, static_cast<const T*>(out_a), lse_a,
+                                                    static_cast<const T*>(out_b), lse_b, static_cast<T*>(out), lse);
+    };
+    if (g->dtype == CF_BF16) {
+        if (g->head_dim == 128) run(merge_attn_kernel<__nv_bfloat16, 128>, (__nv_bfloat16*)nullptr);
+        else run(merge_attn_kernel<__nv_bfloat16, 64>, (__nv_bfloat16*)nullptr);
+    } else {
+        if (g->head_dim == 128) run(merge_attn_kernel<float, 128>, (float*)nullptr);
+        else run(merge_attn_kernel<float, 64>, (float*)nullptr);
+    }
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
 template <typename T, int D>

@@ -99,6 +99,8 @@ struct LayerSpan {
 int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int mode,
                 const int* order, const int* kept_count, int query_start, const float* score_accum,
                 int keep, const int* keep_per_request, int strategy, cudaStream_t stream);
+int launch_merge_attn(const cf_geom* g, long long n_rows, int q_len, const void* out_a, const float* lse_a,
+                      const void* out_b, const float* lse_b, void* out, float* lse, cudaStream_t stream);
 int launch_clear_status(const PlanView& pv, cudaStream_t stream);
 int launch_reposition(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers,
                       long long layer_stride, const void* k_in, void* k_out, cudaStream_t stream);

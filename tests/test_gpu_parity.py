@@ -529,3 +529,67 @@ def test_query_self_block_when_a_request_has_no_documents():
         assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
         assert np.all(np.abs(lse[0, 1].cpu().numpy() - lse_ref) <= 1e-2)
         assert np.allclose(scores[0].cpu().numpy(), s_ref, rtol=2e-2, atol=1e-3)
+
+
+def test_pinned_prefix_attended_by_its_own_call_and_merged():
+    """A shared prefix cache (Algorithm 2, C_prefix): attended by a call of its own with delta 0, merged
+    with the documents' result by cf_merge_attn; it is in no kept list, so it is never pruned and the
+    documents' scores are those of the documents alone."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    hq, hkv, d, lq, prefix, pos_range, theta = 8, 2, 128, 6, 40, 4096, 1e4
+    lens = np.array([130, 64, 17, 96, 200], dtype=np.int32)
+    gen = torch.Generator().manual_seed(2)
+    q = torch.randn((2, 1, lq, hq, d), generator=gen).bfloat16()
+    k = torch.randn((2, int(lens.sum()), hkv, d), generator=gen).bfloat16()
+    v = torch.randn((2, int(lens.sum()), hkv, d), generator=gen).bfloat16()
+    kp = torch.randn((2, prefix, hkv, d), generator=gen).bfloat16()          # prefix keys, as cached at positions 0..39
+    vp = torch.randn((2, prefix, hkv, d), generator=gen).bfloat16()
+    docs = Session(hq, hkv, d, torch.bfloat16, pos_range, theta, lq, lens, np.array([0, 5], dtype=np.int32),
+                   np.full(5, prefix, dtype=np.int32), tail_reserve=lq, prefix_len=prefix)
+    qs = pos_range - lq
+    # the prefix as the one "document" of a batch of its own; cached where the allocation will put it => delta 0
+    pre = Session(hq, hkv, d, torch.bfloat16, pos_range, theta, lq, np.array([prefix], dtype=np.int32),
+                  np.array([0, 1], dtype=np.int32), np.array([qs - prefix], dtype=np.int32), tail_reserve=lq)
+    qg, kg, vg, kpg, vpg = [t.cuda() for t in (q, k, v, kp, vp)]
+    docs.init()
+    pre.init()
+    assert int(pre.read_plan()["dst_start"][0]) == qs - prefix
+    out_a, out_b = torch.empty_like(qg), torch.empty_like(qg)
+    lse_a = torch.empty((2, 1, hq, lq), device="cuda")
+    lse_b = torch.empty_like(lse_a)
+    scores = torch.empty((2, 5), device="cuda")
+    for layer in range(2):
+        docs.attend(qg[layer], kg[layer], vg[layer], out_a[layer], lse_a[layer])
+        scores[layer].copy_(docs.doc_scores)
+        pre.attend(qg[layer], kpg[layer], vpg[layer], out_b[layer], lse_b[layer])
+        if layer == 0:
+            docs.prune(3, oracle.ALLOC_ALIGN)
+    out = torch.empty_like(qg)
+    lse = torch.empty_like(lse_a)
+    cf.cf_merge_attn(docs.geom, out_a, lse_a, out_b, lse_b, out, lse)
+    torch.cuda.synchronize()
+    assert docs.status() == 0 and pre.status() == 0
+    # oracle: one softmax over the prefix (keys as cached) and the kept documents (keys re-positioned)
+    offsets = np.concatenate([[0], np.cumsum(lens)])
+    order = list(range(5))
+    accum = np.zeros(5)
+    for layer in range(2):
+        dst, _, _, _ = oracle.allocate_positions(lens, order, pos_range, prefix, lq)
+        assert np.all(dst[order] >= prefix)                                  # documents stay clear of the prefix positions
+        k_rot = oracle.reposition_keys(k[layer].double().numpy(), offsets, np.full(5, prefix), dst, order, theta)
+        k_all = np.concatenate([kp[layer].double().numpy(), k_rot])
+        v_all = np.concatenate([vp[layer].double().numpy(), v[layer].double().numpy()])
+        off_all = np.concatenate([[0], prefix + offsets])
+        o_ref, lse_ref, _, _ = oracle.query_prefill_attn(q[layer, 0].double().numpy(), k_all, v_all, off_all,
+                                                         [0] + [1 + i for i in order], 6)
+        _, _, _, s_docs = oracle.query_prefill_attn(q[layer, 0].double().numpy(), k_rot, v[layer].double().numpy(),
+                                                    offsets, order, 5)
+        got = out[layer, 0].float().cpu().numpy()
+        assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
+        assert np.all(np.abs(lse[layer, 0].cpu().numpy() - lse_ref) <= 1e-2)
+        assert np.allclose(scores[layer].cpu().numpy(), s_docs, rtol=2e-2, atol=1e-3)
+        accum += s_docs
+        if layer == 0:
+            order = oracle.prune_topk(accum, order, 3, oracle.ALLOC_ALIGN)
+    assert docs.read_plan()["order"][0] == order
