@@ -593,3 +593,56 @@ def test_pinned_prefix_attended_by_its_own_call_and_merged():
         if layer == 0:
             order = oracle.prune_topk(accum, order, 3, oracle.ALLOC_ALIGN)
     assert docs.read_plan()["order"][0] == order
+
+
+def test_decoding_step_over_the_assembled_final_cache():
+    """A new token's query row attends a request's final cache straight out of cf_assemble_final_cache:
+    each request's packed rows are one "document" cached where the allocation puts it (delta 0), the
+    unused tail of its slot a second document that is never kept."""
+    from paper_2502_11101_b200.session import Session
+    cfg = W.WorkloadConfig("decode", 2, 8, 2, 128, "bf16", 1e4, 4096, 7, 20, 150, 5, 2, 2, ((1, 3),))
+    seed = _pick_seed(cfg, oracle.ALLOC_ALIGN, 1e-3)
+    meta = W.make_meta(cfg, seed)
+    q, (k, v), (k_self, v_self) = W.make_q(meta), W.make_kv(meta), W.make_kv_self(meta)
+    ref = harness.oracle_stack(meta, q, k, v, oracle.ALLOC_ALIGN)
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, 128, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta, cfg.q_len,
+                   meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+    qg, kg, vg, ksg, vsg = [t.cuda() for t in (q, k, v, k_self, v_self)]
+    sess.run_stack(qg, kg, vg, cfg.schedule, oracle.ALLOC_ALIGN, torch.empty_like(qg))
+    out_rows = 3 * 150 + cfg.q_len + 9
+    k_out = torch.zeros((cfg.n_layers, cfg.batch, out_rows, cfg.n_kv_heads, 128), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.zeros_like(k_out)
+    final_rows = torch.zeros(cfg.batch, dtype=torch.int32, device="cuda")
+    sess.assemble(kg, vg, ksg, vsg, k_out, v_out, final_rows)
+    rows = final_rows.cpu().numpy()
+    # the decoding batch: per request (final cache, unused tail), only the first kept
+    doc_len = np.stack([rows, out_rows - rows], axis=1).reshape(-1).astype(np.int32)
+    qs = cfg.pos_range - 1
+    src = np.stack([qs - rows, np.zeros_like(rows)], axis=1).reshape(-1).astype(np.int32)
+    dec = Session(cfg.n_q_heads, cfg.n_kv_heads, 128, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta, 1, doc_len,
+                  np.arange(cfg.batch + 1, dtype=np.int32) * 2, src, tail_reserve=1, n_reuse=1)
+    order = torch.tensor([0, 1] * cfg.batch, dtype=torch.int32, device="cuda")
+    kept_count = torch.ones(cfg.batch, dtype=torch.int32, device="cuda")
+    dec.set_live_docs(1)
+    dec.init(order, kept_count)
+    gen = torch.Generator().manual_seed(3)
+    q_new = torch.randn((cfg.n_layers, cfg.batch, 1, cfg.n_q_heads, 128), generator=gen).bfloat16().cuda()
+    out = torch.empty_like(q_new)
+    lse = torch.empty((cfg.n_layers, cfg.batch, cfg.n_q_heads, 1), device="cuda")
+    dec.attend_layers(q_new, k_out.view(cfg.n_layers, cfg.batch * out_rows, cfg.n_kv_heads, 128),
+                      v_out.view(cfg.n_layers, cfg.batch * out_rows, cfg.n_kv_heads, 128), out, lse)
+    torch.cuda.synchronize()
+    assert dec.status() == 0 and sess.status() == 0
+    assert [len(o) for o in dec.read_plan()["order"]] == [1] * cfg.batch
+    for b in range(cfg.batch):
+        lo = int(meta.req_doc_begin[b])
+        for l in range(cfg.n_layers):
+            kf, vf = oracle.assemble_final_cache(ref[b]["k_final"][l], v[l].double().numpy(), meta.doc_offsets,
+                                                 ref[b]["order"], k_self[l, b].double().numpy(),
+                                                 v_self[l, b].double().numpy(), doc_base=lo)
+            assert kf.shape[0] == rows[b]
+            o_ref, lse_ref, _, _ = oracle.query_prefill_attn(q_new[l, b].double().cpu().numpy(), kf, vf,
+                                                             [0, kf.shape[0]], [0], 1)
+            got = out[l, b].float().cpu().numpy()
+            assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
+            assert np.all(np.abs(lse[l, b].cpu().numpy() - lse_ref) <= 1e-2)
