@@ -181,7 +181,7 @@ int cf_reposition_keys(const cf_geom* geom, const cf_batch* batch, const void* p
  * own (a batch whose only "document" is the prefix, cached and kept at the same positions, so its
  * delta is 0; it is in no kept list, hence never pruned, and the documents' scores are untouched).
  *   out_a, out_b, out  device [n_blocks][q_len][n_q_heads][head_dim], storage type (out may be out_a or out_b)
- *   lse_a, lse_b, lse  device float [n_blocks][n_q_heads][q_len], natural log; lse may be NULL
+ *   lse_a, lse_b, lse  device float [n_blocks][n_q_heads][q_len], natural log; lse may be NULL, lse_a or lse_b
  *   n_blocks           layers x requests covered by the buffers */
 int cf_merge_attn(const cf_geom* geom, int32_t n_blocks, int32_t q_len, const void* out_a, const float* lse_a,
                   const void* out_b, const float* lse_b, void* out, float* lse, void* stream);
@@ -194,8 +194,9 @@ int cf_merge_attn(const cf_geom* geom, int32_t n_blocks, int32_t q_len, const vo
  *   k_out, v_out      device [n_layers][n_requests][out_rows][n_kv_heads][head_dim], dense; request b
  *                     receives final_rows[b] rows per layer, rows beyond stay untouched
  *   final_rows        device int32 [n_requests]: tokens of the survivors + q_len
- * A request whose rows do not fit out_rows is not written and CF_ERR_WORKSPACE is recorded in the
- * plan's status word. */
+ * A request whose rows do not fit out_rows raises CF_ERR_WORKSPACE in the plan's status word; its
+ * final_rows entry is not written, the leading tiles that do fit may have been copied, and nothing
+ * is ever written beyond out_rows. */
 int cf_assemble_final_cache(const cf_geom* geom, const cf_batch* batch, const void* plan,
                             int32_t n_layers, int64_t layer_stride, const void* k_cache, const void* v_cache,
                             int64_t self_layer_stride, const void* k_self, const void* v_self,
@@ -305,19 +306,60 @@ int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
                   const float* score_accum, int32_t keep, const int32_t* keep_per_request,
                   int32_t strategy, void* stream);
 
-/* Selects the attention kernel: 0 = automatic (tensor-core kernel when the geometry allows),
- * 1 = force the portable CUDA-core kernel.  Process-wide; meant for tests and debugging. */
-int cf_set_attn_path(int32_t path);
+/* Host-side mirror of the pruning step alone (Algorithm 2: argsort of S, prun), integers and scores
+ * in host memory, nothing launched: among the documents of `order` (n_kept distinct local ids, rank
+ * order) keeps the min(keep, n_kept) with the largest score_accum[id] (ties: lower id) and writes
+ * them to order_out (capacity min(keep, n_kept)): in their previous relative order for CF_ALLOC_NONE
+ * and CF_ALLOC_ALIGN, best first for CF_ALLOC_SORT.  *n_out receives their number.  The device call
+ * cf_prune_topk takes the same decisions; this one serves callers that hold S on the host, and tests. */
+int cf_prune_topk_host(int32_t n_docs, const float* score_accum, const int32_t* order, int32_t n_kept,
+                       int32_t keep, int32_t strategy, int32_t* order_out, int32_t* n_out);
 
-/* Timing aid for benchmarks (not part of the method).  cf_profile_begin(n) makes every later
- * cf_query_prefill_attn call bracket its main attention kernel (the fused re-position +
- * QK^T + softmax + PV kernel, without the small merge kernels) with a pair of CUDA events on
- * the launching stream, for at most n calls.  cf_profile_end() waits for those events, writes
- * the kernel durations in milliseconds to the host array `ms` (capacity entries), the number
- * of recorded launches to *count, and switches recording off.  Do not use inside stream
- * capture.  The events are created by cf_profile_begin and destroyed by cf_profile_end. */
-int cf_profile_begin(int32_t max_records);
-int cf_profile_end(float* ms, int32_t capacity, int32_t* count);
+/* Algorithm 2, Phases 1 and 2, for a whole layer stack whose per-layer query states are given up
+ * front (benchmarks, replay, scoring passes with stored queries; inside a running model layer l+1's
+ * queries come out of layer l, and the per-layer calls above apply).  The struct is host memory read
+ * during the call; the buffers it names are device memory unless marked host. */
+typedef struct cf_stack {
+    int32_t n_layers;
+    int32_t n_prune;              /* pruning layers in the schedule                                   */
+    const int32_t* prune_layer;   /* host [n_prune]: 1-based layers, strictly ascending; pruning
+                                     happens after that layer's scores are accumulated                */
+    const int32_t* prune_keep;    /* host [n_prune]: documents kept per request from then on          */
+    int32_t strategy;             /* CF_ALLOC_NONE | CF_ALLOC_ALIGN | CF_ALLOC_SORT                   */
+    int32_t batch_layers;         /* 0: one attention launch chain per layer; 1: one per run of layers
+                                     between two pruning layers (same results up to the tolerance of
+                                     the split-KV merge)                                              */
+    float   softmax_scale;        /* 0 selects 1/sqrt(head_dim)                                       */
+    int32_t reserved;
+    const void* q;                /* [n_layers][n_requests][q_len][n_q_heads][head_dim]               */
+    int64_t q_layer_stride;       /* elements between layers, as in cf_query_prefill_attn_layers      */
+    const void* k_cache;          /* the store, n_layers layers                                       */
+    const void* v_cache;
+    int64_t kv_layer_stride;
+    const void* k_self;           /* NULL, or the query tokens' own keys/values: every layer then     */
+    const void* v_self;           /* also attends the causal query-self block (..._attn_full)         */
+    int64_t self_layer_stride;
+    void*   out;                  /* [n_layers][n_requests][q_len][n_q_heads][head_dim]               */
+    int64_t out_layer_stride;
+    float*  lse;                  /* [n_layers][n_requests][n_q_heads][q_len] or NULL                 */
+    float*  layer_scores;         /* [n_layers][n_docs_total] every layer's s^l, or NULL              */
+    float*  score_accum;          /* [n_docs_total] S: cleared by the call, holds the sums at the end */
+    void*   k_final;              /* NULL, or a store-shaped buffer that receives Phase 2 (may be
+                                     k_cache itself)                                                  */
+    const int32_t* doc_len_host;        /* host [n_docs_total] or NULL: lets the call size its grids  */
+    const int32_t* req_doc_begin_host;  /* host [n_requests+1] or NULL    to the documents still kept */
+} cf_stack;
+
+/* Scratch needed by cf_run_stack (the largest of its attention calls); 0 on invalid arguments. */
+size_t cf_run_stack_workspace_bytes(const cf_geom* geom, const cf_batch* batch, const cf_stack* stack);
+
+/* Runs Init (S = 0, every document kept in retrieval order, first allocation), then for l = 1..L
+ * layer_l's attention over the kept caches with S <- S + s^l and, after a scheduled layer, argsort /
+ * prun / re-allocation; finally Phase 2 if k_final is given.  Everything is queued on `stream`; the
+ * plan holds the final kept lists and positions afterwards.  Equivalent to the sequence
+ * cf_plan_init, cf_query_prefill_attn[_layers|_full] ..., cf_prune_topk ..., cf_reposition_keys. */
+int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* stack, void* plan,
+                 size_t plan_bytes, void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,11 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
-           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn", "cf_query_prefill_attn_static", "cf_prune_topk", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end"]
+           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn",
+           "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
+           "cf_run_stack", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
+_SIZE_T_EXPORTS = ("cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers", "cf_attn_workspace_bytes_full",
+                   "cf_run_stack_workspace_bytes")
 
 
 class cf_geom(ctypes.Structure):
@@ -47,6 +51,20 @@ class cf_plan_layout(ctypes.Structure):
                 ("total_bytes", "status", "kept", "kept_count", "dst_start", "group", "n_reuse", "query_start",
                  "n_tiles", "tile_begin", "doc_tile_begin", "doc_tile_count", "tile_doc", "tile_row0", "tile_len", "trig")] + \
                [("max_tiles", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class cf_stack(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_prune", ctypes.c_int32),
+                ("prune_layer", ctypes.c_void_p), ("prune_keep", ctypes.c_void_p),
+                ("strategy", ctypes.c_int32), ("batch_layers", ctypes.c_int32),
+                ("softmax_scale", ctypes.c_float), ("reserved", ctypes.c_int32),
+                ("q", ctypes.c_void_p), ("q_layer_stride", ctypes.c_int64),
+                ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p), ("kv_layer_stride", ctypes.c_int64),
+                ("k_self", ctypes.c_void_p), ("v_self", ctypes.c_void_p), ("self_layer_stride", ctypes.c_int64),
+                ("out", ctypes.c_void_p), ("out_layer_stride", ctypes.c_int64),
+                ("lse", ctypes.c_void_p), ("layer_scores", ctypes.c_void_p), ("score_accum", ctypes.c_void_p),
+                ("k_final", ctypes.c_void_p),
+                ("doc_len_host", ctypes.c_void_p), ("req_doc_begin_host", ctypes.c_void_p)]
 
 
 class CacheFocusError(RuntimeError):
@@ -93,12 +111,17 @@ def load_library() -> ctypes.CDLL:
                                                vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_query_prefill_attn_static.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
+    lib.cf_prune_topk_host.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp]
+    sp = ctypes.POINTER(cf_stack)
+    lib.cf_run_stack_workspace_bytes.restype = ctypes.c_size_t
+    lib.cf_run_stack_workspace_bytes.argtypes = [gp, bp, sp]
+    lib.cf_run_stack.argtypes = [gp, bp, sp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+    lib.cf_debug_wait_timeout.argtypes = [gp, bp, vp, i64, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
     lib.cf_profile_end.argtypes = [vp, i32, vp]
     for name in EXPORTS:
-        if name not in ("cf_error_string", "cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers",
-                        "cf_attn_workspace_bytes_full"):
+        if name != "cf_error_string" and name not in _SIZE_T_EXPORTS:
             getattr(lib, name).restype = ctypes.c_int
     _LIB = lib
     return lib
@@ -313,6 +336,68 @@ def cf_prune_topk(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, score_accu
     rc = load_library().cf_prune_topk(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), score_accum.data_ptr(),
                                       keep, _ptr(keep_per_request), strategy, _stream(stream))
     _check(rc, "cf_prune_topk")
+
+
+def cf_prune_topk_host(score_accum: Sequence[float], order: Sequence[int], keep: int, strategy: int) -> List[int]:
+    """Host-side pruning step: `score_accum` float32 by local id, `order` the kept ids by rank."""
+    scores = np.ascontiguousarray(np.asarray(score_accum, dtype=np.float32))
+    order = _i32(order)
+    out = np.zeros(max(1, len(order)), np.int32)
+    n_out = ctypes.c_int32(0)
+    rc = load_library().cf_prune_topk_host(len(scores), scores.ctypes.data, order.ctypes.data, len(order), keep,
+                                           strategy, out.ctypes.data, ctypes.addressof(n_out))
+    _check(rc, "cf_prune_topk_host")
+    return [int(x) for x in out[:n_out.value]]
+
+
+def make_stack(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+               score_accum: torch.Tensor, schedule: Sequence[Tuple[int, int]], strategy: int, batch_layers: bool,
+               lse: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
+               k_final: Optional[torch.Tensor] = None, k_self: Optional[torch.Tensor] = None,
+               v_self: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+               doc_len: Optional[np.ndarray] = None, req_doc_begin: Optional[np.ndarray] = None):
+    """A cf_stack over torch buffers (dimension 0 = layers, may be strided; the rest of a layer dense).
+    Returns (struct, keepalive): the host arrays the struct points to live in `keepalive`."""
+    n_layers = q.shape[0]
+    assert k_cache.shape[0] == n_layers and v_cache.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k_cache.stride(0) == v_cache.stride(0)
+    for t in (lse, layer_scores):
+        assert t is None or (t.shape[0] == n_layers and t.is_contiguous())
+    if k_final is not None:
+        assert k_final.shape == k_cache.shape and k_final.stride(0) == k_cache.stride(0)
+    if k_self is not None:
+        assert k_self.shape[0] == n_layers and k_self.stride(0) == v_self.stride(0)
+    sched = sorted((int(l), int(kp)) for l, kp in schedule)
+    layers, keeps = _i32([l for l, _ in sched]), _i32([kp for _, kp in sched])
+    keep = [layers, keeps]
+    dl = rb = None
+    if doc_len is not None and req_doc_begin is not None:
+        dl, rb = _i32(doc_len), _i32(req_doc_begin)
+        keep += [dl, rb]
+    st = cf_stack(n_layers, len(sched), layers.ctypes.data if len(sched) else None,
+                  keeps.ctypes.data if len(sched) else None, strategy, 1 if batch_layers else 0, softmax_scale, 0,
+                  q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(0),
+                  _ptr(k_self), _ptr(v_self), 0 if k_self is None else k_self.stride(0),
+                  out.data_ptr(), out.stride(0), _ptr(lse), _ptr(layer_scores), score_accum.data_ptr(),
+                  _ptr(k_final), None if dl is None else dl.ctypes.data, None if rb is None else rb.ctypes.data)
+    return st, keep
+
+
+def cf_run_stack_workspace_bytes(geom: cf_geom, batch: cf_batch, stack: cf_stack) -> int:
+    return int(load_library().cf_run_stack_workspace_bytes(ctypes.byref(geom), ctypes.byref(batch), ctypes.byref(stack)))
+
+
+def cf_run_stack(geom: cf_geom, batch: cf_batch, stack: cf_stack, plan: torch.Tensor, workspace: torch.Tensor,
+                 stream=None) -> None:
+    rc = load_library().cf_run_stack(ctypes.byref(geom), ctypes.byref(batch), ctypes.byref(stack), plan.data_ptr(),
+                                     plan.numel() * plan.element_size(), workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_run_stack")
+
+
+def cf_debug_wait_timeout(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, limit_cycles: int, stream=None) -> None:
+    _check(load_library().cf_debug_wait_timeout(ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(),
+                                                limit_cycles, _stream(stream)), "cf_debug_wait_timeout")
 
 
 def cf_set_attn_path(path: int) -> None:

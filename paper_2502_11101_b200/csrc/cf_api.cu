@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <mutex>
 #include <vector>
 
 #include "cf_common.cuh"
@@ -114,15 +115,20 @@ PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan) {
     return v;
 }
 
+int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
 int sm_count() {
-    static std::atomic<int> cached{0};
-    int n = cached.load();
+    static std::atomic<int> cached[kMaxDevices] = {};
+    const int dev = current_device();
+    int n = dev >= 0 ? cached[dev].load() : 0;
     if (n > 0) return n;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+    if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
         return 148;
-    cached.store(n);
+    cached[dev].store(n);
     return n;
 }
 
@@ -210,10 +216,21 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
 static std::atomic<int> g_attn_path{0};
 int attn_path() { return g_attn_path.load(); }
 
-// Event pairs around the main attention kernel (cf_profile_begin / cf_profile_end).
+// Event pairs around the main attention kernel (cf_profile_begin / cf_profile_end); the three
+// variables change together under g_prof_mutex.
+static std::mutex g_prof_mutex;
 static std::vector<cudaEvent_t> g_prof_events;
 static int g_prof_capacity = 0;
 static int g_prof_used = 0;
+
+// Claims the next event pair if recording is on; returns its index or -1.
+static int prof_claim(cudaEvent_t* start, cudaEvent_t* stop) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (g_prof_used >= g_prof_capacity) return -1;
+    *start = g_prof_events[2 * g_prof_used];
+    *stop = g_prof_events[2 * g_prof_used + 1];
+    return g_prof_used++;
+}
 
 static int check_plan(const cf_geom* geom, const cf_batch* batch, const void* plan) {
     if (!batch || !plan) return CF_ERR_INVALID_ARG;
@@ -267,15 +284,16 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
         rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, scale * kLog2e, ws, s);
         if (rc != CF_OK) return rc;
     }
-    const bool timed = g_prof_used < g_prof_capacity;
-    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used], s);
+    cudaEvent_t ev_start, ev_stop;
+    const bool timed = prof_claim(&ev_start, &ev_stop) >= 0;
+    if (timed) cudaEventRecord(ev_start, s);
     if (tensor_core) {
         ws.part_bf16 = 1;
         ws.self_mode = with_self ? 2 : 0;             // the block rides along as one more key tile
         rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, k_self, v_self, self_stride, scale * kLog2e, ws, s);
     } else
         rc = launch_attn_simt(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
-    if (timed) cudaEventRecord(g_prof_events[2 * g_prof_used++ + 1], s);
+    if (timed) cudaEventRecord(ev_stop, s);
     if (rc != CF_OK) return rc;
     return launch_combine(geom, batch, pv, span, ws, out, lse, doc_scores, score_accum, s);
 }
@@ -467,6 +485,7 @@ size_t cf_attn_workspace_bytes(const cf_geom* geom, const cf_batch* batch) {
 }
 
 int cf_profile_begin(int32_t max_records) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
     if (max_records <= 0 || max_records > (1 << 20) || g_prof_capacity != 0) return CF_ERR_INVALID_ARG;
     g_prof_events.resize(2 * (size_t)max_records);
     for (auto& e : g_prof_events)
@@ -478,6 +497,7 @@ int cf_profile_begin(int32_t max_records) {
 
 int cf_profile_end(float* ms, int32_t capacity, int32_t* count) {
     if (!count || capacity < 0 || (capacity > 0 && !ms)) return CF_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
     int rc = CF_OK;
     const int n = g_prof_used;
     for (int i = 0; i < n; ++i) {

@@ -126,14 +126,11 @@ int launch_self_typed(const cf_geom* g, const cf_batch* b, const LayerSpan& span
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const size_t smem = self_keys_bytes<T, D>(b->q_len) + (size_t)b->q_len * D * sizeof(T) +
                         (size_t)(kSelfThreads / 32) * D * sizeof(float);
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(self_block_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(self_keys_bytes<T, D>(kSelfMaxLq) + (size_t)kSelfMaxLq * D * sizeof(T) +
-                                       (kSelfThreads / 32) * D * sizeof(float))) != cudaSuccess)
-            return CF_ERR_CUDA;
-        configured = true;
-    }
+    static PerDeviceOnce configured;
+    if (configure_smem_once(configured, self_block_kernel<T, D>,
+                            (int)(self_keys_bytes<T, D>(kSelfMaxLq) + (size_t)kSelfMaxLq * D * sizeof(T) +
+                                  (kSelfThreads / 32) * D * sizeof(float))) != CF_OK)
+        return CF_ERR_CUDA;
     dim3 grid((unsigned)((rows + kSelfRows - 1) / kSelfRows), (unsigned)g->n_kv_heads,
               (unsigned)(b->n_requests * span.n_layers));
     self_block_kernel<T, D><<<grid, kSelfThreads, smem, stream>>>(

@@ -353,9 +353,8 @@ score_kernel(BatchView bv, PlanView pv, AttnWorkspace ws, int rows_total, float*
 // one warp per (block, query token, head); weights 2^(lse - max) so nothing overflows.
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-merge_attn_kernel(long long n_rows, int n_q_heads, int lq, const T* __restrict__ out_a, const float* __restrict__ lse_a,
-                  const T* __restrict__ out_b, const float* __restrict__ lse_b, T* __restrict__ out,
-                  float* __restrict__ lse) {
+merge_attn_kernel(long long n_rows, int n_q_heads, int lq, const T* out_a, const float* lse_a,
+                  const T* out_b, const float* lse_b, T* out, float* lse) {   // out may alias out_a or out_b, lse likewise
     constexpr int V = D / 32;
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // index into out: (block, token, head)
@@ -406,13 +405,9 @@ static int launch_simt_typed(const cf_geom* g, const cf_batch* b, const PlanView
     dim3 grid((unsigned)ws.n_splits, (unsigned)(g->n_kv_heads * row_chunks), (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
     const size_t smem = simt_smem_bytes<D>();
-    static bool configured[2] = {false, false};      // per (T, D) instantiation and slice layout
+    static PerDeviceOnce configured[2];              // per (T, D) instantiation and slice layout
     auto run = [&](auto kernel, int which) {
-        if (!configured[which]) {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return CF_ERR_CUDA;
-            configured[which] = true;
-        }
+        if (configure_smem_once(configured[which], kernel, (int)smem) != CF_OK) return CF_ERR_CUDA;
         kernel<<<grid, kSimtThreads, smem, stream>>>(bv, pv, ws, span, g->n_q_heads, g->n_kv_heads, scale_log2,
                                                      static_cast<const T*>(q), static_cast<const T*>(k),
                                                      static_cast<const T*>(v));

@@ -134,13 +134,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             return false;
         }
@@ -723,6 +724,24 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     }
 }
 
+// Exercises the bounded wait by itself: one CTA initialises an mbarrier that nothing ever arrives on,
+// every thread waits on it with the given limit, the wait gives up, and the CTA reports
+// CF_ERR_TIMEOUT through the status word exactly as the attention kernel does.  No tensor memory,
+// no copies in flight: the kernel returns by itself after about `limit_cycles` clocks.
+__global__ void __launch_bounds__(128) wait_probe_kernel(int* status, long long limit_cycles) {
+    __shared__ unsigned long long bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_word, limit_cycles);
+    __syncthreads();
+    if (threadIdx.x == 0 && !ok && abort_word) atomicCAS(status, 0, CF_ERR_TIMEOUT);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -780,6 +799,11 @@ int make_self_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf
 
 }  // namespace
 
+int launch_wait_probe(const PlanView& pv, long long limit_cycles, cudaStream_t stream) {
+    wait_probe_kernel<<<1, 128, 0, stream>>>(pv.status, limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
+
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
     return g->dtype == CF_BF16 && g->head_dim == 128 && b->total_tokens > 0 && b->n_docs_total < (1 << 23);
 }
@@ -812,13 +836,9 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
     dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
               (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
-    static bool configured[2] = {false, false};
+    static PerDeviceOnce configured[2];
     auto run = [&](auto kernel, int which) {
-        if (!configured[which]) {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-                return CF_ERR_CUDA;
-            configured[which] = true;
-        }
+        if (configure_smem_once(configured[which], kernel, kSmemBytes) != CF_OK) return CF_ERR_CUDA;
         kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, bv, pv, ws, span.q_stride, g->n_q_heads,
                                                        g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q),
                                                        k_self ? 1 : 0);

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "cachefocus.h"
+#include "cachefocus_debug.h"
 
 namespace cf {
 
@@ -58,6 +59,24 @@ BatchView make_batch_view(const cf_batch* b);
 PlanView make_plan_view(const cf_geom* g, const cf_batch* b, void* plan);
 int validate(const cf_geom* g, const cf_batch* b);
 int sm_count();
+// Index of the current device for per-device caches (attributes such as the dynamic shared memory
+// limit of a kernel and the SM count belong to a device, not to the process); -1 if unknown.
+constexpr int kMaxDevices = 64;
+int current_device();
+// One flag per device: true once the calling site has configured its kernel on that device.
+struct PerDeviceOnce {
+    bool done[kMaxDevices] = {};
+};
+// Sets the dynamic shared memory limit of `kernel` once per device; CF_OK or CF_ERR_CUDA.
+template <typename K>
+int configure_smem_once(PerDeviceOnce& once, K kernel, int bytes) {
+    const int dev = current_device();
+    if (dev >= 0 && once.done[dev]) return CF_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+        return CF_ERR_CUDA;
+    if (dev >= 0) once.done[dev] = true;
+    return CF_OK;
+}
 int choose_splits(const cf_geom* g, const cf_batch* b, int n_layers);
 int choose_row_group(const cf_geom* g, const cf_batch* b);
 int tiles_per_request_bound(const cf_batch* b);
@@ -102,6 +121,7 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
 int launch_merge_attn(const cf_geom* g, long long n_rows, int q_len, const void* out_a, const float* lse_a,
                       const void* out_b, const float* lse_b, void* out, float* lse, cudaStream_t stream);
 int launch_clear_status(const PlanView& pv, cudaStream_t stream);
+int launch_wait_probe(const PlanView& pv, long long limit_cycles, cudaStream_t stream);
 int launch_reposition(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers,
                       long long layer_stride, const void* k_in, void* k_out, cudaStream_t stream);
 int launch_assemble(const cf_geom* g, const cf_batch* b, const PlanView& pv, int n_layers, long long layer_stride,

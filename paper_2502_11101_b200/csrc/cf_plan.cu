@@ -154,12 +154,15 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     if (mode == 0) {
         n_kept = kept_count_in ? kept_count_in[b] : n_docs;
         n_kept = max(0, min(n_kept, n_docs));
+        for (int i = tid; i < n_docs; i += kPlanThreads) s_cnt[i] = 0;
+        __syncthreads();
         for (int r = tid; r < n_kept; r += kPlanThreads) {
             int id = order ? order[doc0 + r] : r;
             if (id < 0 || id >= n_docs) {
                 raise_status(pv.status, CF_ERR_INVALID_ARG);
                 id = 0;
             }
+            if (atomicAdd(&s_cnt[id], 1) != 0) raise_status(pv.status, CF_ERR_INVALID_ARG);   // an id listed twice
             s_ids[r] = id;
         }
     } else {

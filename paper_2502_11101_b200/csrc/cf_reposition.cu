@@ -128,9 +128,9 @@ reposition_kernel(BatchView bv, PlanView pv, int n_kv_heads, long long layer_str
 
 // Algorithm 2, Phase 2, assembled: per layer and request, the re-positioned keys and the values of
 // the surviving documents, packed in rank order, followed by the query tokens' own keys and values.
-// Block x of a (layer, request) handles key tile x of the plan's list (tiles are listed in rank
-// order, so a tile's first output row is the sum of the lengths of the tiles before it); block
-// n_tiles appends the query rows.  Everything is moved in 16-byte vectors.
+// The blocks of a (layer, request) stride over the key tiles of the plan's list (tiles are listed
+// in rank order, so a tile's first output row is the sum of the lengths of the tiles before it);
+// index n_tiles stands for the query rows, appended last.  Everything is moved in 16-byte vectors.
 template <typename T, int D, int LAYOUT>
 __global__ void __launch_bounds__(kRepoThreads)
 assemble_kernel(BatchView bv, PlanView pv, int n_kv_heads, long long layer_stride, long long self_stride,
@@ -143,75 +143,77 @@ assemble_kernel(BatchView bv, PlanView pv, int n_kv_heads, long long layer_strid
     const int b = blockIdx.z, layer = blockIdx.y;
     const int base = pv.tile_begin[b];                              // = tile_base of the request, one load instead of two
     const int n_tiles = pv.n_tiles[b];
-    const int ti = blockIdx.x;
-    if (ti > n_tiles) return;
-    // rows of the tiles before this one (ti == n_tiles: of all tiles)
-    int before = 0;
-    for (int t = threadIdx.x; t < ti; t += kRepoThreads) before += pv.tile_len[base + t];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = before;
-    __syncthreads();
-    before = 0;
-#pragma unroll
-    for (int w = 0; w < kRepoThreads / 32; ++w) before += s_red[w];
-
     const int row_vecs = n_kv_heads * kVecPerHead;                  // 16-byte vectors of one dense output row
     const long long out_base = (((long long)layer * bv.n_requests + b) * out_rows) * (long long)n_kv_heads * D;
-    if (ti == n_tiles) {                                            // the query tokens' own keys and values
-        const int lq = bv.q_len;
-        if (before + lq > out_rows) {
-            if (threadIdx.x == 0) atomicCAS(pv.status, 0, CF_ERR_WORKSPACE);
-            return;
-        }
-        if (layer == 0 && threadIdx.x == 0) final_rows[b] = before + lq;
-        const long long src0 = (long long)layer * self_stride + (long long)b * lq * n_kv_heads * D;
-        for (int idx = threadIdx.x; idx < lq * row_vecs; idx += kRepoThreads) {
-            const long long off = (long long)idx * E;
-            const long long dst = out_base + (long long)before * n_kv_heads * D + off;
-            *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(k_self + src0 + off);
-            *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(v_self + src0 + off);
-        }
-        return;
-    }
-    const int len = pv.tile_len[base + ti];
-    if (before + len > out_rows) return;                            // reported by the block of the query rows
-    const long long row0 = pv.tile_row0[base + ti];
-    const float2* trig = pv.trig + (size_t)pv.tile_doc[base + ti] * (D / 2);
-    const T* ksrc = k_in + (long long)layer * layer_stride;
-    const T* vsrc = v_in + (long long)layer * layer_stride;
     constexpr int kItemsPerHead = LAYOUT == CF_ROPE_HALF ? kVecPerHead / 2 : kVecPerHead;
     constexpr int kPartner = LAYOUT == CF_ROPE_HALF ? (D / 2) : 0;
     const int items_per_row = n_kv_heads * kItemsPerHead;
-    for (int it = threadIdx.x; it < len * items_per_row; it += kRepoThreads) {
-        const int row = it / items_per_row;
-        const int rem = it - row * items_per_row;
-        const int head = rem / kItemsPerHead;
-        const int vec = rem - head * kItemsPerHead;
-        const long long src = (row0 + row) * bv.token_stride + head * D + vec * E;
-        const long long dst = out_base + ((long long)(before + row) * n_kv_heads + head) * D + vec * E;
-        const int slice0 = LAYOUT == CF_ROPE_HALF ? vec * E : vec * (E / 2);
-        float a[E], ya[E];
-        unpack<T>(*reinterpret_cast<const uint4*>(ksrc + src), a);
-        *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(vsrc + src);
-        if (LAYOUT == CF_ROPE_HALF) {
-            float c[E], yc[E];
-            unpack<T>(*reinterpret_cast<const uint4*>(ksrc + src + kPartner), c);
-            *reinterpret_cast<uint4*>(v_out + dst + kPartner) = *reinterpret_cast<const uint4*>(vsrc + src + kPartner);
+    // blocks stride over the tiles, so a grid smaller than the tile count still covers every tile
+    for (int ti = blockIdx.x; ti <= n_tiles; ti += gridDim.x) {
+        // rows of the tiles before this one (ti == n_tiles: of all tiles)
+        int before = 0;
+        for (int t = threadIdx.x; t < ti; t += kRepoThreads) before += pv.tile_len[base + t];
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float2 cs = __ldg(trig + slice0 + e);
-                rotate_pair(a[e], c[e], cs.x, cs.y, ya[e], yc[e]);
-            }
-            *reinterpret_cast<uint4*>(k_out + dst) = pack<T>(ya);
-            *reinterpret_cast<uint4*>(k_out + dst + kPartner) = pack<T>(yc);
-        } else {
+        for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+        __syncthreads();                                            // the previous round's readers are done
+        if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = before;
+        __syncthreads();
+        before = 0;
 #pragma unroll
-            for (int e = 0; e < E; e += 2) {
-                const float2 cs = __ldg(trig + slice0 + e / 2);
-                rotate_pair(a[e], a[e + 1], cs.x, cs.y, ya[e], ya[e + 1]);
+        for (int w = 0; w < kRepoThreads / 32; ++w) before += s_red[w];
+
+        if (ti == n_tiles) {                                        // the query tokens' own keys and values
+            const int lq = bv.q_len;
+            if (before + lq > out_rows) {
+                if (threadIdx.x == 0) atomicCAS(pv.status, 0, CF_ERR_WORKSPACE);
+                continue;
             }
-            *reinterpret_cast<uint4*>(k_out + dst) = pack<T>(ya);
+            if (layer == 0 && threadIdx.x == 0) final_rows[b] = before + lq;
+            const long long src0 = (long long)layer * self_stride + (long long)b * lq * n_kv_heads * D;
+            for (int idx = threadIdx.x; idx < lq * row_vecs; idx += kRepoThreads) {
+                const long long off = (long long)idx * E;
+                const long long dst = out_base + (long long)before * n_kv_heads * D + off;
+                *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(k_self + src0 + off);
+                *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(v_self + src0 + off);
+            }
+            continue;
+        }
+        const int len = pv.tile_len[base + ti];
+        if (before + len > out_rows) continue;                      // reported by the block of the query rows
+        const long long row0 = pv.tile_row0[base + ti];
+        const float2* trig = pv.trig + (size_t)pv.tile_doc[base + ti] * (D / 2);
+        const T* ksrc = k_in + (long long)layer * layer_stride;
+        const T* vsrc = v_in + (long long)layer * layer_stride;
+        for (int it = threadIdx.x; it < len * items_per_row; it += kRepoThreads) {
+            const int row = it / items_per_row;
+            const int rem = it - row * items_per_row;
+            const int head = rem / kItemsPerHead;
+            const int vec = rem - head * kItemsPerHead;
+            const long long src = (row0 + row) * bv.token_stride + head * D + vec * E;
+            const long long dst = out_base + ((long long)(before + row) * n_kv_heads + head) * D + vec * E;
+            const int slice0 = LAYOUT == CF_ROPE_HALF ? vec * E : vec * (E / 2);
+            float a[E], ya[E];
+            unpack<T>(*reinterpret_cast<const uint4*>(ksrc + src), a);
+            *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(vsrc + src);
+            if (LAYOUT == CF_ROPE_HALF) {
+                float c[E], yc[E];
+                unpack<T>(*reinterpret_cast<const uint4*>(ksrc + src + kPartner), c);
+                *reinterpret_cast<uint4*>(v_out + dst + kPartner) = *reinterpret_cast<const uint4*>(vsrc + src + kPartner);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const float2 cs = __ldg(trig + slice0 + e);
+                    rotate_pair(a[e], c[e], cs.x, cs.y, ya[e], yc[e]);
+                }
+                *reinterpret_cast<uint4*>(k_out + dst) = pack<T>(ya);
+                *reinterpret_cast<uint4*>(k_out + dst + kPartner) = pack<T>(yc);
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; e += 2) {
+                    const float2 cs = __ldg(trig + slice0 + e / 2);
+                    rotate_pair(a[e], a[e + 1], cs.x, cs.y, ya[e], ya[e + 1]);
+                }
+                *reinterpret_cast<uint4*>(k_out + dst) = pack<T>(ya);
+            }
         }
     }
 }
@@ -221,8 +223,8 @@ static int launch_assemble_typed(const cf_geom* g, const cf_batch* b, const Plan
                                  long long layer_stride, long long self_stride, int out_rows, const void* k_in,
                                  const void* v_in, const void* k_self, const void* v_self, void* k_out, void* v_out,
                                  int* final_rows, cudaStream_t stream) {
-    const int tiles = tiles_per_request_bound(b);
-    if (n_layers > 65535 || b->n_requests > 65535 || tiles >= (1 << 30)) return CF_ERR_INVALID_ARG;
+    const int tiles = std::min(tiles_per_request_bound(b), 1 << 16);
+    if (n_layers > 65535 || b->n_requests > 65535) return CF_ERR_INVALID_ARG;
     dim3 grid((unsigned)tiles + 1, (unsigned)n_layers, (unsigned)b->n_requests);
     BatchView bv = make_batch_view(b);
     auto args = [&](auto kernel) {

@@ -13,7 +13,6 @@ namespace cf {
 // cudaGetSymbolAddress (static_scratch_address below).
 static __device__ __align__(256) unsigned char g_static_scratch[CF_STATIC_WORKSPACE_BYTES];
 
-constexpr int kMaxDevices = 64;
 static std::mutex g_static_mutex;
 static void* g_static_address[kMaxDevices] = {};
 

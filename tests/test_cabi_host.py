@@ -21,7 +21,8 @@ def lib():
 
 
 def test_every_declared_symbol_is_exported(lib):
-    header = open(os.path.join(ROOT, "include", "cachefocus.h")).read()
+    header = "".join(open(os.path.join(ROOT, "include", name)).read()
+                     for name in sorted(os.listdir(os.path.join(ROOT, "include"))) if name.endswith(".h"))
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     declared = set(re.findall(r"\b(cf_[a-z_0-9]+)\s*\(", header))
     assert declared == set(cf.EXPORTS), declared ^ set(cf.EXPORTS)
@@ -102,3 +103,67 @@ def test_workspace_size_of_layer_batched_calls(lib):
     assert cf.cf_attn_workspace_bytes_full(geom, batch, 0) == 0
     assert cf.cf_attn_workspace_bytes_layers(geom, batch, 0) == 0
     assert cf.cf_attn_workspace_bytes_layers(geom, batch, cf.CF_MAX_LAYERS_PER_CALL + 1) == 0
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_host_pruning_step_matches_oracle(lib, seed):
+    """cf_prune_topk_host against the oracle's prune_topk: kept set and order bit-exact, ties included."""
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 80))
+    n_kept = int(rng.integers(1, n + 1))
+    order = [int(i) for i in rng.permutation(n)[:n_kept]]
+    # scores drawn from a handful of float32 values so that ties are common
+    scores = rng.choice(np.array([0.0, 0.125, 0.25, 0.3, 0.7, 1.5], dtype=np.float32), size=n).astype(np.float32)
+    if seed % 3 == 0:
+        scores = rng.random(n).astype(np.float32)
+    for strategy in (oracle.ALLOC_NONE, oracle.ALLOC_ALIGN, oracle.ALLOC_SORT):
+        for keep in (0, 1, n_kept // 2, n_kept, n_kept + 3):
+            want = oracle.prune_topk(scores, order, keep, strategy)
+            assert cf.cf_prune_topk_host(scores, order, keep, strategy) == want
+
+
+def test_host_pruning_step_rejects_bad_input(lib):
+    for bad in ([0, 0], [3], [-1]):
+        with pytest.raises(cf.CacheFocusError) as e:
+            cf.cf_prune_topk_host([0.1, 0.2, 0.3], bad, 1, oracle.ALLOC_ALIGN)
+        assert e.value.code == cf.CF_ERR_INVALID_ARG
+    with pytest.raises(cf.CacheFocusError):
+        cf.cf_prune_topk_host([0.1, 0.2], [0, 1], 1, 7)
+    assert cf.cf_prune_topk_host([], [], 3, oracle.ALLOC_SORT) == []
+
+
+def test_stack_driver_checks_its_arguments_on_the_host(lib):
+    """cf_run_stack and its workspace query through ctypes; every case returns before anything is launched
+    (the device pointers of the descriptors are never dereferenced)."""
+    geom = cf.make_geom(12, 2, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256
+    batch = cf.cf_batch(1, 50, 48, 0, 48, 0, 0, 0, 8000, 2 * 128, fake, fake, fake)
+
+    def stack(layers, keeps, n_layers=28, strategy=cf.CF_ALLOC_ALIGN, batch_layers=1, q=fake):
+        la, ke = np.asarray(layers, np.int32), np.asarray(keeps, np.int32)
+        st = cf.cf_stack(n_layers, len(la), la.ctypes.data if len(la) else None, ke.ctypes.data if len(ke) else None,
+                         strategy, batch_layers, 0.0, 0, q, 1 << 20, fake, fake, 1 << 22, None, None, 0, fake, 1 << 20,
+                         None, None, fake, None, None, None)
+        return st, (la, ke)
+
+    good, keep = stack([4, 12, 20], [25, 12, 6])
+    per_call = [cf.cf_attn_workspace_bytes_layers(geom, batch, m) for m in (4, 8)]
+    assert cf.cf_run_stack_workspace_bytes(geom, batch, good) == max(per_call) > 0
+    one_by_one, keep2 = stack([4, 12, 20], [25, 12, 6], batch_layers=0)
+    assert cf.cf_run_stack_workspace_bytes(geom, batch, one_by_one) == cf.cf_attn_workspace_bytes(geom, batch)
+    # document lengths on the host let the call shrink its grids to the documents still kept
+    lens = np.full(50, 160, np.int32)
+    begin = np.array([0, 50], np.int32)
+    hinted, keep3 = stack([4, 12, 20], [25, 12, 6])
+    hinted.doc_len_host, hinted.req_doc_begin_host = lens.ctypes.data, begin.ctypes.data
+    assert 0 < cf.cf_run_stack_workspace_bytes(geom, batch, hinted) <= max(per_call)
+    for st, _ in (stack([4, 4], [25, 12]), stack([12, 4], [25, 12]), stack([0], [5]), stack([4], [-1]),
+                  stack([4], [5], n_layers=0), stack([4], [5], strategy=9)):
+        assert cf.cf_run_stack_workspace_bytes(geom, batch, st) == 0
+        rc = lib.cf_run_stack(ctypes.byref(geom), ctypes.byref(batch), ctypes.byref(st), fake, 1 << 20, fake, 1 << 20, None)
+        assert rc == cf.CF_ERR_INVALID_ARG
+    null_q, _ = stack([4], [5], q=None)
+    assert lib.cf_run_stack(ctypes.byref(geom), ctypes.byref(batch), ctypes.byref(null_q), fake, 1 << 20, fake,
+                            1 << 20, None) == cf.CF_ERR_INVALID_ARG
+    assert lib.cf_debug_wait_timeout(ctypes.byref(geom), ctypes.byref(batch), fake, 0, None) == cf.CF_ERR_INVALID_ARG
+    assert lib.cf_debug_wait_timeout(ctypes.byref(geom), ctypes.byref(batch), fake + 8, 1000, None) == cf.CF_ERR_WORKSPACE
