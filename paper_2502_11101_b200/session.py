@@ -141,7 +141,7 @@ class Session:
             B.cf_run_stack(self.geom, self.batch, st, self.plan, self.workspace)
             del keepalive
             return
-        assert driver == "calls" and softmax_scale == 0.0
+        assert driver == "calls"
         sched = dict(schedule)
         n_layers = q.shape[0]
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))
@@ -153,7 +153,7 @@ class Session:
                 for lo in range(first, last, B.CF_MAX_LAYERS_PER_CALL):
                     hi = min(last, lo + B.CF_MAX_LAYERS_PER_CALL)
                     self.attend_layers(q[lo:hi], k[lo:hi], v[lo:hi], out[lo:hi], None if lse is None else lse[lo:hi],
-                                       None if layer_scores is None else layer_scores[lo:hi],
+                                       None if layer_scores is None else layer_scores[lo:hi], softmax_scale,
                                        k_self=None if k_self is None else k_self[lo:hi],
                                        v_self=None if v_self is None else v_self[lo:hi])
                 if last in sched:
@@ -163,13 +163,13 @@ class Session:
             for layer in range(1, n_layers + 1):
                 i = layer - 1
                 if k_self is None:
-                    self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i])
+                    self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i], softmax_scale)
                     if layer_scores is not None:
                         layer_scores[i].copy_(self.doc_scores)
                 else:
                     self.attend_layers(q[i:i + 1], k[i:i + 1], v[i:i + 1], out[i:i + 1],
                                        None if lse is None else lse[i:i + 1],
-                                       None if layer_scores is None else layer_scores[i:i + 1],
+                                       None if layer_scores is None else layer_scores[i:i + 1], softmax_scale,
                                        k_self=k_self[i:i + 1], v_self=v_self[i:i + 1])
                 if layer in sched:
                     self.prune(sched[layer], strategy)

@@ -40,7 +40,8 @@ def rotated_key_tolerance(want: np.ndarray, dtype: str, interleaved: bool = Fals
 
 
 def oracle_stack(meta: W.WorkloadMeta, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, strategy: int,
-                 schedule=None, final_reposition: bool = True, n_reuse: int = 0) -> List[Dict]:
+                 schedule=None, final_reposition: bool = True, n_reuse: int = 0, scale: Optional[float] = None
+                 ) -> List[Dict]:
     cfg = meta.cfg
     qd, kd, vd = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
     res = []
@@ -50,7 +51,7 @@ def oracle_stack(meta: W.WorkloadMeta, q: torch.Tensor, k: torch.Tensor, v: torc
                                     meta.doc_src_start[lo:hi], cfg.rope_theta, cfg.pos_range,
                                     cfg.schedule if schedule is None else schedule, strategy,
                                     tail_reserve=cfg.q_len, n_reuse=n_reuse, doc_base=lo,
-                                    final_reposition=final_reposition))
+                                    final_reposition=final_reposition, scale=scale))
     return res
 
 
@@ -72,35 +73,64 @@ def cut_margins(meta: W.WorkloadMeta, ref: List[Dict], strategy: int, schedule=N
 
 
 def add_self_block(meta: W.WorkloadMeta, ref: List[Dict], q: torch.Tensor, k_self: torch.Tensor,
-                   v_self: torch.Tensor) -> None:
+                   v_self: torch.Tensor, scale: Optional[float] = None) -> None:
     """Replace every layer's output and log-sum-exp of the oracle run by the merge with the causal
     query-self block (document scores are defined on the documents alone and stay)."""
     qd, ks, vs = q.double().cpu().numpy(), k_self.double().cpu().numpy(), v_self.double().cpu().numpy()
     for b in range(meta.cfg.batch):
         for l, rec in enumerate(ref[b]["layers"]):
-            o_self, lse_self = oracle.query_self_block(qd[l, b], ks[l, b], vs[l, b])
+            o_self, lse_self = oracle.query_self_block(qd[l, b], ks[l, b], vs[l, b], scale)
             rec["out"], rec["lse"] = oracle.merge_softmax_blocks(rec["out"], rec["lse"], o_self, lse_self)
 
 
+PAD_SENTINEL = 12288.0                   # exact in bf16 and fp32: fills the padding of a padded store
+
+
+def padded_store(t: torch.Tensor, token_stride: int, device) -> torch.Tensor:
+    """`t` [L, T, Hkv, D] on `device` as a view into a store whose rows are `token_stride` elements
+    apart; the padding behind every row holds PAD_SENTINEL."""
+    n_layers, total, hkv, d = t.shape
+    base = torch.full((n_layers, total, token_stride), PAD_SENTINEL, dtype=t.dtype, device=device)
+    view = base[:, :, :hkv * d].view(n_layers, total, hkv, d)
+    view.copy_(t)
+    return view
+
+
+def padding_of(view: torch.Tensor, token_stride: int) -> torch.Tensor:
+    """The padding columns of a store made by padded_store."""
+    n_layers, total, hkv, d = view.shape
+    base = torch.as_strided(view, (n_layers, total, token_stride), (total * token_stride, token_stride, 1))
+    return base[:, :, hkv * d:]
+
+
 def gpu_stack(meta: W.WorkloadMeta, q, k, v, strategy: int, schedule=None, device="cuda:0", n_reuse: int = 0,
-              with_final: bool = True, batch_layers: bool = False, k_self=None, v_self=None):
+              with_final: bool = True, batch_layers: bool = False, k_self=None, v_self=None,
+              driver: str = "library", softmax_scale: float = 0.0, token_stride: Optional[int] = None):
     from paper_2502_11101_b200.session import Session
     cfg = meta.cfg
     sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
                    cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len,
-                   n_reuse=n_reuse, device=device)
-    qg, kg, vg = q.to(device), k.to(device), v.to(device)
+                   n_reuse=n_reuse, token_stride=token_stride, device=device)
+    qg = q.to(device)
+    if token_stride is None:
+        kg, vg = k.to(device), v.to(device)
+        k_final = kg.clone() if with_final else None
+    else:
+        kg, vg = padded_store(k, token_stride, device), padded_store(v, token_stride, device)
+        k_final = padded_store(k, token_stride, device) if with_final else None
     n_layers = q.shape[0]
     out = torch.full_like(qg, float("nan"))
     lse = torch.full((n_layers, cfg.batch, cfg.n_q_heads, cfg.q_len), float("nan"), device=device)
     scores = torch.full((n_layers, meta.n_docs_total), float("nan"), device=device)
-    k_final = kg.clone() if with_final else None
     sched = cfg.schedule if schedule is None else schedule
     sess.run_stack(qg, kg, vg, sched, strategy, out, lse, k_final, scores, batch_layers=batch_layers,
                    k_self=None if k_self is None else k_self.to(device),
-                   v_self=None if v_self is None else v_self.to(device))
+                   v_self=None if v_self is None else v_self.to(device), driver=driver, softmax_scale=softmax_scale)
     torch.cuda.synchronize()
     status = sess.status()
+    if token_stride is not None:                            # nothing may be written between the rows
+        for t in (kg, vg) + ((k_final,) if with_final else ()):
+            assert bool(torch.all(padding_of(t, token_stride) == PAD_SENTINEL)), "padding of the store was written"
     return {"out": out.float().cpu().numpy(), "lse": lse.cpu().numpy(), "scores": scores.cpu().numpy(),
             "accum": sess.score_accum.cpu().numpy(), "plan": sess.read_plan(), "status": status,
             "k_final": None if k_final is None else k_final.float().cpu().numpy(), "session": sess}
@@ -170,19 +200,22 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
 
 def run_and_compare(cfg: W.WorkloadConfig, seed: int, strategy: int, device="cuda:0", n_reuse: int = 0,
                     min_margin: float = 2e-3, doc_len_override=None, batch_layers: bool = False,
-                    self_block: bool = False) -> Dict[str, float]:
+                    self_block: bool = False, driver: str = "library", softmax_scale: float = 0.0,
+                    token_stride: Optional[int] = None) -> Dict[str, float]:
     meta = W.make_meta(cfg, seed, doc_len_override)
     q = W.make_q(meta)
     k, v = W.make_kv(meta)
-    ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse)
+    scale = softmax_scale if softmax_scale else None
+    ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse, scale=scale)
     margin = cut_margins(meta, ref, strategy)
     assert margin >= min_margin, f"workload rejected: decisive score gap {margin:.2e} below {min_margin:.0e}"
     k_self = v_self = None
     if self_block:
         k_self, v_self = W.make_kv_self(meta)
-        add_self_block(meta, ref, q, k_self, v_self)
+        add_self_block(meta, ref, q, k_self, v_self, scale)
     got = gpu_stack(meta, q, k, v, strategy, device=device, n_reuse=n_reuse, batch_layers=batch_layers,
-                    k_self=k_self, v_self=v_self)
+                    k_self=k_self, v_self=v_self, driver=driver, softmax_scale=softmax_scale,
+                    token_stride=token_stride)
     report = compare(meta, ref, got, k)
     report["margin"] = margin
     return report

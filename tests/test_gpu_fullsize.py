@@ -96,3 +96,82 @@ def test_config5_four_layers_full_batch_sampled(batch_layers):
     cfg = W.scaled_config(W.CONFIGS[5], n_layers=4, schedule=schedule)
     plan0 = _run_full(cfg, samples=[(0, 0), (5, 17), (7, 31)], batch_layers=batch_layers)
     assert all(int(x) == 6 for x in plan0["n_reuse"])
+
+
+def _run_against_whole_oracle(cfg, sample_heads):
+    """The stack issued call by call (one attention call per layer) with the plan read back after
+    every pruning step, against oracle.run_stack request by request: kept set, order, positions and
+    windows bit-exact after every cut; every layer's document scores and log-sum-exp of the sampled
+    heads, and their outputs, within tolerance."""
+    meta = W.make_meta(cfg, 0)
+    dev = "cuda:0"
+    q = W.make_q(meta, dev)
+    k, v = W.make_kv(meta, dev)
+    # the oracle's inputs: the same seeded tensors, widened exactly (bf16 -> fp32) and upcast per layer inside
+    q_h, k_h, v_h = q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy()
+    ref = []
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        ref.append(oracle.run_stack(q_h[:, b], k_h, v_h, meta.doc_len[lo:hi], meta.doc_offsets, meta.doc_src_start[lo:hi],
+                                    cfg.rope_theta, cfg.pos_range, cfg.schedule, oracle.ALLOC_ALIGN,
+                                    tail_reserve=cfg.q_len, doc_base=lo, final_reposition=False))
+    from tests import harness
+    assert harness.cut_margins(meta, ref, oracle.ALLOC_ALIGN) >= 5e-4
+    sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                   cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len, device=dev)
+    sess.set_live_docs(cfg.n_docs)
+    sess.init()
+    sched = dict(cfg.schedule)
+    out = torch.empty_like(q[0])
+    lse = torch.empty((cfg.batch, cfg.n_q_heads, cfg.q_len), device=dev)
+    for layer in range(1, cfg.n_layers + 1):
+        sess.attend(q[layer - 1], k[layer - 1], v[layer - 1], out, lse)
+        s_got = sess.doc_scores.cpu().numpy()
+        o_got, l_got = out.float().cpu().numpy(), lse.cpu().numpy()
+        for b in range(cfg.batch):
+            lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+            rec = ref[b]["layers"][layer - 1]
+            n_kept = len(rec["order_in"])
+            s_err = np.abs(s_got[lo:hi] - rec["doc_scores"])
+            assert np.all(s_err <= 1e-2 / n_kept + 2e-2 * np.abs(rec["doc_scores"])), (layer, b)
+            assert set(np.nonzero(s_got[lo:hi])[0]) == set(rec["order_in"]), (layer, b)
+            for h in sample_heads:
+                assert np.all(np.abs(o_got[b, :, h] - rec["out"][:, h]) <= 1e-2 + 2e-2 * np.abs(rec["out"][:, h])), (layer, b, h)
+                assert np.all(np.abs(l_got[b, h] - rec["lse"][h]) <= 1e-2), (layer, b, h)
+        if layer in sched:
+            sess.prune(sched[layer], oracle.ALLOC_ALIGN)
+            plan = sess.read_plan()
+            for b in range(cfg.batch):
+                lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+                rec = ref[b]["layers"][layer - 1]
+                assert plan["order"][b] == rec["order_out"], (layer, b)
+                if layer < cfg.n_layers:
+                    nxt = ref[b]["layers"][layer]
+                    assert np.array_equal(plan["dst_start"][lo:hi], nxt["dst_start"]), (layer, b)
+                    assert int(plan["n_reuse"][b]) == nxt["n_reuse"], (layer, b)
+    assert sess.status() == 0
+    plan = sess.read_plan()
+    for b in range(cfg.batch):
+        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+        assert plan["order"][b] == ref[b]["order"]
+        assert np.array_equal(plan["dst_start"][lo:hi], ref[b]["dst_start"])
+        assert np.array_equal(plan["group"][lo:hi], ref[b]["group"])
+        assert np.all(np.abs(sess.score_accum.cpu().numpy()[lo:hi] - ref[b]["score_accum"])
+                      <= 1e-2 + 2e-2 * np.abs(ref[b]["score_accum"]))
+
+
+def test_config4_full_size_every_cut_against_the_oracle():
+    _run_against_whole_oracle(W.CONFIGS[4], sample_heads=(0, 13, 27))
+
+
+def test_config5_four_layers_every_cut_against_the_oracle():
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=4, schedule=((1, 60), (2, 30), (3, 15)))
+    _run_against_whole_oracle(cfg, sample_heads=(0, 17, 31))
+
+
+def test_config5_sixteen_layers_full_batch_sampled():
+    # half of the 32-layer stack: 45 GB of keys and values resident, the schedule's first two cuts at
+    # their own layers (4 and 12); the 32-layer store (90.6 GB plus the final keys) is not run
+    cfg = W.scaled_config(W.CONFIGS[5], n_layers=16, schedule=((4, 60), (12, 30)))
+    plan0 = _run_full(cfg, samples=[(0, 0), (3, 9), (7, 31)], batch_layers=True)
+    assert all(int(x) == 6 for x in plan0["n_reuse"])

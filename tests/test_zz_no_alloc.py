@@ -4,6 +4,7 @@ that stops at the first failure has then already seen every other test."""
 import pytest
 import torch
 
+import oracle
 import paper_2502_11101_b200 as cf
 from paper_2502_11101_b200 import workloads as W
 from paper_2502_11101_b200.session import Session
@@ -46,6 +47,17 @@ def test_static_scratch_entry_point_matches_the_ordinary_one():
         assert torch.all((got_s - want_s).abs() <= 1e-2 / cfg.n_docs + 2e-2 * want_s.abs())
         assert torch.all((got_acc - want_acc).abs() <= 1e-2 / cfg.n_docs + 2e-2 * want_acc.abs())
         assert abs(float(got_s.sum()) - 1.0) < 1e-3
+        # and against the oracle itself, on the same seeded inputs
+        kd = k[layer].double().cpu().numpy()
+        dst, _, _, _ = oracle.allocate_positions(meta.doc_len, range(cfg.n_docs), cfg.pos_range, 0, cfg.q_len)
+        k_rot = oracle.reposition_keys(kd, meta.doc_offsets, meta.doc_src_start, dst, range(cfg.n_docs), cfg.rope_theta)
+        o_ref, lse_ref, _, s_ref = oracle.query_prefill_attn(q[layer, 0].double().cpu().numpy(), k_rot,
+                                                             v[layer].double().cpu().numpy(), meta.doc_offsets,
+                                                             range(cfg.n_docs), cfg.n_docs)
+        o_got = got_out[0].float().cpu().numpy()
+        assert (abs(o_got - o_ref) <= 1e-2 + 2e-2 * abs(o_ref)).all()
+        assert (abs(got_lse[0].cpu().numpy() - lse_ref) <= 1e-2).all()
+        assert (abs(got_s.cpu().numpy() - s_ref) <= 1e-2 / cfg.n_docs + 2e-2 * abs(s_ref)).all()
 
 
 def test_static_scratch_entry_point_refuses_batches_that_do_not_fit():
