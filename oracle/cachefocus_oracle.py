@@ -18,13 +18,17 @@ What it follows, step by step:
   "document-wise" (footnote of Sec. 2.4);
 * Layer-Adaptive Cache Pruning: scores accumulate over layers, every pruning layer keeps
   the best documents and the survivors are re-allocated ("align" / "sort", Sec. 2.5)
-  (Algorithm 2, Phases 1 and 2); the linear pruning schedule of App. C.
+  (Algorithm 2, Phases 1 and 2); the linear pruning schedule of App. C;
+* the attention of the offline cache construction (Sec. 2.2): every document attends the shared
+  prefix cache and itself, causally, independently of the other documents.
 
 Pins (tests/test_oracle_*.py): closed forms of the rotation group, the identity of
 Eq. 5, an independent complex-number statement of rotary encoding, the printed examples
 of Sec. 3.3 (k=20, N_reuse=k/5) and App. C (L=28, n=4, k=40, k_finish=5), allocation
 invariants checked by brute force, brute-force attention with Python loops, the
-N_reuse=1 special case against a library attention routine, the closed form for Q=0.
+N_reuse=1 special case against a library attention routine, the closed form for Q=0; for the
+cache-construction attention a library causal attention over [prefix; document], Python loops, the
+Q=0 closed form, causality and the composition of the pinned prefix and self blocks.
 
 Parity unpinned (conventions the paper leaves open, no figure or code to compare with):
 which two coordinates form a slice (both common layouts are implemented), round-robin
@@ -243,6 +247,46 @@ def merge_softmax_blocks(out_a: np.ndarray, lse_a: np.ndarray, out_b: np.ndarray
     wa = np.exp(lse_a - lse).T[:, :, None]
     wb = np.exp(lse_b - lse).T[:, :, None]
     return wa * out_a + wb * out_b, lse
+
+
+def document_prefill_attn(q_doc: np.ndarray, k_doc: np.ndarray, v_doc: np.ndarray,
+                           k_prefix: Optional[np.ndarray] = None, v_prefix: Optional[np.ndarray] = None,
+                           scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """The attention inside the offline cache construction C_d <- LLM(C_prefix, d) of Sec. 2.2 (the two
+    unnumbered equations there; O(l_c^2 k) in the complexity paragraph of Sec. 3.3), one layer, one
+    document: token t of the document attends the shared prefix cache and the document's own tokens
+    0..t under the causal mask of Eq. 1; other documents are invisible (documents are cached in
+    parallel, independently of each other and of any query).
+
+    q_doc[len, Hq, D]; k_doc, v_doc[len, Hkv, D]; k_prefix, v_prefix[P, Hkv, D] or None (P = 0).
+    Queries and keys are taken as already rotary-encoded (prefix at 0..P-1, the document right behind
+    it).  Returns out[len, Hq, D] and lse[Hq, len]."""
+    q_doc = np.asarray(q_doc, dtype=np.float64)
+    k_doc = np.asarray(k_doc, dtype=np.float64)
+    v_doc = np.asarray(v_doc, dtype=np.float64)
+    n, hq, d = q_doc.shape
+    hkv = k_doc.shape[1]
+    g = hq // hkv
+    if k_prefix is None or len(k_prefix) == 0:
+        k_prefix = np.zeros((0, hkv, d))
+        v_prefix = np.zeros((0, hkv, d))
+    k_all = np.concatenate([np.asarray(k_prefix, dtype=np.float64), k_doc])
+    v_all = np.concatenate([np.asarray(v_prefix, dtype=np.float64), v_doc])
+    p_len = k_all.shape[0] - n
+    if scale is None or scale == 0.0:
+        scale = 1.0 / math.sqrt(d)
+    out = np.zeros((n, hq, d))
+    lse = np.zeros((hq, n))
+    for h in range(hq):
+        kvh = h // g
+        for t in range(n):
+            vis = p_len + t + 1                               # the prefix, then document tokens 0..t
+            s = (k_all[:vis, kvh, :] @ q_doc[t, h, :]) * scale
+            m = s.max()
+            e = np.exp(s - m)
+            out[t, h, :] = (e / e.sum()) @ v_all[:vis, kvh, :]
+            lse[h, t] = m + math.log(e.sum())
+    return out, lse
 
 
 def assemble_final_cache(k_rot: np.ndarray, v_store: np.ndarray, doc_offsets: Sequence[int],
