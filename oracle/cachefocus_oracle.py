@@ -84,6 +84,14 @@ def rope_rotate(x: np.ndarray, delta, theta: float, layout: int = ROPE_HALF) -> 
     return y
 
 
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Values of `x` rounded to the nearest bfloat16 (8 significand bits, ties to even), returned
+    as float64: the storage format of a 16-bit cache, written out from its definition."""
+    bits = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return bits.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
 # ------------------------------------------------------------------------- allocation
 def n_reuse_eq6(n_kept: int, capacity: int, cache_len: int) -> int:
     """Eq. 6: ceil(k / (L / l_C)).  L / l_C, the number of caches that fit without
@@ -342,8 +350,8 @@ def run_stack(q_layers: np.ndarray, k_store: np.ndarray, v_store: np.ndarray,
               theta: float, pos_range: int, schedule: Sequence[Tuple[int, int]], strategy: int,
               tail_reserve: int, prefix_len: int = 0, n_reuse: int = 0,
               order0: Optional[Sequence[int]] = None, layout: int = ROPE_HALF,
-              scale: Optional[float] = None, doc_base: int = 0, final_reposition: bool = True
-              ) -> Dict[str, object]:
+              scale: Optional[float] = None, doc_base: int = 0, final_reposition: bool = True,
+              key_round=None) -> Dict[str, object]:
     """Algorithm 2 for one request.  `q_layers[L, Lq, Hq, D]` holds each layer's query
     states (the projections and feed-forward blocks that would produce them are outside
     this path); `k_store`, `v_store[L, T, Hkv, D]`; `doc_len`, `doc_src_start` are the
@@ -351,7 +359,11 @@ def run_stack(q_layers: np.ndarray, k_store: np.ndarray, v_store: np.ndarray,
 
     Per layer l = 1..L: re-position the kept caches, attend, S += s^l; after a layer
     named in `schedule` keep the top documents and re-allocate them (same query start).
-    Phase 2 re-positions the final survivors in every layer."""
+    Phase 2 re-positions the final survivors in every layer.
+
+    `key_round`, if given, is applied to the re-positioned keys before a layer attends them: the
+    re-positioned cache of Eq. 5 is again a cache and may be held in the cache's storage type (a
+    rounding function such as round_to_bf16); by default the keys stay exact."""
     n_layers = q_layers.shape[0]
     n_docs = len(doc_len)
     order = list(range(n_docs)) if order0 is None else [int(i) for i in order0]
@@ -363,6 +375,8 @@ def run_stack(q_layers: np.ndarray, k_store: np.ndarray, v_store: np.ndarray,
     layers = []
     for l in range(1, n_layers + 1):
         k_rot = reposition_keys(k_store[l - 1], local_off, doc_src_start, dst, order, theta, layout)
+        if key_round is not None:
+            k_rot = key_round(k_rot)
         out, lse, mass, scores = query_prefill_attn(q_layers[l - 1], k_rot, v_store[l - 1],
                                                     local_off, order, n_docs, scale)
         accum = accum + scores

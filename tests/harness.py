@@ -40,8 +40,9 @@ def rotated_key_tolerance(want: np.ndarray, dtype: str, interleaved: bool = Fals
 
 
 def oracle_stack(meta: W.WorkloadMeta, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, strategy: int,
-                 schedule=None, final_reposition: bool = True, n_reuse: int = 0, scale: Optional[float] = None
-                 ) -> List[Dict]:
+                 schedule=None, final_reposition: bool = True, n_reuse: int = 0, scale: Optional[float] = None,
+                 key_round=None) -> List[Dict]:
+    """`key_round` (e.g. oracle.round_to_bf16): the layers attend re-positioned keys held in the store's type."""
     cfg = meta.cfg
     qd, kd, vd = q.double().cpu().numpy(), k.double().cpu().numpy(), v.double().cpu().numpy()
     res = []
@@ -51,7 +52,7 @@ def oracle_stack(meta: W.WorkloadMeta, q: torch.Tensor, k: torch.Tensor, v: torc
                                     meta.doc_src_start[lo:hi], cfg.rope_theta, cfg.pos_range,
                                     cfg.schedule if schedule is None else schedule, strategy,
                                     tail_reserve=cfg.q_len, n_reuse=n_reuse, doc_base=lo,
-                                    final_reposition=final_reposition, scale=scale))
+                                    final_reposition=final_reposition, scale=scale, key_round=key_round))
     return res
 
 
@@ -201,12 +202,12 @@ def compare(meta: W.WorkloadMeta, ref: List[Dict], got: Dict, k_store: torch.Ten
 def run_and_compare(cfg: W.WorkloadConfig, seed: int, strategy: int, device="cuda:0", n_reuse: int = 0,
                     min_margin: float = 2e-3, doc_len_override=None, batch_layers: bool = False,
                     self_block: bool = False, driver: str = "library", softmax_scale: float = 0.0,
-                    token_stride: Optional[int] = None) -> Dict[str, float]:
+                    token_stride: Optional[int] = None, key_round=None) -> Dict[str, float]:
     meta = W.make_meta(cfg, seed, doc_len_override)
     q = W.make_q(meta)
     k, v = W.make_kv(meta)
     scale = softmax_scale if softmax_scale else None
-    ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse, scale=scale)
+    ref = oracle_stack(meta, q, k, v, strategy, n_reuse=n_reuse, scale=scale, key_round=key_round)
     margin = cut_margins(meta, ref, strategy)
     assert margin >= min_margin, f"workload rejected: decisive score gap {margin:.2e} below {min_margin:.0e}"
     k_self = v_self = None

@@ -136,3 +136,16 @@ def test_a_planted_sign_error_is_caught():
     wrong = oracle.rope_rotate(x, -np.arange(4.0) - 1.0, 1e4)      # what a sign slip would compute
     right = _complex_rope(x, np.arange(4.0) + 1.0, 1e4, ROPE_HALF)
     assert not np.allclose(wrong, right, atol=1e-3)
+
+
+def test_round_to_bf16_matches_the_format_definition():
+    """Against a library conversion, and on hand-picked ties: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    (ties to even: down), 1 + 3 * 2^-8 halfway between 1 + 2^-7 and 1 + 2^-6 (up)."""
+    import torch
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096), [0.0, -0.0, 1.0, -3.5]])
+    want = torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(oracle.round_to_bf16(x), want)
+    assert oracle.round_to_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert oracle.round_to_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+    assert oracle.round_to_bf16(np.array([1.0 + 2.0 ** -8 + 2.0 ** -20]))[0] == 1.0 + 2.0 ** -7
