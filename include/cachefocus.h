@@ -306,6 +306,44 @@ int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
                   const float* score_accum, int32_t keep, const int32_t* keep_per_request,
                   int32_t strategy, void* stream);
 
+/* A batch of documents for the offline cache construction: a packed store like cf_batch's, without
+ * requests, allocation or plan.  doc_offsets is DEVICE memory owned by the caller. */
+typedef struct cf_doc_batch {
+    int32_t n_docs;
+    int32_t max_doc_len;      /* upper bound of the documents' token counts (sizes the grid; a document
+                                 longer than this is only partly processed)                           */
+    int32_t prefix_len;       /* tokens of the shared prefix cache, 0 = none                          */
+    int32_t reserved;
+    int64_t total_tokens;     /* rows of one layer of the packed tensors                              */
+    int64_t token_stride;     /* elements between consecutive key/value rows, >= n_kv_heads*head_dim  */
+    const int32_t* doc_offsets;   /* device [n_docs+1]: document i owns rows doc_offsets[i] .. [i+1]-1 */
+} cf_doc_batch;
+
+/* Attention of the offline, query-independent cache construction C_d <- LLM(C_prefix, d) (Sec. 2.2;
+ * the O(l_c^2 k) term of the complexity paragraph in Sec. 3.3): in every layer, token t of a document
+ * attends the shared prefix cache and the document's own tokens 0..t (causal mask of Eq. 1); documents
+ * are processed in parallel and do not see each other.  Queries and keys are used as given: the
+ * caller has already rotary-encoded them (prefix at positions 0..prefix_len-1, every document right
+ * behind it), so no re-positioning happens here; the keys and values passed in ARE the document
+ * caches that the query-time calls above later consume.
+ *   q, out          device [n_layers][total_tokens][n_q_heads][head_dim], layers q_layer_stride /
+ *                   out_layer_stride elements apart
+ *   k, v            device [n_layers][total_tokens][n_kv_heads][head_dim] with docs->token_stride
+ *                   between rows, layers kv_layer_stride elements apart
+ *   k_prefix, v_prefix  device [n_layers][prefix_len][n_kv_heads][head_dim] dense, layers
+ *                   prefix_layer_stride elements apart; ignored when prefix_len = 0
+ *   softmax_scale   0 selects 1/sqrt(head_dim)
+ *   lse             device float [n_layers][n_q_heads][total_tokens], natural log of each row's softmax
+ *                   denominator; may be NULL
+ *   status          device int32 or NULL: receives CF_ERR_TIMEOUT if a bounded device-side wait of the
+ *                   tensor-core kernel expired (it is only ever written on failure: clear it first)
+ * Needs no workspace.  Errors: CF_ERR_INVALID_ARG (null or misaligned pointers, strides). */
+int cf_document_prefill_attn(const cf_geom* geom, const cf_doc_batch* docs, int32_t n_layers,
+                             const void* q, int64_t q_layer_stride, const void* k, const void* v,
+                             int64_t kv_layer_stride, const void* k_prefix, const void* v_prefix,
+                             int64_t prefix_layer_stride, float softmax_scale, void* out,
+                             int64_t out_layer_stride, float* lse, int32_t* status, void* stream);
+
 /* Host-side mirror of the pruning step alone (Algorithm 2: argsort of S, prun), integers and scores
  * in host memory, nothing launched: among the documents of `order` (n_kept distinct local ids, rank
  * order) keeps the min(keep, n_kept) with the largest score_accum[id] (ties: lower id) and writes

@@ -26,7 +26,7 @@ EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
            "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn",
            "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
-           "cf_run_stack", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
+           "cf_run_stack", "cf_document_prefill_attn", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
 _SIZE_T_EXPORTS = ("cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers", "cf_attn_workspace_bytes_full",
                    "cf_run_stack_workspace_bytes")
 
@@ -51,6 +51,12 @@ class cf_plan_layout(ctypes.Structure):
                 ("total_bytes", "status", "kept", "kept_count", "dst_start", "group", "n_reuse", "query_start",
                  "n_tiles", "tile_begin", "doc_tile_begin", "doc_tile_count", "tile_doc", "tile_row0", "tile_len", "trig")] + \
                [("max_tiles", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class cf_doc_batch(ctypes.Structure):
+    _fields_ = [("n_docs", ctypes.c_int32), ("max_doc_len", ctypes.c_int32), ("prefix_len", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("total_tokens", ctypes.c_int64), ("token_stride", ctypes.c_int64),
+                ("doc_offsets", ctypes.c_void_p)]
 
 
 class cf_stack(ctypes.Structure):
@@ -117,6 +123,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_run_stack_workspace_bytes.argtypes = [gp, bp, sp]
     lib.cf_run_stack.argtypes = [gp, bp, sp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
     lib.cf_debug_wait_timeout.argtypes = [gp, bp, vp, i64, vp]
+    lib.cf_document_prefill_attn.argtypes = [gp, ctypes.POINTER(cf_doc_batch), i32, vp, i64, vp, vp, i64, vp, vp, i64,
+                                             ctypes.c_float, vp, i64, vp, vp, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
     lib.cf_profile_end.argtypes = [vp, i32, vp]
@@ -393,6 +401,32 @@ def cf_run_stack(geom: cf_geom, batch: cf_batch, stack: cf_stack, plan: torch.Te
                                      plan.numel() * plan.element_size(), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_run_stack")
+
+
+def cf_document_prefill_attn(geom: cf_geom, doc_offsets: torch.Tensor, max_doc_len: int, q: torch.Tensor,
+                             k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                             k_prefix: Optional[torch.Tensor] = None, v_prefix: Optional[torch.Tensor] = None,
+                             lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                             token_stride: Optional[int] = None, status: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
+    """Attention of the offline cache construction.  q, out [L, T, Hq, D]; k, v [L, T, Hkv, D] (rows may be
+    padded to `token_stride`); k_prefix, v_prefix [L, P, Hkv, D] dense; lse [L, Hq, T]; doc_offsets int32
+    device [n_docs + 1].  Dimension 0 may be strided."""
+    n_layers, total = q.shape[0], q.shape[1]
+    assert doc_offsets.dtype == torch.int32 and doc_offsets.is_contiguous()
+    assert k.shape[0] == n_layers and v.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k.stride(0) == v.stride(0) and (lse is None or lse.is_contiguous())
+    prefix_len = 0 if k_prefix is None else k_prefix.shape[1]
+    if prefix_len:
+        assert k_prefix.stride(0) == v_prefix.stride(0)
+    stride = k.shape[2] * k.shape[3] if token_stride is None else token_stride
+    docs = cf_doc_batch(doc_offsets.numel() - 1, max_doc_len, prefix_len, 0, total, stride, doc_offsets.data_ptr())
+    rc = load_library().cf_document_prefill_attn(
+        ctypes.byref(geom), ctypes.byref(docs), n_layers, q.data_ptr(), q.stride(0), k.data_ptr(), v.data_ptr(),
+        k.stride(0), _ptr(k_prefix) if prefix_len else None, _ptr(v_prefix) if prefix_len else None,
+        k_prefix.stride(0) if prefix_len else 0, softmax_scale, out.data_ptr(), out.stride(0), _ptr(lse),
+        _ptr(status), _stream(stream))
+    _check(rc, "cf_document_prefill_attn")
 
 
 def cf_debug_wait_timeout(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, limit_cycles: int, stream=None) -> None:

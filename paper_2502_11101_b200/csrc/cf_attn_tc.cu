@@ -26,23 +26,17 @@
 // P (bf16) and the sums (fp32) keep their relative precision.
 // Every wait on an mbarrier is bounded; when a wait expires the CTA raises CF_ERR_TIMEOUT in the
 // plan's status word, all roles leave their loops, and the CTA frees its tensor memory and exits.
-#include <cuda.h>
-
 #include <algorithm>
-#include <mutex>
 
-#include "cf_common.cuh"
+#include "cf_tc_util.cuh"
 
 namespace cf {
 
 namespace {
 
+using namespace tc;
+
 constexpr int kThreads = 512;
-constexpr int kD = 128;
-constexpr int kHalfBytes = kTile * 128;            // one 64-column half of a 128-row tile, 128 B per row
-constexpr int kTileBytes = 2 * kHalfBytes;         // 32 KiB: a K tile, a V tile, a Q tile or a P tile
-constexpr int kBoxRows = 32;                       // TMA boxes are 32, 64, 96 or 128 rows high
-constexpr int kBoxBytes = kBoxRows * 128;
 
 // Tensor maps of the key store and of the value store, one per box height: a tile is fetched by
 // two bulk copies (one per 64-column half) whatever its length.
@@ -55,7 +49,6 @@ constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose d
 constexpr int kSmemBytes = kSmemTiles * kTileBytes + 1024 + 512 + kMetaTiles * 8;   // tiles, alignment slack, barriers, tile list
 constexpr int kMaxStages = 6;
 constexpr int kRotateThreads = 192;
-constexpr long long kWaitLimitCycles = 2000000000LL;      // about a second
 constexpr float kRescaleThreshold = 8.0f;          // log2 units: the reference maximum moves only
                                                    // when a tile exceeds it by more than 2^8
 
@@ -109,179 +102,6 @@ __device__ __forceinline__ int ring_mod(int x, bool six) { return six ? x % 6 : 
 __device__ __forceinline__ int ring_div(int x, bool six) { return six ? x / 6 : x / 5; }
 // Loads of one kind (keys or values) a stage has received before the one of tile `it`.
 __device__ __forceinline__ int ring_uses(int it, bool six) { return six ? it / 3 : it / 5; }
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          long long limit_cycles = kWaitLimitCycles) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > limit_cycles) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
-        : "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major; B K-major or MN-major.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
-}
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Same with the A operand (bf16, two elements per 32-bit column) in tensor memory.
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// 32 consecutive fp32 columns of this thread's TMEM lane; returns after the data has arrived.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-// Asynchronous 32-column load: the registers may only be used after tmem_ld_wait(v).
-__device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                 : "r"(taddr)
-                 : "memory");
-}
-// Waits for all outstanding tensor-memory loads of this thread; naming the registers keeps the
-// compiler from moving their uses above the wait.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
-    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31]) : : "memory");
-}
-// 16 columns, synchronous (used on the rare rescaling path).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};\n"
-        "tcgen05.wait::st.sync.aligned;"
-        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(taddr)
-        : "memory");
-}
-// 16 columns (32 packed bf16) of the P operand; completion is awaited once per tile.
-__device__ __forceinline__ void tmem_st16_async(uint32_t taddr, const uint32_t (&v)[32]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
-                 : : "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(taddr)
-                 : "memory");
-}
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-// Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128B-swizzled half tile.
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-    return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
-}
-
-// Maximum of the first `valid` of 32 logits (MASKED=false: all 32).
-template <bool MASKED>
-__device__ __forceinline__ float chunk_max(const uint32_t (&v)[32], int valid) {
-    float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-        m0 = fmaxf(m0, (!MASKED || i < valid) ? __uint_as_float(v[i]) : -INFINITY);
-        m1 = fmaxf(m1, (!MASKED || i + 1 < valid) ? __uint_as_float(v[i + 1]) : -INFINITY);
-    }
-    return fmaxf(m0, m1);
-}
-// p = 2^(s*scale - ref) for 32 key columns (keys at or beyond `valid` give 0), packed in place to
-// bf16 pairs: v[0..15] become 16 tensor-memory columns of the P operand.  Returns the row sum.
-template <bool MASKED>
-__device__ __forceinline__ float chunk_exp(uint32_t (&v)[32], int valid, float scale_log2, float neg_ref) {
-    float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-        float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2, neg_ref));
-        float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2, neg_ref));
-        if (MASKED) {
-            p0 = i < valid ? p0 : 0.f;
-            p1 = i + 1 < valid ? p1 : 0.f;
-        }
-        sum0 += p0;
-        sum1 += p1;
-        v[i >> 1] = pack_bf16(p0, p1);
-    }
-    return sum0 + sum1;
-}
 
 template <int LAYOUT>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -742,59 +562,23 @@ __global__ void __launch_bounds__(128) wait_probe_kernel(int* status, long long 
     if (threadIdx.x == 0 && !ok && abort_word) atomicCAS(status, 0, CF_ERR_TIMEOUT);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult status;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &status) == cudaSuccess &&
-            status == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    });
-    return fn;
-}
-
-// The store as a 4-D tensor (head_dim, kv heads, rows, layers); boxes of 64 x 1 x 32 x 1.  Rows past
-// the end of a layer read as zero, they never reach into the next layer.
+// The store as a 4-D tensor (head_dim, kv heads, rows, layers).
 int make_store_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span,
                    int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return CF_ERR_CUDA;
-    const cuuint64_t layer_bytes = span.n_layers > 1 ? (cuuint64_t)span.kv_stride * 2
-                                                     : (cuuint64_t)b->total_tokens * (cuuint64_t)b->token_stride * 2;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, (cuuint64_t)b->total_tokens,
-                                (cuuint64_t)span.n_layers};
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)b->token_stride * 2, layer_bytes};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
-    const cuuint32_t elem[4] = {1, 1, 1, 1};
-    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
+    const unsigned long long layer_bytes = span.n_layers > 1 ? (unsigned long long)span.kv_stride * 2
+                                                             : (unsigned long long)b->total_tokens * b->token_stride * 2;
+    return make_rows_map(map, base, g->n_kv_heads, (unsigned long long)b->total_tokens,
+                         (unsigned long long)b->token_stride * 2, span.n_layers, layer_bytes, box_rows);
 }
 
 // Keys or values of the query tokens, [layers][requests][q_len][kv heads][head_dim], as a 4-D tensor
 // (head_dim, kv heads, requests * q_len rows, layers).
 int make_self_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf_batch* b, const LayerSpan& span,
                   long long self_stride, int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return CF_ERR_CUDA;
-    const cuuint64_t rows = (cuuint64_t)b->n_requests * (cuuint64_t)b->q_len;
-    const cuuint64_t row_bytes = (cuuint64_t)g->n_kv_heads * kD * 2;
-    const cuuint64_t layer_bytes = span.n_layers > 1 ? (cuuint64_t)self_stride * 2 : rows * row_bytes;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g->n_kv_heads, rows, (cuuint64_t)span.n_layers};
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, row_bytes, layer_bytes};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
-    const cuuint32_t elem[4] = {1, 1, 1, 1};
-    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS ? CF_OK : CF_ERR_CUDA;
+    const unsigned long long rows = (unsigned long long)b->n_requests * b->q_len;
+    const unsigned long long row_bytes = (unsigned long long)g->n_kv_heads * kD * 2;
+    const unsigned long long layer_bytes = span.n_layers > 1 ? (unsigned long long)self_stride * 2 : rows * row_bytes;
+    return make_rows_map(map, base, g->n_kv_heads, rows, row_bytes, span.n_layers, layer_bytes, box_rows);
 }
 
 }  // namespace

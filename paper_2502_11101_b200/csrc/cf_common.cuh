@@ -147,6 +147,20 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t stream);
 
+// Arguments of the cache-construction attention kernels (cf_document_prefill_attn).
+struct DocAttnArgs {
+    int n_docs, n_layers, max_doc_len, prefix_len, n_q_heads, n_kv_heads;
+    long long total_tokens, token_stride, q_layer_stride, kv_layer_stride, prefix_layer_stride, out_layer_stride;
+    const int* doc_offsets;
+    float scale_log2;
+};
+int launch_docattn_simt(const cf_geom* g, const DocAttnArgs& a, const void* q, const void* k, const void* v,
+                        const void* kp, const void* vp, void* out, float* lse, cudaStream_t stream);
+bool docattn_tc_supported(const cf_geom* g, const cf_doc_batch* docs);
+int launch_docattn_tc(const cf_geom* g, const DocAttnArgs& a, const void* q, const void* k, const void* v,
+                      const void* kp, const void* vp, void* out, float* lse, int* status, cudaStream_t stream);
+int attn_path();
+
 // ---- device helpers -----------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
