@@ -32,10 +32,9 @@ if ROOT not in sys.path:
 from paper_2502_11101_b200 import workloads as W  # noqa: E402
 
 METRIC = "cached KV tokens/s through reposition+query-prefill attn"
-# DRAM bytes (read + write) of one attention-kernel launch, averaged over the four launches of a step of
-# workload 3 in the default configuration, from the ncu capture summarised in
-# profiles/attn_tc_kernel_workload3.md (102.8 MB per step).  Only valid for that kernel state and workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {("configs[2]", "layer-batched", "tcgen05"): 25.70e6}
+# DRAM bytes (read + write) of one attention-kernel launch, averaged over the launches of a step, from the
+# ncu capture summarised under profiles/; quoted only while the kernel's sources still hash to `kernel_sha`.
+NCU_TRAFFIC = {}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 
@@ -119,7 +118,7 @@ class GpuWorkload:
     """A ring of resident input sets (distinct seeds) so that consecutive steps never find their
     inputs in L2, plus the session and output buffers of the library."""
 
-    def __init__(self, cfg, seed, device, ring, batch_layers=True, self_block=False):
+    def __init__(self, cfg, seed, device, ring, batch_layers=True, self_block=False, n_reuse=0):
         from paper_2502_11101_b200.session import Session
         self.cfg, self.device = cfg, device
         self.batch_layers = batch_layers
@@ -128,7 +127,7 @@ class GpuWorkload:
         m = self.meta
         self.sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range,
                             cfg.rope_theta, cfg.q_len, m.doc_len, m.req_doc_begin, m.doc_src_start,
-                            tail_reserve=cfg.q_len, device=device)
+                            tail_reserve=cfg.q_len, n_reuse=n_reuse, device=device)
         self.slots = []
         self.self_kv = []
         for r in range(ring):
@@ -183,11 +182,12 @@ class GpuWorkload:
 
     def launches_per_step(self):
         cfg = self.cfg
-        # plan init + per attention call (attention, merge, scores; the query-self block if asked for) +
-        # prune/plan kernels + final re-positioning
+        # clear status + plan init + per attention call (attention, merge, scores; the query-self block if asked
+        # for) + prune/plan kernels + final re-positioning
         # (on the tensor-core path the block is a key tile of the attention kernel, not a launch)
         per_call = 4 if self.self_kernel else 3
-        return 1 + per_call * len(self.calls()) + len(cfg.schedule) + 1
+        prunes = sum(1 for l, _ in cfg.schedule if l <= cfg.n_layers)
+        return 2 + per_call * len(self.calls()) + prunes + 1
 
 
 def time_steps(fn, steps, warmup, world):
@@ -346,136 +346,55 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, help="1-based index into the named configurations")
-    ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--ring", type=int, default=3, help="distinct resident input sets cycled between steps")
-    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
-    ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
-    ap.add_argument("--per-layer", action="store_true",
-                    help="one attention call per layer instead of one per run of layers between two pruning layers")
-    ap.add_argument("--skip-per-layer", action="store_true",
-                    help="do not also time the step with one attention call per layer")
-    ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
-    ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
-    ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
-    ap.add_argument("--self-block", action="store_true",
-                    help="variant: every layer also attends the query tokens themselves (cf_query_prefill_attn_full)")
-    ap.add_argument("--schedule", default="config", choices=["config", "linear"],
-                    help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
-                         "a constant number of documents, down to 5)")
-    args = ap.parse_args()
-    cfg = W.CONFIGS[args.workload]
-    if args.layers:
-        cfg = W.scaled_config(cfg, n_layers=args.layers,
-                              schedule=tuple(s for s in cfg.schedule if s[0] <= args.layers))
-    if args.q_len:
-        cfg = W.scaled_config(cfg, q_len=args.q_len)
-    if args.schedule == "linear":
-        # App. C, integers only: prune after layers 4, 8, ...; floor((k - k_finish) / prunes) documents each
-        # time, the remainder at the last pruning layer
-        prunes = cfg.n_layers // 4
-        step_docs = (cfg.n_docs - 5) // max(prunes, 1)
-        cfg = W.scaled_config(cfg, schedule=tuple((4 * j, 5 if j == prunes else cfg.n_docs - j * step_docs)
-                                                  for j in range(1, prunes + 1)))
-    rank, world, local = dist_env()
+def kernel_source_sha():
+    """Digest of the attention kernel's sources: an ncu capture is only quoted for the kernel it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("cf_attn_tc.cu", "cf_tc_util.cuh"):
+        with open(os.path.join(ROOT, "paper_2502_11101_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
 
-    if args.impl == "reference":
-        args.steps = 10 if args.steps is None else args.steps
-        args.warmup = 1 if args.warmup is None else args.warmup
-        run_reference(args, cfg, rank)
-        return
 
-    args.steps = 3000 if args.steps is None else args.steps      # about half a second: several clock samples
-    args.warmup = 10 if args.warmup is None else max(3, args.warmup)
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
-    torch.cuda.set_device(local)
-    device = f"cuda:{local}"
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(device))
-    import paper_2502_11101_b200 as cf
-    from paper_2502_11101_b200 import build as cf_build
-    if rank == 0:
-        cf_build.build()
-    if world > 1:
-        dist.barrier()
-    cf.load_library()
-    if args.force_simt:
-        cf.cf_set_attn_path(1)
-    peaks = load_peaks()
+def time_blocks(fn, steps, warmup, world, min_seconds=0.3, max_blocks=400):
+    """W warm-up steps, then blocks of exactly `steps` steps, each bracketed by a barrier and a device
+    synchronisation and timed with CUDA events, repeated until `min_seconds` have passed so that the clock
+    sampler sees the timed work.  Returns (median block ms, wall start, wall end, blocks)."""
+    import torch.distributed as dist
+    for i in range(warmup):
+        fn(i)
+    times = []
+    t0 = time.time()
+    it = warmup
+    while True:
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for i in range(steps):
+            fn(it + i)
+        stop.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        it += steps
+        times.append(start.elapsed_time(stop))
+        enough = time.time() - t0 >= min_seconds or len(times) >= max_blocks
+        if world > 1:                                        # every rank must leave the loop together
+            flag = torch.tensor([1.0 if enough else 0.0], device="cuda")
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            enough = bool(flag.item() > 0.5)
+        if enough:
+            break
+    return float(np.median(times)), t0, time.time(), len(times)
 
-    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
-                     self_block=args.self_block)
-    wl.self_kernel = args.self_block and (args.force_simt or not _tc_used(cf, wl))
-    kept, survivors = wl.kept_per_layer()
-    per_layer_tokens = token_layers(cfg, wl.meta, kept)
-    tokens_per_step = sum(per_layer_tokens)
-    final_tokens = sum(int(wl.meta.doc_len[int(wl.meta.req_doc_begin[b]) + i]) for b in range(cfg.batch)
-                       for i in survivors[b]) * cfg.n_layers
-    assert wl.sess.status() == 0
 
-    # ---- CUDA graphs: one per ring slot (pointers differ) -------------------------------------
-    def capture():
-        if args.no_graph:
-            return None
-        try:
-            wl.step(0)
-            torch.cuda.synchronize()
-            made = []
-            side = torch.cuda.Stream()
-            for r in range(args.ring):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    wl.step(r)
-                made.append(g)
-            return made
-        except Exception as exc:  # capture not possible: time eager launches and say so
-            sys.stderr.write(f"[bench] graph capture failed, timing eager launches: {exc}\n")
-            torch.cuda.synchronize()
-            return None
-
-    graphs = capture()
-
-    def run(i):
-        if graphs is not None:
-            graphs[i % args.ring].replay()
-        else:
-            wl.step(i)
-
-    sampler = ClockSampler(local) if rank == 0 else None
-    ms, t0, t1 = time_steps(run, args.steps, args.warmup, world)
-    clocks = sampler.stop(t0, t1) if sampler else None
-    assert wl.sess.status() == 0
-
-    ms_max, tokens_all, value = whole_job(ms, tokens_per_step, args.steps, world, device)
-
-    # ---- the same step with one attention call per layer (what a running model can issue) ------
-    per_layer = None
-    if wl.batch_layers and world == 1 and not args.skip_per_layer:
-        main_graphs = graphs
-        wl.batch_layers = False
-        graphs = capture()
-        pl_steps = max(1, min(args.steps, 100))
-        pl_ms, _, _ = time_steps(run, pl_steps, 3, world)
-        assert wl.sess.status() == 0
-        per_layer = {"value": tokens_per_step * pl_steps / (pl_ms * 1e-3), "unit": UNIT, "ms_per_step": pl_ms / pl_steps,
-                     "steps": pl_steps, "gpu_launches_per_step": wl.launches_per_step(),
-                     "note": "one cf_query_prefill_attn call per layer"}
-        wl.batch_layers = True
-        graphs, main_graphs = main_graphs, None
-
-    # ---- the dominant kernel alone: event pairs around every attention-kernel launch ----------
-    # Launches are issued eagerly here; a spin kernel queued first keeps the GPU busy until the host
-    # has enqueued the whole step, so the event pairs time kernels running back to back and not the
-    # host's launch latency.
-    prof_steps = max(1, min(args.steps, 20))
+def attention_roofline(cf, wl, cfg, per_layer_tokens, peaks, prof_steps):
+    """Event pairs around every attention-kernel launch of a few eagerly issued steps.  A spin kernel
+    queued first keeps the GPU busy until the host has enqueued the whole step, so the pairs time kernels
+    running back to back and not the host's launch latency."""
     host_s = []
     for i in range(3):
         torch.cuda.synchronize()
@@ -497,10 +416,9 @@ def main():
     launch_bytes = np.tile(np.array(per_call_tokens, dtype=np.float64) * kv_bytes_per_token, prof_steps)
     launch_flops = np.tile(np.array(per_call_tokens, dtype=np.float64) * flops_per_token, prof_steps)
     n = min(len(durations), len(launch_bytes))
+    per_call_us = None
     if n == prof_steps * len(calls):
-        per_call = durations[:n].reshape(prof_steps, len(calls)).mean(axis=0) * 1e3
-        sys.stderr.write("[bench] attention launches of a step, mean us (layers first-last): " +
-                         " ".join(f"{lo + 1}-{hi}:{x:.1f}" for (lo, hi), x in zip(calls, per_call)) + "\n")
+        per_call_us = [float(x) for x in durations[:n].reshape(prof_steps, len(calls)).mean(axis=0) * 1e3]
     dur_s = durations[:n].sum() * 1e-3
     gbs = launch_bytes[:n].sum() / dur_s / 1e9
     tfs = launch_flops[:n].sum() / dur_s / 1e12
@@ -512,58 +430,255 @@ def main():
     else:
         roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": gbs / peaks["hbm_gbs"]}
-    traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer",
-                   "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05")
-    traffic = None if (args.layers or args.q_len or args.self_block or args.schedule != "config") else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(traffic_key)
-    roofline.update({"traffic": traffic, "traffic_unit": "bytes per launch (ncu dram read + write)",
-                     "algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()), "kernel": "fused re-position + query-prefill attention",
-                     "peak_source": peaks["source"], "avg_launch_us": 1e3 * durations[:n].mean(),
-                     "launches_timed": int(n), "hbm_gbs": gbs, "tflops": tfs,
+    roofline.update({"algorithmic_bytes_per_launch": float(launch_bytes[:n].mean()),
+                     "kernel": "fused re-position + query-prefill attention", "peak_source": peaks["source"],
+                     "avg_launch_us": 1e3 * durations[:n].mean(), "launches_timed": int(n),
+                     "attention_us_per_step": 1e3 * durations[:n].sum() / prof_steps, "hbm_gbs": gbs, "tflops": tfs,
                      "frac_of_applicable_roofline": max(t_hbm, t_tc) / dur_s})
+    if per_call_us is not None:
+        roofline["launch_us_by_call"] = [{"layers": f"{lo + 1}-{hi}", "us": us} for (lo, hi), us in zip(calls, per_call_us)]
+    return roofline
+
+
+def capture_graphs(wl, ring, no_graph):
+    """One CUDA graph of the whole step per ring slot (the pointers differ)."""
+    if no_graph:
+        return None
+    try:
+        wl.step(0)
+        torch.cuda.synchronize()
+        made = []
+        side = torch.cuda.Stream()
+        for r in range(ring):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                wl.step(r)
+            made.append(g)
+        return made
+    except Exception as exc:  # capture not possible: time eager launches and say so
+        sys.stderr.write(f"[bench] graph capture failed, timing eager launches: {exc}\n")
+        torch.cuda.synchronize()
+        return None
+
+
+def other_workload(cf, number, cfg, device, peaks, local, note):
+    """One more configuration in the same line: whole step as a CUDA graph, the attention kernel's
+    roofline fraction, and the SM clock seen while it ran."""
+    t_begin = time.time()
+    wl = GpuWorkload(cfg, 0, device, ring=1, batch_layers=True)
+    kept, _ = wl.kept_per_layer()
+    per_layer_tokens = token_layers(cfg, wl.meta, kept)
+    tokens = sum(per_layer_tokens)
+    graphs = capture_graphs(wl, 1, False)
+
+    def run(i):
+        if graphs is not None:
+            graphs[0].replay()
+        else:
+            wl.step(i)
+
+    sampler = ClockSampler(local)
+    steps = 5
+    ms, t0, t1, blocks = time_blocks(run, steps, 3, 1, min_seconds=0.4, max_blocks=200)
+    clocks = sampler.stop(t0, t1)
+    assert wl.sess.status() == 0
+    roof = attention_roofline(cf, wl, cfg, per_layer_tokens, peaks, prof_steps=3)
+    assert wl.sess.status() == 0
+    slot_mb = sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6
+    out = {"workload": f"configs[{number - 1}] {cfg.name}", "n_layers": cfg.n_layers, "requests": cfg.batch,
+           "note": note, "ms_per_step": ms / steps, "value": tokens * steps / (ms * 1e-3), "unit": UNIT,
+           "tokens_per_step": tokens, "resident_input_mb": slot_mb, "blocks_timed": blocks,
+           "attention_calls_per_step": len(wl.calls()), "gpu_launches_per_step": wl.launches_per_step(),
+           "roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac", "avg_launch_us",
+                                             "attention_us_per_step", "hbm_gbs", "tflops")},
+           "sm_mhz": clocks["sm_mhz"], "clock_reasons": clocks["reasons"], "seconds": None}
+    del wl, graphs
+    torch.cuda.empty_cache()
+    out["seconds"] = time.time() - t_begin
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, help="1-based index into the named configurations")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--ring", type=int, default=3, help="distinct resident input sets cycled between steps")
+    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core attention kernel")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="one attention call per layer instead of one per run of layers between two pruning layers")
+    ap.add_argument("--skip-per-layer", action="store_true",
+                    help="do not also time the step with one attention call per layer")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-reposition", action="store_true", help="do not time the standalone re-positioning kernel")
+    ap.add_argument("--skip-others", action="store_true", help="do not also measure the other configurations")
+    ap.add_argument("--skip-e2e", action="store_true", help="do not time the step from pinned host memory")
+    ap.add_argument("--layers", type=int, default=0, help="experiment only: truncate the stack to this many layers")
+    ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
+    ap.add_argument("--self-block", action="store_true",
+                    help="variant: every layer also attends the query tokens themselves (cf_query_prefill_attn_full)")
+    ap.add_argument("--schedule", default="config", choices=["config", "linear"],
+                    help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
+                         "a constant number of documents, down to 5)")
+    ap.add_argument("--n-reuse", default="eq6", choices=["eq6", "k", "1", "k/5", "5"],
+                    help="number of parallel windows (Sec. 3.3): Eq. 6, one window per document, a single window, "
+                         "a fifth of the documents, or five")
+    args = ap.parse_args()
+    cfg = W.CONFIGS[args.workload]
+    if args.layers:
+        cfg = W.scaled_config(cfg, n_layers=args.layers,
+                              schedule=tuple(s for s in cfg.schedule if s[0] <= args.layers))
+    if args.q_len:
+        cfg = W.scaled_config(cfg, q_len=args.q_len)
+    rank, world, local = dist_env()
+
+    if args.impl == "reference":
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        if args.schedule == "linear":
+            import oracle
+            cfg = W.scaled_config(cfg, schedule=tuple(oracle.prune_schedule_linear(cfg.n_layers, 4, cfg.n_docs, 5)))
+        run_reference(args, cfg, rank)
+        return
+
+    args.steps = 200 if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else max(3, args.warmup)
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200 import build as cf_build
+    if rank == 0:
+        cf_build.build()
+    if world > 1:
+        dist.barrier()
+    cf.load_library()
+    if args.schedule == "linear":                             # App. C, from the library
+        cfg = W.scaled_config(cfg, schedule=tuple(cf.cf_schedule_linear(cfg.n_layers, 4, cfg.n_docs, 5)))
+    if args.force_simt:
+        cf.cf_set_attn_path(1)
+    peaks = load_peaks()
+    n_reuse = {"eq6": 0, "k": cfg.n_docs, "1": 1, "k/5": max(1, cfg.n_docs // 5), "5": 5}[args.n_reuse]
+
+    wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
+                     self_block=args.self_block, n_reuse=n_reuse)
+    wl.self_kernel = args.self_block and (args.force_simt or not _tc_used(cf, wl))
+    kept, survivors = wl.kept_per_layer()
+    per_layer_tokens = token_layers(cfg, wl.meta, kept)
+    tokens_per_step = sum(per_layer_tokens)
+    final_tokens = sum(int(wl.meta.doc_len[int(wl.meta.req_doc_begin[b]) + i]) for b in range(cfg.batch)
+                       for i in survivors[b]) * cfg.n_layers
+    assert wl.sess.status() == 0, f"device status {wl.sess.status()}"
+    windows = [int(x) for x in wl.sess.read_plan()["n_reuse"]]
+
+    graphs = capture_graphs(wl, args.ring, args.no_graph)
+
+    def run(i):
+        if graphs is not None:
+            graphs[i % args.ring].replay()
+        else:
+            wl.step(i)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, t0, t1, blocks = time_blocks(run, args.steps, args.warmup, world)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    assert wl.sess.status() == 0
+
+    ms_max, tokens_all, value = whole_job(ms, tokens_per_step, args.steps, world, device)
+
+    # ---- the same step with one attention call per layer (what a running model can issue) ------
+    per_layer = None
+    if wl.batch_layers and world == 1 and not args.skip_per_layer:
+        main_graphs = graphs
+        wl.batch_layers = False
+        graphs = capture_graphs(wl, args.ring, args.no_graph)
+        pl_steps = max(1, min(args.steps, 50))
+        pl_ms, _, _, _ = time_blocks(run, pl_steps, 3, world, min_seconds=0.1)
+        assert wl.sess.status() == 0
+        per_layer = {"value": tokens_per_step * pl_steps / (pl_ms * 1e-3), "unit": UNIT, "ms_per_step": pl_ms / pl_steps,
+                     "steps": pl_steps, "gpu_launches_per_step": wl.launches_per_step(),
+                     "note": "one cf_query_prefill_attn call per layer"}
+        wl.batch_layers = True
+        graphs, main_graphs = main_graphs, None
+
+    # ---- the dominant kernel alone --------------------------------------------------------------
+    roofline = attention_roofline(cf, wl, cfg, per_layer_tokens, peaks, max(1, min(args.steps, 20)))
+    if "launch_us_by_call" in roofline:
+        sys.stderr.write("[bench] attention launches of a step, mean us (layers first-last): " +
+                         " ".join(f"{c['layers']}:{c['us']:.1f}" for c in roofline["launch_us_by_call"]) + "\n")
+    attn_kernel = "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05"
+    traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer", attn_kernel)
+    default_variant = not (args.layers or args.q_len or args.self_block or args.schedule != "config" or args.n_reuse != "eq6")
+    capture = NCU_TRAFFIC.get(traffic_key) if default_variant else None
+    sha = kernel_source_sha()
+    roofline.update({"traffic": capture["bytes_per_launch"] if capture and capture["kernel_sha"] == sha else None,
+                     "traffic_unit": "bytes per launch (ncu dram read + write)", "kernel_sha": sha,
+                     "traffic_note": None if capture and capture["kernel_sha"] == sha else
+                     "no ncu capture of this kernel state is on record (profiles/ holds the last one)"})
 
     # ---- end to end: query and cache store start in pinned host memory every step --------------
-    q0, k0, v0 = wl.slots[0]
-    resident = [q0, k0, v0] + [t for t in wl.self_kv[0] if t is not None]
-    host = [t.cpu().pin_memory() for t in resident]
-    out_h = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
-    acc_h = torch.empty(wl.sess.score_accum.shape, dtype=torch.float32).pin_memory()
-    kept_h = torch.empty(wl.sess.n_docs_total, dtype=torch.int32).pin_memory()
+    e2e = None
+    if not args.skip_e2e:
+        q0, k0, v0 = wl.slots[0]
+        resident = [q0, k0, v0] + [t for t in wl.self_kv[0] if t is not None]
+        host = [t.cpu().pin_memory() for t in resident]
+        out_h = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
+        acc_h = torch.empty(wl.sess.score_accum.shape, dtype=torch.float32).pin_memory()
+        kept_h = torch.empty(wl.sess.n_docs_total, dtype=torch.int32).pin_memory()
 
-    def e2e_step(_):
-        for src, dst in zip(host, resident):
-            dst.copy_(src, non_blocking=True)
-        wl.step(0)
-        out_h.copy_(wl.out, non_blocking=True)
-        acc_h.copy_(wl.sess.score_accum, non_blocking=True)
-        kept_h.copy_(wl.sess.field("kept", wl.sess.n_docs_total), non_blocking=True)
+        def e2e_step(_):
+            for src, dst in zip(host, resident):
+                dst.copy_(src, non_blocking=True)
+            wl.step(0)
+            out_h.copy_(wl.out, non_blocking=True)
+            acc_h.copy_(wl.sess.score_accum, non_blocking=True)
+            kept_h.copy_(wl.sess.field("kept", wl.sess.n_docs_total), non_blocking=True)
 
-    e2e_steps = max(1, min(args.steps, 20))
-    e2e_ms, _, _ = time_steps(e2e_step, e2e_steps, 3, world)
-    e2e_ms_max, _, e2e_value = whole_job(e2e_ms, tokens_per_step, e2e_steps, world, device)
-    h2d = sum(t.numel() * t.element_size() for t in host)
-    d2h = sum(t.numel() * t.element_size() for t in (out_h, acc_h, kept_h))
-    e2e = {"value": e2e_value, "unit": UNIT,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+        e2e_steps = max(1, min(args.steps, 20))
+        e2e_ms, _, _ = time_steps(e2e_step, e2e_steps, 3, world)
+        e2e_ms_max, _, e2e_value = whole_job(e2e_ms, tokens_per_step, e2e_steps, world, device)
+        h2d = sum(t.numel() * t.element_size() for t in host)
+        d2h = sum(t.numel() * t.element_size() for t in (out_h, acc_h, kept_h))
+        e2e = {"value": e2e_value, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+        del host, q0, k0, v0, resident
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    attn_kernel = "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05"
-    launches = wl.launches_per_step() * args.steps
+    launches = wl.launches_per_step() * args.steps * blocks
     n_calls = len(wl.calls())
     slot_mb = sum(t.numel() * t.element_size() for t in wl.slots[0]) / 1e6
     launch_mode = "cuda graph per ring slot" if graphs is not None else "eager"
     call_mode = ("one attention call per run of layers between two pruning layers (every layer's query states "
                  "are inputs of the step)") if wl.batch_layers else "one attention call per layer"
+    launches_per_step = wl.launches_per_step()
+    del wl, graphs
+    torch.cuda.empty_cache()
     repo = assemble = None
     if world == 1 and not args.skip_reposition:
-        del wl, graphs, host, q0, k0, v0, resident
-        torch.cuda.empty_cache()
         repo = reposition_roofline(device, peaks)
         torch.cuda.empty_cache()
         assemble = assemble_roofline(device, peaks)
+        torch.cuda.empty_cache()
+
+    others = None
+    if world == 1 and not args.skip_others and default_variant and args.workload == 3 and not args.force_simt:
+        others = [other_workload(cf, 2, W.CONFIGS[2], device, peaks, local, "single layer; the whole configuration"),
+                  other_workload(cf, 4, W.CONFIGS[4], device, peaks, local, "the whole configuration"),
+                  other_workload(cf, 5, W.scaled_config(W.CONFIGS[5], n_layers=16, schedule=((4, 60), (12, 30))),
+                                 device, peaks, local,
+                                 "first 16 of 32 layers (45 GB of keys and values resident; the full store is 90.6 GB "
+                                 "plus the final keys)")]
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -584,17 +699,20 @@ def main():
                        "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                        "docs_per_request": cfg.n_docs, "requests": cfg.batch, "q_len": cfg.q_len,
                        "schedule": [list(s) for s in cfg.schedule], "schedule_kind": args.schedule, "strategy": "align",
+                       "n_reuse_policy": args.n_reuse, "windows_at_init": windows,
                        "query_self_block": bool(args.self_block),
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
                              f"{slot_mb:.0f} MB) cycled between steps",
-                       "launch": launch_mode, "attention_calls": call_mode,
-                       "attention_calls_per_step": n_calls,
+                       "timing": f"median of {blocks} blocks of {args.steps} steps, each block between device "
+                                 "synchronisations, CUDA events",
+                       "launch": launch_mode, "stack_driver": "cf_run_stack (C ABI)", "attention_calls": call_mode,
+                       "attention_calls_per_step": n_calls, "gpu_launches_per_step": launches_per_step,
                        "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble,
-            "cpu_baseline": cpu}
+            "other_workloads": others, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
