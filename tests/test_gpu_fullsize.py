@@ -4,6 +4,8 @@ outputs the oracle computes one by one and on properties that hold at any size.
 
 Nothing the oracle consumes comes from the CUDA path: layer 1 attends every document in retrieval
 order, so its allocation and outputs are fixed by the inputs alone."""
+import types
+
 import numpy as np
 import pytest
 import torch
@@ -98,25 +100,34 @@ def test_config5_four_layers_full_batch_sampled(batch_layers):
     assert all(int(x) == 6 for x in plan0["n_reuse"])
 
 
-def _run_against_whole_oracle(cfg, sample_heads):
+def _run_against_whole_oracle(cfg, sample_heads, min_margin=5e-4):
     """The stack issued call by call (one attention call per layer) with the plan read back after
     every pruning step, against oracle.run_stack request by request: kept set, order, positions and
     windows bit-exact after every cut; every layer's document scores and log-sum-exp of the sampled
     heads, and their outputs, within tolerance."""
-    meta = W.make_meta(cfg, 0)
-    dev = "cuda:0"
-    q = W.make_q(meta, dev)
-    k, v = W.make_kv(meta, dev)
-    # the oracle's inputs: the same seeded tensors, widened exactly (bf16 -> fp32) and upcast per layer inside
-    q_h, k_h, v_h = q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy()
-    ref = []
-    for b in range(cfg.batch):
-        lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
-        ref.append(oracle.run_stack(q_h[:, b], k_h, v_h, meta.doc_len[lo:hi], meta.doc_offsets, meta.doc_src_start[lo:hi],
-                                    cfg.rope_theta, cfg.pos_range, cfg.schedule, oracle.ALLOC_ALIGN,
-                                    tail_reserve=cfg.q_len, doc_base=lo, final_reposition=False))
     from tests import harness
-    assert harness.cut_margins(meta, ref, oracle.ALLOC_ALIGN) >= 5e-4
+    dev = "cuda:0"
+    one = types.SimpleNamespace(cfg=W.scaled_config(cfg, batch=1))      # cut_margins reads the configuration only
+    # the first seed whose decisive score gaps (every cut, every request) are clear of the score error
+    for seed in range(6):
+        meta = W.make_meta(cfg, seed)
+        q = W.make_q(meta, dev)
+        k, v = W.make_kv(meta, dev)
+        # the oracle's inputs: the same seeded tensors, widened exactly (bf16 -> fp32) and upcast per layer inside
+        q_h, k_h, v_h = q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy()
+        ref = []
+        for b in range(cfg.batch):
+            lo, hi = int(meta.req_doc_begin[b]), int(meta.req_doc_begin[b + 1])
+            ref.append(oracle.run_stack(q_h[:, b], k_h, v_h, meta.doc_len[lo:hi], meta.doc_offsets, meta.doc_src_start[lo:hi],
+                                        cfg.rope_theta, cfg.pos_range, cfg.schedule, oracle.ALLOC_ALIGN,
+                                        tail_reserve=cfg.q_len, doc_base=lo, final_reposition=False))
+            if harness.cut_margins(one, ref[-1:], oracle.ALLOC_ALIGN) < min_margin:
+                break                                       # this seed is rejected: no need for its other requests
+        else:
+            break
+        del q, k, v
+    assert len(ref) == cfg.batch and harness.cut_margins(meta, ref, oracle.ALLOC_ALIGN) >= min_margin, \
+        "no seed with clear margins"
     sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
                    cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len, device=dev)
     sess.set_live_docs(cfg.n_docs)
