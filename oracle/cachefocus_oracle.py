@@ -20,7 +20,9 @@ What it follows, step by step:
   the best documents and the survivors are re-allocated ("align" / "sort", Sec. 2.5)
   (Algorithm 2, Phases 1 and 2); the linear pruning schedule of App. C;
 * the attention of the offline cache construction (Sec. 2.2): every document attends the shared
-  prefix cache and itself, causally, independently of the other documents.
+  prefix cache and itself, causally, independently of the other documents;
+* decoding over the final cache (Algorithm 2, Phase 3): each new token's key/value row is appended and
+  its query row attends the whole cache.
 
 Pins (tests/test_oracle_*.py): closed forms of the rotation group, the identity of
 Eq. 5, an independent complex-number statement of rotary encoding, the printed examples
@@ -28,7 +30,9 @@ of Sec. 3.3 (k=20, N_reuse=k/5) and App. C (L=28, n=4, k=40, k_finish=5), alloca
 invariants checked by brute force, brute-force attention with Python loops, the
 N_reuse=1 special case against a library attention routine, the closed form for Q=0; for the
 cache-construction attention a library causal attention over [prefix; document], Python loops, the
-Q=0 closed form, causality and the composition of the pinned prefix and self blocks.
+Q=0 closed form, causality and the composition of the pinned prefix and self blocks; for the decoding
+steps the rows of a library causal attention over [cache; new tokens], the Q=0 closed form and the
+agreement of a step with the pinned query_prefill_attn over the cache it has grown.
 
 Parity unpinned (conventions the paper leaves open, no figure or code to compare with):
 which two coordinates form a slice (both common layouts are implemented), round-robin
@@ -311,6 +315,37 @@ def assemble_final_cache(k_rot: np.ndarray, v_store: np.ndarray, doc_offsets: Se
     ks.append(np.asarray(k_self, dtype=np.float64))
     vs.append(np.asarray(v_self, dtype=np.float64))
     return np.concatenate(ks), np.concatenate(vs)
+
+
+def decode_steps(k_final: np.ndarray, v_final: np.ndarray, q_new: np.ndarray, k_new: np.ndarray,
+                 v_new: np.ndarray, scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Decoding over a final cache (Algorithm 2, Phase 3: Y <- LLM(C_final); the "Decoding" loop of
+    Algorithm 1), one layer, one request, attention only: step t appends the new token's key and value
+    to the cache (K <- concat(K_past, K_current) in the text under Eq. 1) and the token's single query
+    row per head attends every row of the cache, its own included (Eq. 1).
+
+    k_final, v_final[n, Hkv, D] (keys already at their final positions); q_new[a, Hq, D];
+    k_new, v_new[a, Hkv, D] with the keys rotary-encoded at the tokens' own positions.
+    Returns out[a, Hq, D] and lse[a, Hq]."""
+    k_cache = np.asarray(k_final, dtype=np.float64)
+    v_cache = np.asarray(v_final, dtype=np.float64)
+    q_new = np.asarray(q_new, dtype=np.float64)
+    a, hq, d = q_new.shape
+    g = hq // k_cache.shape[1]
+    if scale is None or scale == 0.0:
+        scale = 1.0 / math.sqrt(d)
+    out = np.zeros((a, hq, d))
+    lse = np.zeros((a, hq))
+    for t in range(a):
+        k_cache = np.concatenate([k_cache, np.asarray(k_new[t], dtype=np.float64)[None]])
+        v_cache = np.concatenate([v_cache, np.asarray(v_new[t], dtype=np.float64)[None]])
+        for h in range(hq):
+            s = (k_cache[:, h // g, :] @ q_new[t, h, :]) * scale
+            m = s.max()
+            e = np.exp(s - m)
+            out[t, h, :] = (e / e.sum()) @ v_cache[:, h // g, :]
+            lse[t, h] = m + math.log(e.sum())
+    return out, lse
 
 
 def prune_topk(score_accum: Sequence[float], order: Sequence[int], keep: int, strategy: int
