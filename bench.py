@@ -284,6 +284,51 @@ def assemble_roofline(device, peaks, layers=2, iters=5):
             "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
 
 
+def decode_roofline(cf, device, peaks, label, n_q_heads, n_kv_heads, requests, rows_used, layers, layers_per_call, iters=10):
+    """One decoding step's attention over final caches of `rows_used` rows per request (cf_decode_attn; Algorithm 2,
+    Phase 3): one query row per head streams the cache once.  Bytes = the keys and values attended."""
+    geom = cf.make_geom(n_q_heads, n_kv_heads, 128, torch.bfloat16, 1 << 20, 1e4)
+    cache_rows = rows_used + 64
+    k_fin = torch.empty((layers, requests, cache_rows, n_kv_heads, 128), dtype=torch.bfloat16, device=device).normal_()
+    v_fin = torch.empty_like(k_fin).normal_()
+    q = torch.empty((layers, requests, n_q_heads, 128), dtype=torch.bfloat16, device=device).normal_()
+    out = torch.empty_like(q)
+    rows = torch.full((requests,), rows_used - 1, dtype=torch.int32, device=device)
+    plan = torch.zeros(cf.cf_decode_plan_bytes(geom, requests, cache_rows), dtype=torch.uint8, device=device)
+    work = torch.empty(cf.cf_decode_workspace_bytes(geom, requests, cache_rows, layers_per_call), dtype=torch.uint8, device=device)
+    cf.cf_decode_plan(geom, requests, cache_rows, rows, 1, plan)
+
+    def step():
+        for l0 in range(0, layers, layers_per_call):
+            l1 = l0 + layers_per_call
+            cf.cf_decode_attn(geom, requests, cache_rows, plan, q[l0:l1], k_fin[l0:l1], v_fin[l0:l1], out[l0:l1], work)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+    graph.replay()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(iters):
+        graph.replay()
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / iters
+    assert cf.cf_decode_status(geom, requests, cache_rows, plan) == 0
+    nbytes = 2 * layers * requests * rows_used * n_kv_heads * 128 * 2
+    gbs = nbytes / ms / 1e6
+    return {"kernel": "cf_decode_attn", "workload": label, "q_heads": n_q_heads, "kv_heads": n_kv_heads,
+            "requests": requests, "rows_per_request": rows_used, "layers_resident": layers,
+            "layers_per_call": layers_per_call, "bound": "hbm", "bytes_per_step": nbytes, "ms_per_step": ms,
+            "us_per_layer": 1e3 * ms / layers, "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
+
+
 def whole_job(ms, tokens_per_step, steps, world, device):
     """Whole-job numbers of a replica run: every rank processed `tokens_per_step` tokens per step in `ms`
     milliseconds for `steps` steps; the job's time is the slowest rank's, its work the sum over ranks.
@@ -671,6 +716,14 @@ def main():
         assemble = assemble_roofline(device, peaks)
         torch.cuda.empty_cache()
 
+    decode = None
+    if world == 1 and not args.skip_reposition:
+        # the decoding step (one query row per head) over final caches with every document of the configuration kept
+        decode = [decode_roofline(cf, device, peaks, "configs[4]-shaped final caches, one call per layer", 32, 32, 8, 21600, 4, 1),
+                  decode_roofline(cf, device, peaks, "configs[3]-shaped final caches, one call per layer", 28, 4, 4, 16000, 8, 1),
+                  decode_roofline(cf, device, peaks, "configs[3]-shaped final caches, eight layers per call", 28, 4, 4, 16000, 8, 8)]
+        torch.cuda.empty_cache()
+
     others = None
     if world == 1 and not args.skip_others and default_variant and args.workload == 3 and not args.force_simt:
         others = [other_workload(cf, 2, W.CONFIGS[2], device, peaks, local, "single layer; the whole configuration"),
@@ -711,7 +764,7 @@ def main():
                        "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble,
+            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble, "decode": decode,
             "other_workloads": others, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:

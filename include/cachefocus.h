@@ -306,6 +306,54 @@ int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,
                   const float* score_accum, int32_t keep, const int32_t* keep_per_request,
                   int32_t strategy, void* stream);
 
+/* ------------------------------------------------------------------------------- decoding
+ * Algorithm 2, Phase 3 (Y <- LLM(C_final)) and the "Decoding" loop of Algorithm 1: every generated
+ * token appends its key/value rows to each request's final cache and attends all of its rows; the cost
+ * is the O((2 l_c n + a) a / 2) term of Sec. 3.3 and the decode columns of Table 2.  The caches are the
+ * packed buffers cf_assemble_final_cache writes, [n_layers][n_requests][cache_rows][n_kv_heads][head_dim]
+ * with request b using its first rows[b] rows (`rows` = that call's final_rows, device int32
+ * [n_requests], never modified here).  Their keys are already re-positioned, so nothing is rotated; the
+ * new token's key must come rotary-encoded at its own position.  A step t = 0, 1, ... of the loop is
+ *     cf_decode_append(..., rows, t, k_new, v_new, ...)      rows[b] + t receives the new rows
+ *     cf_decode_plan(..., rows, t + 1, decode_plan, ...)     once per step: rows[b] + t + 1 rows in use
+ *     cf_decode_attn(..., decode_plan, ...)                  per layer, or for several layers at once
+ * All three are asynchronous on `stream`.  cache_rows is the row capacity of a request's slot. */
+
+/* Bytes of the decode-plan buffer (device memory, 256-byte aligned) for this batch shape. */
+size_t cf_decode_plan_bytes(const cf_geom* geom, int32_t n_requests, int32_t cache_rows);
+
+/* Describes one decoding step to the attention kernels: request b attends rows 0 .. rows[b] +
+ * extra_rows - 1 of its slot.  A request whose count is below 1 or above cache_rows raises CF_ERR_RANGE
+ * in the buffer's status word (read it with cf_decode_status) and is clamped. */
+int cf_decode_plan(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, const int32_t* rows,
+                   int32_t extra_rows, void* decode_plan, size_t decode_plan_bytes, void* stream);
+
+/* Copies the status word of a decode plan back (synchronises `stream`); returns it as the error code. */
+int cf_decode_status(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, const void* decode_plan,
+                     void* stream);
+
+/* Scratch of cf_decode_attn for calls over up to n_layers layers. */
+size_t cf_decode_workspace_bytes(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, int32_t n_layers);
+
+/* The new token's attention (Eq. 1, one query row per head) over the rows the decode plan names.
+ *   q, out    device [n_layers][n_requests][n_q_heads][head_dim], layers q_layer_stride / out_layer_stride
+ *             elements apart (n_layers = 1 inside a running model: layer l+1's query comes out of layer l)
+ *   k_final, v_final  the final caches, layers kv_layer_stride elements apart
+ *   lse       device float [n_layers][n_requests][n_q_heads] or NULL
+ *   workspace at least cf_decode_workspace_bytes(..., n_layers) bytes, 256-byte aligned */
+int cf_decode_attn(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, const void* decode_plan,
+                   int32_t n_layers, const void* q, int64_t q_layer_stride, const void* k_final,
+                   const void* v_final, int64_t kv_layer_stride, float softmax_scale, void* out,
+                   int64_t out_layer_stride, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Appends one token per request: row rows[b] + step of request b's slot receives k_new / v_new
+ * ([n_layers][n_requests][n_kv_heads][head_dim], layers new_layer_stride elements apart) in every layer.
+ * A request without room raises CF_ERR_RANGE in *status (device int32, may be NULL; only written on
+ * failure) and is skipped. */
+int cf_decode_append(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, int32_t n_layers,
+                     void* k_final, void* v_final, int64_t kv_layer_stride, const int32_t* rows, int32_t step,
+                     const void* k_new, const void* v_new, int64_t new_layer_stride, int32_t* status, void* stream);
+
 /* A batch of documents for the offline cache construction: a packed store like cf_batch's, without
  * requests, allocation or plan.  doc_offsets is DEVICE memory owned by the caller. */
 typedef struct cf_doc_batch {

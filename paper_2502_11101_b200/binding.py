@@ -26,9 +26,10 @@ EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
            "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn",
            "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
-           "cf_run_stack", "cf_document_prefill_attn", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
+           "cf_run_stack", "cf_document_prefill_attn", "cf_decode_plan_bytes", "cf_decode_plan", "cf_decode_status",
+           "cf_decode_workspace_bytes", "cf_decode_attn", "cf_decode_append", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
 _SIZE_T_EXPORTS = ("cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers", "cf_attn_workspace_bytes_full",
-                   "cf_run_stack_workspace_bytes")
+                   "cf_run_stack_workspace_bytes", "cf_decode_plan_bytes", "cf_decode_workspace_bytes")
 
 
 class cf_geom(ctypes.Structure):
@@ -125,6 +126,15 @@ def load_library() -> ctypes.CDLL:
     lib.cf_debug_wait_timeout.argtypes = [gp, bp, vp, i64, vp]
     lib.cf_document_prefill_attn.argtypes = [gp, ctypes.POINTER(cf_doc_batch), i32, vp, i64, vp, vp, i64, vp, vp, i64,
                                              ctypes.c_float, vp, i64, vp, vp, vp]
+    lib.cf_decode_plan_bytes.restype = ctypes.c_size_t
+    lib.cf_decode_plan_bytes.argtypes = [gp, i32, i32]
+    lib.cf_decode_plan.argtypes = [gp, i32, i32, vp, i32, vp, ctypes.c_size_t, vp]
+    lib.cf_decode_status.argtypes = [gp, i32, i32, vp, vp]
+    lib.cf_decode_workspace_bytes.restype = ctypes.c_size_t
+    lib.cf_decode_workspace_bytes.argtypes = [gp, i32, i32, i32]
+    lib.cf_decode_attn.argtypes = [gp, i32, i32, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64, vp, vp,
+                                   ctypes.c_size_t, vp]
+    lib.cf_decode_append.argtypes = [gp, i32, i32, i32, vp, vp, i64, vp, i32, vp, vp, i64, vp, vp]
     lib.cf_set_attn_path.argtypes = [i32]
     lib.cf_profile_begin.argtypes = [i32]
     lib.cf_profile_end.argtypes = [vp, i32, vp]
@@ -448,6 +458,57 @@ def cf_profile_end(capacity: int) -> np.ndarray:
     count = ctypes.c_int32(0)
     _check(load_library().cf_profile_end(ms.ctypes.data, capacity, ctypes.addressof(count)), "cf_profile_end")
     return ms[:min(capacity, count.value)]
+
+
+def cf_decode_plan_bytes(geom: cf_geom, n_requests: int, cache_rows: int) -> int:
+    return int(load_library().cf_decode_plan_bytes(ctypes.byref(geom), n_requests, cache_rows))
+
+
+def cf_decode_workspace_bytes(geom: cf_geom, n_requests: int, cache_rows: int, n_layers: int) -> int:
+    return int(load_library().cf_decode_workspace_bytes(ctypes.byref(geom), n_requests, cache_rows, n_layers))
+
+
+def cf_decode_plan(geom: cf_geom, n_requests: int, cache_rows: int, rows: torch.Tensor, extra_rows: int,
+                   decode_plan: torch.Tensor, stream=None) -> None:
+    """One decoding step's description: request b attends rows 0 .. rows[b] + extra_rows - 1 of its slot."""
+    rc = load_library().cf_decode_plan(ctypes.byref(geom), n_requests, cache_rows, rows.data_ptr(), extra_rows,
+                                       decode_plan.data_ptr(), decode_plan.numel() * decode_plan.element_size(),
+                                       _stream(stream))
+    _check(rc, "cf_decode_plan")
+
+
+def cf_decode_status(geom: cf_geom, n_requests: int, cache_rows: int, decode_plan: torch.Tensor, stream=None) -> int:
+    return int(load_library().cf_decode_status(ctypes.byref(geom), n_requests, cache_rows, decode_plan.data_ptr(),
+                                               _stream(stream)))
+
+
+def cf_decode_attn(geom: cf_geom, n_requests: int, cache_rows: int, decode_plan: torch.Tensor, q: torch.Tensor,
+                   k_final: torch.Tensor, v_final: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor,
+                   lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, stream=None) -> None:
+    """q, out [n_layers, B, Hq, D]; k_final, v_final [n_layers, B, cache_rows, Hkv, D]; lse [n_layers, B, Hq]."""
+    n_layers = q.shape[0]
+    assert k_final.shape[0] == n_layers and v_final.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k_final.stride(0) == v_final.stride(0) and (lse is None or lse.is_contiguous())
+    rc = load_library().cf_decode_attn(ctypes.byref(geom), n_requests, cache_rows, decode_plan.data_ptr(), n_layers,
+                                       q.data_ptr(), q.stride(0), k_final.data_ptr(), v_final.data_ptr(),
+                                       k_final.stride(0), softmax_scale, out.data_ptr(), out.stride(0), _ptr(lse),
+                                       workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                       _stream(stream))
+    _check(rc, "cf_decode_attn")
+
+
+def cf_decode_append(geom: cf_geom, n_requests: int, cache_rows: int, k_final: torch.Tensor, v_final: torch.Tensor,
+                     rows: torch.Tensor, step: int, k_new: torch.Tensor, v_new: torch.Tensor,
+                     status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """k_new, v_new [n_layers, B, Hkv, D] become row rows[b] + step of request b's slot in every layer."""
+    n_layers = k_final.shape[0]
+    assert v_final.shape[0] == n_layers and k_new.shape[0] == n_layers and v_new.shape[0] == n_layers
+    assert k_final.stride(0) == v_final.stride(0) and k_new.stride(0) == v_new.stride(0)
+    rc = load_library().cf_decode_append(ctypes.byref(geom), n_requests, cache_rows, n_layers, k_final.data_ptr(),
+                                         v_final.data_ptr(), k_final.stride(0), rows.data_ptr(), step,
+                                         k_new.data_ptr(), v_new.data_ptr(), k_new.stride(0), _ptr(status),
+                                         _stream(stream))
+    _check(rc, "cf_decode_append")
 
 
 def plan_field(plan: torch.Tensor, layout: cf_plan_layout, name: str, count: int, dtype=torch.int32) -> torch.Tensor:
