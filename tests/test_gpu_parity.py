@@ -81,6 +81,15 @@ def test_forced_window_counts():
         harness.run_and_compare(cfg, 0, oracle.ALLOC_ALIGN, n_reuse=n_reuse, min_margin=1e-3)
 
 
+def test_window_count_policies_of_the_reuse_study():
+    """The policies of Sec. 3.3 on k = 20 documents (the case its text works through): N_reuse = k, 1, k/5
+    (four windows of five documents, each position used four times) and a fixed 5, besides Eq. 6."""
+    cfg = W.scaled_config(W.CONFIGS[2], n_docs=20, n_planted=4, schedule=((1, 10),))
+    for n_reuse in (20, 1, 20 // 5, 5, 0):
+        report = harness.run_and_compare(cfg, 0, oracle.ALLOC_ALIGN, n_reuse=n_reuse, min_margin=1e-3)
+        assert report["margin"] >= 1e-3
+
+
 def test_keep_larger_than_live_set_and_no_pruning():
     cfg = W.scaled_config(W.CONFIGS[3], n_layers=3, n_docs=9, n_planted=2, schedule=((1, 20), (2, 9)))
     harness.run_and_compare(cfg, 0, oracle.ALLOC_SORT, min_margin=1e-3)
