@@ -329,6 +329,47 @@ def decode_roofline(cf, device, peaks, label, n_q_heads, n_kv_heads, requests, r
             "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
 
 
+def docattn_roofline(cf, device, peaks, n_q_heads=12, n_kv_heads=2, n_docs=400, lo=128, hi=192, layers=4, prefix=64, iters=10):
+    """cf_document_prefill_attn (offline cache construction, Sec. 2.2): documents shaped like the benchmark's attend a
+    shared prefix and themselves under the causal mask.  Flops = 4 * head_dim * visible (row, key) pairs per query head
+    (QK^T and PV, the masked half of the square not counted)."""
+    rng = np.random.default_rng(0)
+    lens = rng.integers(lo, hi + 1, size=n_docs)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(off[-1])
+    geom = cf.make_geom(n_q_heads, n_kv_heads, 128, torch.bfloat16, 32768, 1e6)
+    q = torch.empty((layers, total, n_q_heads, 128), dtype=torch.bfloat16, device=device).normal_()
+    k = torch.empty((layers, total, n_kv_heads, 128), dtype=torch.bfloat16, device=device).normal_()
+    v = torch.empty_like(k).normal_()
+    kp = torch.empty((layers, prefix, n_kv_heads, 128), dtype=torch.bfloat16, device=device).normal_()
+    vp = torch.empty_like(kp).normal_()
+    out = torch.empty_like(q)
+    off_d = torch.from_numpy(off).to(device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def step():
+        cf.cf_document_prefill_attn(geom, off_d, int(lens.max()), q, k, v, out, kp, vp, None, status=status)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(iters):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / iters
+    assert int(status.item()) == 0
+    pairs = float(sum(int(n) * prefix + int(n) * (int(n) + 1) // 2 for n in lens))
+    flops = 4.0 * 128 * pairs * n_q_heads * layers
+    tfs = flops / ms / 1e9
+    return {"kernel": "cf_document_prefill_attn", "workload": f"{n_docs} documents of {lo}-{hi} tokens behind a {prefix}-token "
+            f"prefix, {n_q_heads}/{n_kv_heads} heads, {layers} layers per call", "bound": "tensor", "flops_per_launch": flops,
+            "ms_per_launch": ms, "achieved": tfs, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": tfs / peaks["tflops"],
+            "tokens_per_s": total * layers / (ms * 1e-3), "peak_source": peaks["source"]}
+
+
 def whole_job(ms, tokens_per_step, steps, world, device):
     """Whole-job numbers of a replica run: every rank processed `tokens_per_step` tokens per step in `ms`
     milliseconds for `steps` steps; the job's time is the slowest rank's, its work the sum over ranks.
@@ -723,15 +764,15 @@ def main():
                   decode_roofline(cf, device, peaks, "configs[3]-shaped final caches, one call per layer", 28, 4, 4, 16000, 8, 1),
                   decode_roofline(cf, device, peaks, "configs[3]-shaped final caches, eight layers per call", 28, 4, 4, 16000, 8, 8)]
         torch.cuda.empty_cache()
+    docattn = docattn_roofline(cf, device, peaks) if world == 1 and not args.skip_reposition else None
 
     others = None
     if world == 1 and not args.skip_others and default_variant and args.workload == 3 and not args.force_simt:
         others = [other_workload(cf, 2, W.CONFIGS[2], device, peaks, local, "single layer; the whole configuration"),
                   other_workload(cf, 4, W.CONFIGS[4], device, peaks, local, "the whole configuration"),
-                  other_workload(cf, 5, W.scaled_config(W.CONFIGS[5], n_layers=16, schedule=((4, 60), (12, 30))),
-                                 device, peaks, local,
-                                 "first 16 of 32 layers (45 GB of keys and values resident; the full store is 90.6 GB "
-                                 "plus the final keys)")]
+                  other_workload(cf, 5, W.CONFIGS[5], device, peaks, local,
+                                 "the whole configuration: 32 layers, 90.6 GB of keys and values plus 45.3 GB of final "
+                                 "keys resident")]
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -764,7 +805,7 @@ def main():
                        "attention_kernel": attn_kernel,
                        "parallelism": f"replicas x{world}"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble, "decode": decode,
+            "roofline": roofline, "per_layer_launch": per_layer, "reposition": repo, "assemble": assemble, "decode": decode, "document_prefill": docattn,
             "other_workloads": others, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
