@@ -257,46 +257,77 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             // Sequence entry n: warpgroup w = n & 1, its item j = n >> 1, key tile = n (alternating)
             // or j (side by side).  Issue order: S(0) S(1), then PV(n) followed by S(n + 2): the
             // next QK^T of a warpgroup follows its own PV in the pipe, so S may overwrite the P it aliases.
+            // This one thread is the pacemaker of the CTA: whatever it executes between two bursts of
+            // tcgen05.mma is time in which the tensor cores idle.  Its ring positions and barrier parities are
+            // therefore running counters, and every descriptor is a precomputed base plus a stage offset.
             const uint32_t idesc_o = instr_desc(kD, true);
+            const uint32_t idesc_s0 = instr_desc(0, false);
             const int n_seq = alternate ? n_it : 2 * n_it;
+            const int period = alternate ? 3 : 5;                   // tiles after which a stage's parity flips
+            const uint64_t a_desc0 = smem_desc(q_base, 16, 1024);
+            const uint64_t a_desc1 = alternate ? a_desc0 : smem_desc(q_base + kTileBytes, 16, 1024);
+            const uint64_t bk_desc = smem_desc(ring_base, 16, 1024);
+            const uint64_t bv_desc = smem_desc(ring_base, kHalfBytes, 1024);
+            const uint32_t bar_k_ready = smem_u32(&bars->k_ready[0]), bar_kv_full = smem_u32(&bars->kv_full[0][0]);
+            const uint32_t bar_kv_empty = smem_u32(&bars->kv_empty[0]);
+            const uint32_t bar_s_full = smem_u32(&bars->s_full[0]), bar_p_ready = smem_u32(&bars->p_ready[0]);
+            const uint32_t bar_o_done = smem_u32(&bars->o_done[0]);
+            // position of the next tile of one kind (keys: stages 0, 2, 4, ...; values: 1, 3, 5, ...) in the ring
+            struct Cursor {
+                int stage, parity, count, tile;
+            };
+            auto advance = [&](Cursor& c) {
+                c.stage += 2;
+                if (c.stage >= n_stages) c.stage -= n_stages;
+                if (++c.count == period) {
+                    c.count = 0;
+                    c.parity ^= 1;
+                }
+                ++c.tile;
+            };
+            auto keys_of = [&](int it) -> int {                     // MMA extent of a tile: its rows rounded up to 16
+                const int len = it == self_it ? lq : (it < kMetaTiles ? (s_meta[it].y & 0xff) : pv.tile_len[ti0 + it]);
+                return (len + 15) & ~15;
+            };
+            Cursor ck = {0, 0, 0, 0}, cv = {1, 0, 0, 0};            // keys for the next QK^T, values for the next PV
             auto issue_s = [&](int n) -> bool {
                 const int w = n & 1;
-                const int it = alternate ? n : (n >> 1);
-                const int n_keys = (tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len + 15) & ~15;
-                const int stk = ring_mod(2 * it, alternate);
-                const int kuse = ring_uses(it, alternate);
-                if (!mbar_wait(smem_u32(&bars->k_ready[stk]), kuse & 1, abort_flag)) return false;
+                const int n_keys = keys_of(ck.tile);
+                if (!mbar_wait(bar_k_ready + ck.stage * 8, ck.parity, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t a0 = smem_desc(q_base + (alternate ? 0 : w) * kTileBytes, 16, 1024);
-                const uint64_t b0 = smem_desc(ring_base + stk * kTileBytes, 16, 1024);
-                const uint32_t idesc_s = instr_desc(n_keys, false);
+                const uint64_t a0 = w ? a_desc1 : a_desc0;
+                const uint64_t b0 = bk_desc + (uint64_t)(ck.stage * (kTileBytes >> 4));
+                const uint32_t idesc_s = idesc_s0 | ((uint32_t)(n_keys >> 3) << 17);
+                const uint32_t s_tmem = tmem + w * 128;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {                    // 16 dims per instruction
                     const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-                    umma(tmem + w * 128, a0 + off, b0 + off, idesc_s, kk > 0);
+                    umma(s_tmem, a0 + off, b0 + off, idesc_s, kk > 0);
                 }
-                umma_commit(smem_u32(&bars->s_full[w]));
-                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stk]));   // last reader of the keys
+                umma_commit(bar_s_full + w * 8);
+                if (alternate || w == 1) {                          // last reader of the keys
+                    umma_commit(bar_kv_empty + ck.stage * 8);
+                    advance(ck);
+                }
                 return true;
             };
             auto issue_pv = [&](int n) -> bool {
                 const int w = n & 1, j = n >> 1;
-                const int it = alternate ? n : j;
-                const int n_keys = (tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len + 15) & ~15;
-                const int stv = ring_mod(2 * it + 1, alternate);
-                const int vuse = ring_uses(it, alternate);                  // value loads this stage has seen
-                if (!mbar_wait(smem_u32(&bars->kv_full[stv][1]), vuse & 1, abort_flag)) return false;
-                if (!mbar_wait(smem_u32(&bars->p_ready[w]), j & 1, abort_flag)) return false;
+                const int n_steps = keys_of(cv.tile) >> 4;          // 16 keys = 8 packed columns per instruction
+                if (!mbar_wait(bar_kv_full + cv.stage * 16 + 8, cv.parity, abort_flag)) return false;
+                if (!mbar_wait(bar_p_ready + w * 8, j & 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t b0 = smem_desc(ring_base + stv * kTileBytes, kHalfBytes, 1024);
+                const uint64_t b0 = bv_desc + (uint64_t)(cv.stage * (kTileBytes >> 4));
                 const uint32_t o_tmem = tmem + 256 + w * 128, p_tmem = tmem + w * 128;
-                const int n_steps = n_keys >> 4;                    // 16 keys = 8 packed columns per instruction
                 umma_ts(o_tmem, p_tmem, b0, idesc_o, j > 0);
 #pragma unroll
                 for (int kk = 1; kk < kTile / 16; ++kk)
                     if (kk < n_steps) umma_ts(o_tmem, p_tmem + kk * 8, b0 + (uint64_t)(kk * 128), idesc_o, 1u);
-                umma_commit(smem_u32(&bars->o_done[w]));
-                if (alternate || w == 1) umma_commit(smem_u32(&bars->kv_empty[stv]));   // last reader of the values
+                umma_commit(bar_o_done + w * 8);
+                if (alternate || w == 1) {                          // last reader of the values
+                    umma_commit(bar_kv_empty + cv.stage * 8);
+                    advance(cv);
+                }
                 return true;
             };
             bool ok = issue_s(0);
