@@ -129,6 +129,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     __shared__ int s_cnt[kMaxDocs];       // tile count by local id
     __shared__ int s_src[kMaxDocs];       // positions the documents were cached at, by local id
     __shared__ float s_score[kMaxDocs];
+    __shared__ float s_all[kMaxDocs];     // accumulated scores of all documents of the request, by local id
     __shared__ unsigned char s_flag[kMaxDocs];
     __shared__ int s_longest, s_min_cursor;
     __shared__ int s_warp_sum[kPlanThreads / 32 + 1];
@@ -149,8 +150,21 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     const int half = gv.head_dim / 2;
     const int half_log2 = half == 64 ? 6 : 5;
 
-    // ---- stage the inputs -------------------------------------------------------------------
+    // ---- stage the inputs (everything here depends on doc0 alone: one round trip to global memory) ----
     int n_old = 0, keep_b = 0, n_kept = 0;
+    const int kept_count_old = mode == 0 ? 0 : pv.kept_count[b];
+    const int keep_arg = (mode != 0 && keep_per_request) ? keep_per_request[b] : keep;
+    const int kept_raw = (mode != 0 && tid < n_docs) ? pv.kept[doc0 + tid] : 0;    // rank tid, if there is one
+    if (mode != 0 && tid < n_docs) s_all[tid] = score_accum[doc0 + tid];            // S of every document, by local id
+    for (int i = tid; i <= n_docs; i += kPlanThreads) s_row[i] = bv.doc_offsets[doc0 + i];
+    for (int i = tid; i < n_docs; i += kPlanThreads) {
+        s_src[i] = bv.doc_src_start[doc0 + i];
+        s_dst[i] = mode == 0 ? -1 : pv.dst_start[doc0 + i];
+        s_group[i] = mode == 0 ? -1 : pv.group[doc0 + i];
+    }
+    int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
+                                : pv.query_start[b];
+    int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
     if (mode == 0) {
         n_kept = kept_count_in ? kept_count_in[b] : n_docs;
         n_kept = max(0, min(n_kept, n_docs));
@@ -166,24 +180,10 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
             s_ids[r] = id;
         }
     } else {
-        n_old = max(0, min(pv.kept_count[b], n_docs));
-        keep_b = keep_per_request ? keep_per_request[b] : keep;
-        keep_b = max(0, min(keep_b, n_old));
-        for (int r = tid; r < n_old; r += kPlanThreads) {
-            const int id = max(0, min(pv.kept[doc0 + r], n_docs - 1));
-            s_ids[r] = id;
-            s_score[r] = score_accum[doc0 + id];
-        }
+        n_old = max(0, min(kept_count_old, n_docs));
+        keep_b = max(0, min(keep_arg, n_old));
+        if (tid < n_old) s_ids[tid] = max(0, min(kept_raw, n_docs - 1));
     }
-    for (int i = tid; i <= n_docs; i += kPlanThreads) s_row[i] = bv.doc_offsets[doc0 + i];
-    for (int i = tid; i < n_docs; i += kPlanThreads) {
-        s_src[i] = bv.doc_src_start[doc0 + i];
-        s_dst[i] = mode == 0 ? -1 : pv.dst_start[doc0 + i];
-        s_group[i] = mode == 0 ? -1 : pv.group[doc0 + i];
-    }
-    int query_start = mode == 0 ? (query_start_arg < 0 ? gv.pos_range - bv.tail_reserve : query_start_arg)
-                                : pv.query_start[b];
-    int windows = mode == 0 ? max(1, bv.n_reuse) : pv.n_reuse[b];
     if (tid == 0) {
         s_longest = 0;
         s_min_cursor = 0x7fffffff;
@@ -192,6 +192,8 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
 
     // ---- the kept list, in rank order -------------------------------------------------------
     if (mode != 0) {
+        if (tid < n_old) s_score[tid] = s_all[s_ids[tid]];
+        __syncthreads();
         // rank by counting: how many kept documents beat this one (ties: lower id wins); eight
         // lanes share the count of one document
         for (int r0 = 0; r0 < n_old; r0 += kPlanThreads / 8) {
