@@ -34,7 +34,8 @@ from paper_2502_11101_b200 import workloads as W  # noqa: E402
 METRIC = "cached KV tokens/s through reposition+query-prefill attn"
 # DRAM bytes (read + write) of one attention-kernel launch, averaged over the launches of a step, from the
 # ncu capture summarised under profiles/; quoted only while the kernel's sources still hash to `kernel_sha`.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {("configs[2]", "layer-batched", "tcgen05"):
+               {"bytes_per_launch": 25.66e6, "kernel_sha": "a5fdc19e574e3b26", "summary": "profiles/attn_tc_kernel_workload3.md"}}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 
