@@ -119,7 +119,7 @@ class GpuWorkload:
     """A ring of resident input sets (distinct seeds) so that consecutive steps never find their
     inputs in L2, plus the session and output buffers of the library."""
 
-    def __init__(self, cfg, seed, device, ring, batch_layers=True, self_block=False, n_reuse=0):
+    def __init__(self, cfg, seed, device, ring, batch_layers=True, self_block=False, n_reuse=0, prefix=0):
         from paper_2502_11101_b200.session import Session
         self.cfg, self.device = cfg, device
         self.batch_layers = batch_layers
@@ -128,7 +128,12 @@ class GpuWorkload:
         m = self.meta
         self.sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range,
                             cfg.rope_theta, cfg.q_len, m.doc_len, m.req_doc_begin, m.doc_src_start,
-                            tail_reserve=cfg.q_len, n_reuse=n_reuse, device=device)
+                            tail_reserve=cfg.q_len, n_reuse=n_reuse, prefix_len=prefix, device=device)
+        self.prefix_kv = None
+        if prefix:                                   # a shared prefix cache attended by every layer (random contents)
+            shape = (cfg.n_layers, prefix, cfg.n_kv_heads, cfg.head_dim)
+            self.prefix_kv = (torch.empty(shape, dtype=cfg.torch_dtype, device=device).normal_(),
+                              torch.empty(shape, dtype=cfg.torch_dtype, device=device).normal_())
         self.slots = []
         self.self_kv = []
         for r in range(ring):
@@ -148,7 +153,9 @@ class GpuWorkload:
         q, k, v = self.slots[slot % len(self.slots)]
         k_self, v_self = self.self_kv[slot % len(self.slots)]
         self.sess.run_stack(q, k, v, self.cfg.schedule, STRATEGY_ALIGN, self.out, self.lse, self.k_final,
-                            batch_layers=self.batch_layers, k_self=k_self, v_self=v_self)
+                            batch_layers=self.batch_layers, k_self=k_self, v_self=v_self,
+                            k_prefix=None if self.prefix_kv is None else self.prefix_kv[0],
+                            v_prefix=None if self.prefix_kv is None else self.prefix_kv[1])
 
     def calls(self):
         """(first, last) layer ranges of the attention calls of one step."""
@@ -608,6 +615,9 @@ def main():
     ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
     ap.add_argument("--self-block", action="store_true",
                     help="variant: every layer also attends the query tokens themselves (cf_query_prefill_attn_full)")
+    ap.add_argument("--prefix", type=int, default=0,
+                    help="variant: every layer also attends a shared prefix cache of this many tokens "
+                         "(cf_query_prefill_attn_prefix)")
     ap.add_argument("--schedule", default="config", choices=["config", "linear"],
                     help="pruning schedule: the workload's own, or the paper's linear one (App. C: every 4 layers, "
                          "a constant number of documents, down to 5)")
@@ -655,7 +665,7 @@ def main():
     n_reuse = {"eq6": 0, "k": cfg.n_docs, "1": 1, "k/5": max(1, cfg.n_docs // 5), "5": 5}[args.n_reuse]
 
     wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
-                     self_block=args.self_block, n_reuse=n_reuse)
+                     self_block=args.self_block, n_reuse=n_reuse, prefix=args.prefix)
     wl.self_kernel = args.self_block and (args.force_simt or not _tc_used(cf, wl))
     kept, survivors = wl.kept_per_layer()
     per_layer_tokens = token_layers(cfg, wl.meta, kept)
@@ -702,7 +712,7 @@ def main():
                          " ".join(f"{c['layers']}:{c['us']:.1f}" for c in roofline["launch_us_by_call"]) + "\n")
     attn_kernel = "cuda-core" if args.force_simt or not _tc_used(cf, wl) else "tcgen05"
     traffic_key = (f"configs[{args.workload - 1}]", "layer-batched" if wl.batch_layers else "per-layer", attn_kernel)
-    default_variant = not (args.layers or args.q_len or args.self_block or args.schedule != "config" or args.n_reuse != "eq6")
+    default_variant = not (args.layers or args.q_len or args.self_block or args.prefix or args.schedule != "config" or args.n_reuse != "eq6")
     capture = NCU_TRAFFIC.get(traffic_key) if default_variant else None
     sha = kernel_source_sha()
     roofline.update({"traffic": capture["bytes_per_launch"] if capture and capture["kernel_sha"] == sha else None,
@@ -795,7 +805,7 @@ def main():
                        "docs_per_request": cfg.n_docs, "requests": cfg.batch, "q_len": cfg.q_len,
                        "schedule": [list(s) for s in cfg.schedule], "schedule_kind": args.schedule, "strategy": "align",
                        "n_reuse_policy": args.n_reuse, "windows_at_init": windows,
-                       "query_self_block": bool(args.self_block),
+                       "query_self_block": bool(args.self_block), "prefix_len": args.prefix,
                        "tokens_per_step": tokens_per_step, "final_reposition_tokens": final_tokens,
                        "l2": f"ring of {args.ring} resident input sets ({args.ring} x "
                              f"{slot_mb:.0f} MB) cycled between steps",

@@ -272,6 +272,28 @@ int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const
                                float* lse, float* doc_scores, float* score_accum,
                                void* workspace, size_t workspace_bytes, void* stream);
 
+/* cf_query_prefill_attn_full with the shared prefix cache C_prefix attended in the same call
+ * (Algorithm 2: concat([C_prefix] + [C_d_i ...]); Sec. 2.2: every document was cached behind that prefix):
+ * the prefix's keys are used as cached, at positions 0 .. prefix_len-1 (delta 0, no rotation), every query row
+ * sees all of them, and they ride along as further key tiles of the same kernel.  The prefix is no document: it
+ * is in no kept list, never pruned, and doc_scores stay the documents' shares of the mass that falls on the
+ * documents (they still sum to 1 per request); out and lse cover all key sets.
+ *   k_prefix, v_prefix  device [n_layers][prefix_len][n_kv_heads][head_dim] dense, layers prefix_layer_stride
+ *                   elements apart; one prefix for all requests of the batch; prefix_len <= batch->prefix_len
+ *                   (the positions the allocation keeps clear of documents)
+ *   k_self, v_self  as in cf_query_prefill_attn_full, or both NULL: documents and prefix only
+ *   workspace       at least cf_attn_workspace_bytes_full(geom, batch, n_layers) bytes
+ * Built for bf16 storage with head_dim 128 (the tensor-core kernel); other geometries return
+ * CF_ERR_UNSUPPORTED and join a prefix through a call of its own and cf_merge_attn. */
+int cf_query_prefill_attn_prefix(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                                 int32_t n_layers, const void* q, int64_t q_layer_stride,
+                                 const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                                 const void* k_prefix, const void* v_prefix, int64_t prefix_layer_stride,
+                                 int32_t prefix_len, const void* k_self, const void* v_self,
+                                 int64_t self_layer_stride, float softmax_scale, void* out,
+                                 int64_t out_layer_stride, float* lse, float* doc_scores, float* score_accum,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same computation as cf_query_prefill_attn for callers that cannot allocate device memory
  * (the paper has no counterpart; this is a property of the library, not of the method).
  * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
@@ -434,6 +456,11 @@ typedef struct cf_stack {
                                      k_cache itself)                                                  */
     const int32_t* doc_len_host;        /* host [n_docs_total] or NULL: lets the call size its grids  */
     const int32_t* req_doc_begin_host;  /* host [n_requests+1] or NULL    to the documents still kept */
+    const void* k_prefix;         /* NULL, or the shared prefix cache attended by every layer         */
+    const void* v_prefix;         /* (cf_query_prefill_attn_prefix): [n_layers][prefix_len][kv][dim]  */
+    int64_t prefix_layer_stride;
+    int32_t prefix_len;           /* 0 = no prefix; at most batch->prefix_len                         */
+    int32_t reserved2;
 } cf_stack;
 
 /* Scratch needed by cf_run_stack (the largest of its attention calls); 0 on invalid arguments. */

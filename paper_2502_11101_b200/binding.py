@@ -17,6 +17,7 @@ CF_ROPE_HALF, CF_ROPE_INTERLEAVED = 0, 1
 CF_ALLOC_NONE, CF_ALLOC_ALIGN, CF_ALLOC_SORT = 0, 1, 2
 CF_TILE_TOKENS = 128
 CF_MAX_LAYERS_PER_CALL = 64
+CF_MAX_SPLITS = 64
 TC_KERNEL_BUILT = True      # bf16 / head_dim 128 batches take the tcgen05 attention kernel
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefocus.so")
@@ -24,7 +25,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
-           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_assemble_final_cache", "cf_merge_attn",
+           "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_query_prefill_attn_prefix", "cf_assemble_final_cache", "cf_merge_attn",
            "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
            "cf_run_stack", "cf_document_prefill_attn", "cf_decode_plan_bytes", "cf_decode_plan", "cf_decode_status",
            "cf_decode_workspace_bytes", "cf_decode_attn", "cf_decode_append", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
@@ -71,7 +72,9 @@ class cf_stack(ctypes.Structure):
                 ("out", ctypes.c_void_p), ("out_layer_stride", ctypes.c_int64),
                 ("lse", ctypes.c_void_p), ("layer_scores", ctypes.c_void_p), ("score_accum", ctypes.c_void_p),
                 ("k_final", ctypes.c_void_p),
-                ("doc_len_host", ctypes.c_void_p), ("req_doc_begin_host", ctypes.c_void_p)]
+                ("doc_len_host", ctypes.c_void_p), ("req_doc_begin_host", ctypes.c_void_p),
+                ("k_prefix", ctypes.c_void_p), ("v_prefix", ctypes.c_void_p), ("prefix_layer_stride", ctypes.c_int64),
+                ("prefix_len", ctypes.c_int32), ("reserved2", ctypes.c_int32)]
 
 
 class CacheFocusError(RuntimeError):
@@ -116,6 +119,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes_full.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_full.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, vp, vp, i64, ctypes.c_float,
                                                vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.cf_query_prefill_attn_prefix.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, vp, vp, i64, i32, vp, vp, i64,
+                                                 ctypes.c_float, vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_query_prefill_attn_static.argtypes = [gp, bp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.cf_prune_topk.argtypes = [gp, bp, vp, vp, i32, vp, i32, vp]
     lib.cf_prune_topk_host.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp]
@@ -334,6 +339,30 @@ def cf_query_prefill_attn_full(geom: cf_geom, batch: cf_batch, plan: torch.Tenso
     _check(rc, "cf_query_prefill_attn_full")
 
 
+def cf_query_prefill_attn_prefix(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,
+                                 k_cache: torch.Tensor, v_cache: torch.Tensor, k_prefix: torch.Tensor,
+                                 v_prefix: torch.Tensor, out: torch.Tensor, workspace: torch.Tensor,
+                                 k_self: Optional[torch.Tensor] = None, v_self: Optional[torch.Tensor] = None,
+                                 lse: Optional[torch.Tensor] = None, doc_scores: Optional[torch.Tensor] = None,
+                                 score_accum: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                                 stream=None) -> None:
+    """cf_query_prefill_attn_full with a shared prefix cache attended in the same call: `k_prefix`, `v_prefix`
+    [n_layers, P, Hkv, D] dense; `k_self`, `v_self` [n_layers, B, Lq, Hkv, D] or None."""
+    n_layers = q.shape[0]
+    assert k_cache.shape[0] == n_layers and v_cache.shape[0] == n_layers and out.shape[0] == n_layers
+    assert k_prefix.shape[0] == n_layers and v_prefix.shape == k_prefix.shape and k_prefix.stride(0) == v_prefix.stride(0)
+    assert k_cache.stride(0) == v_cache.stride(0) and (k_self is None) == (v_self is None)
+    for t in (lse, doc_scores):
+        assert t is None or (t.shape[0] == n_layers and t.is_contiguous())
+    rc = load_library().cf_query_prefill_attn_prefix(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), n_layers, q.data_ptr(), q.stride(0),
+        k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(0), k_prefix.data_ptr(), v_prefix.data_ptr(),
+        k_prefix.stride(0), k_prefix.shape[1], _ptr(k_self), _ptr(v_self), 0 if k_self is None else k_self.stride(0),
+        softmax_scale, out.data_ptr(), out.stride(0), _ptr(lse), _ptr(doc_scores), _ptr(score_accum),
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn_prefix")
+
+
 def cf_query_prefill_attn_static(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, q: torch.Tensor,
                                  k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
                                  lse: Optional[torch.Tensor] = None, doc_scores: Optional[torch.Tensor] = None,
@@ -373,7 +402,8 @@ def make_stack(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, ou
                lse: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
                k_final: Optional[torch.Tensor] = None, k_self: Optional[torch.Tensor] = None,
                v_self: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
-               doc_len: Optional[np.ndarray] = None, req_doc_begin: Optional[np.ndarray] = None):
+               doc_len: Optional[np.ndarray] = None, req_doc_begin: Optional[np.ndarray] = None,
+               k_prefix: Optional[torch.Tensor] = None, v_prefix: Optional[torch.Tensor] = None):
     """A cf_stack over torch buffers (dimension 0 = layers, may be strided; the rest of a layer dense).
     Returns (struct, keepalive): the host arrays the struct points to live in `keepalive`."""
     n_layers = q.shape[0]
@@ -397,7 +427,9 @@ def make_stack(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, ou
                   q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(), k_cache.stride(0),
                   _ptr(k_self), _ptr(v_self), 0 if k_self is None else k_self.stride(0),
                   out.data_ptr(), out.stride(0), _ptr(lse), _ptr(layer_scores), score_accum.data_ptr(),
-                  _ptr(k_final), None if dl is None else dl.ctypes.data, None if rb is None else rb.ctypes.data)
+                  _ptr(k_final), None if dl is None else dl.ctypes.data, None if rb is None else rb.ctypes.data,
+                  _ptr(k_prefix), _ptr(v_prefix), 0 if k_prefix is None else k_prefix.stride(0),
+                  0 if k_prefix is None else k_prefix.shape[1], 0)
     return st, keep
 
 

@@ -188,11 +188,12 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
     size_t l = take(nlb * n_splits * rows);
     size_t t = take((size_t)n_layers * max_tiles * rows);
     size_t r = take(nlb * rows);
-    size_t so = 0, sm = 0, sl = 0;
+    size_t so = 0, sm = 0, sl = 0, ld = 0;
     if (with_self) {                                  // behind everything else: the rest of the layout does not move
         so = take(nlb * rows * g->head_dim);
         sm = take(nlb * rows);
         sl = take(nlb * rows);
+        ld = take(nlb * n_splits * rows);
     }
     if (ws) {
         ws->part_o = reinterpret_cast<float*>(base + o);
@@ -208,6 +209,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->self_o = with_self ? reinterpret_cast<float*>(base + so) : nullptr;
         ws->self_m = with_self ? reinterpret_cast<float*>(base + sm) : nullptr;
         ws->self_l = with_self ? reinterpret_cast<float*>(base + sl) : nullptr;
+        ws->part_ld = with_self ? reinterpret_cast<float*>(base + ld) : nullptr;
         ws->self_mode = 0;
     }
     return off;
@@ -244,7 +246,8 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     const void* q, const void* k_cache, const void* v_cache, const void* k_self,
                     const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
-                    size_t workspace_bytes, cudaStream_t s) {
+                    size_t workspace_bytes, cudaStream_t s, const void* k_prefix, const void* v_prefix,
+                    long long prefix_stride, int prefix_len) {
     int rc = check_plan(geom, batch, plan);
     if (rc != CF_OK) return rc;
     if (!q || !k_cache || !v_cache || !out || !workspace) return CF_ERR_INVALID_ARG;
@@ -264,6 +267,13 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
             (span.out_stride * esize) % 16 || (span.kv_stride * esize) % 16)
             return CF_ERR_INVALID_ARG;
     }
+    const bool with_prefix = prefix_len > 0;
+    if (with_prefix) {
+        const long long layer_rows = (long long)prefix_len * geom->n_kv_heads * geom->head_dim;
+        if (!k_prefix || !v_prefix || reinterpret_cast<uintptr_t>(k_prefix) % 16 || reinterpret_cast<uintptr_t>(v_prefix) % 16 ||
+            prefix_len > batch->prefix_len || (span.n_layers > 1 && (prefix_stride < layer_rows || (prefix_stride * esize) % 16)))
+            return CF_ERR_INVALID_ARG;
+    }
     const bool with_self = k_self != nullptr || v_self != nullptr;
     if (with_self) {
         const long long layer_rows = (long long)batch->n_requests * batch->q_len * geom->n_kv_heads * geom->head_dim;
@@ -273,12 +283,14 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     }
     const int n_splits = choose_splits(geom, batch, span.n_layers);
     AttnWorkspace ws;
-    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, with_self, &ws, workspace);
+    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, with_self || with_prefix, &ws, workspace);
     if (workspace_bytes < need) return CF_ERR_WORKSPACE;
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
     const bool tensor_core = g_attn_path.load() == 0 && attn_tc_supported(geom, batch);
     if (with_self && batch->q_len > CF_TILE_TOKENS) return CF_ERR_UNSUPPORTED;
+    if (with_prefix && !tensor_core) return CF_ERR_UNSUPPORTED;   // the CUDA-core path joins a prefix through cf_merge_attn
+    if (!tensor_core) ws.part_ld = nullptr;           // only the tensor-core kernel reports per-part document sums
     if (with_self && !tensor_core) {                  // the CUDA-core path computes the block as a part of its own
         ws.self_mode = 1;
         rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, scale * kLog2e, ws, s);
@@ -289,8 +301,9 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     if (timed) cudaEventRecord(ev_start, s);
     if (tensor_core) {
         ws.part_bf16 = 1;
-        ws.self_mode = with_self ? 2 : 0;             // the block rides along as one more key tile
-        rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, k_self, v_self, self_stride, scale * kLog2e, ws, s);
+        ws.self_mode = (with_self || with_prefix) ? 2 : 0;   // the blocks ride along as further key tiles
+        rc = launch_attn_tc(geom, batch, pv, span, q, k_cache, v_cache, k_self, v_self, self_stride, k_prefix, v_prefix,
+                            prefix_stride, prefix_len, scale * kLog2e, ws, s);
     } else
         rc = launch_attn_simt(geom, batch, pv, span, q, k_cache, v_cache, scale * kLog2e, ws, s);
     if (timed) cudaEventRecord(ev_stop, s);
@@ -555,6 +568,23 @@ int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const
     return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, k_self, v_self, self_layer_stride,
                            softmax_scale, out, lse, doc_scores, score_accum, workspace, workspace_bytes,
                            static_cast<cudaStream_t>(stream));
+}
+
+int cf_query_prefill_attn_prefix(const cf_geom* geom, const cf_batch* batch, const void* plan,
+                                 int32_t n_layers, const void* q, int64_t q_layer_stride,
+                                 const void* k_cache, const void* v_cache, int64_t kv_layer_stride,
+                                 const void* k_prefix, const void* v_prefix, int64_t prefix_layer_stride,
+                                 int32_t prefix_len, const void* k_self, const void* v_self,
+                                 int64_t self_layer_stride, float softmax_scale, void* out,
+                                 int64_t out_layer_stride, float* lse, float* doc_scores, float* score_accum,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (q_layer_stride < 0 || kv_layer_stride < 0 || out_layer_stride < 0 || self_layer_stride < 0 ||
+        prefix_layer_stride < 0 || prefix_len <= 0 || !k_prefix || !v_prefix || (k_self == nullptr) != (v_self == nullptr))
+        return CF_ERR_INVALID_ARG;
+    const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, k_self, v_self, self_layer_stride,
+                           softmax_scale, out, lse, doc_scores, score_accum, workspace, workspace_bytes,
+                           static_cast<cudaStream_t>(stream), k_prefix, v_prefix, prefix_layer_stride, prefix_len);
 }
 
 int cf_prune_topk(const cf_geom* geom, const cf_batch* batch, void* plan,

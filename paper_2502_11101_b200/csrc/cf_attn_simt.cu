@@ -254,12 +254,14 @@ combine_kernel(AttnWorkspace ws, int n_requests, long long n_rows_all, long long
     // the documents' share of the row: what the document scores are measured against
     float docs_l = l_sum;
     if (ws.self_mode == 2) {
-        // the block was the last key tile of one part: that part counts with its sum over documents alone
-        const size_t srow = (size_t)lb * rows_total + rg;
-        const int sp = __float_as_int(ws.self_m[srow]);
-        const float ld = ws.self_l[srow];
-        const float l0 = sp == lane ? ld : l[0], l1 = sp == lane + 32 ? ld : l[1];
-        docs_l = fmaf(l1, w[1], l0 * w[0]);                             // same tree as l_sum, no subtraction
+        // further key blocks were tiles of some parts: every part reports its sum over the documents alone
+        float ld[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int p = lane + 32 * k;
+            ld[k] = (p < n_parts && m[k] > -INFINITY) ? ws.part_ld[slot0 + (size_t)p * rows_total] : 0.f;
+        }
+        docs_l = fmaf(ld[1], w[1], ld[0] * w[0]);                       // same tree as l_sum, no subtraction
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) docs_l += __shfl_xor_sync(0xffffffffu, docs_l, o);
     }

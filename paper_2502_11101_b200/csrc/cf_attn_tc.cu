@@ -43,6 +43,7 @@ constexpr int kThreads = 512;
 struct StoreMaps {
     CUtensorMap k[4], v[4];
     CUtensorMap ks[4], vs[4];      // keys and values of the query tokens themselves (calls with a query-self block)
+    CUtensorMap kp[4], vp[4];      // keys and values of a shared prefix cache (calls that attend one)
 };
 constexpr int kSmemTiles = 7;                      // 2 Q + 5 ring, or 1 Q + 6 ring
 constexpr int kMetaTiles = 128;                    // key tiles of a CTA whose description is staged in shared memory
@@ -74,15 +75,27 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 struct TileInfo {
     int row0, len, doc;
 };
-// The query-self block, when the CTA has it, is its last tile: document -1, rows of the query's own
-// key/value tensors.
-__device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView& pv, int ti0, int it, int self_it = -1,
-                                              int self_row0 = 0, int self_len = 0) {
+// Key blocks besides the kept documents, which the CTA of the last pair of parts takes after its documents'
+// tiles: first the tiles of a shared prefix cache (document -2: rows of the prefix tensors, every row of
+// the query sees them), then the query-self block as one tile (document -1: rows of the query's own
+// key/value tensors under the causal mask).  Neither is rotated, neither is a document that is scored.
+struct ExtraTiles {
+    int first;               // index of the first such tile in the CTA's list = number of its document tiles
+    int n_prefix, prefix_len;
+    int self_it, self_row0, self_len;
+};
+__device__ __forceinline__ TileInfo tile_info(const int2* s_meta, const PlanView& pv, int ti0, int it, const ExtraTiles& ex) {
     TileInfo t;
-    if (it == self_it) {
-        t.row0 = self_row0;
-        t.len = self_len;
-        t.doc = -1;
+    if (it >= ex.first) {
+        if (it == ex.self_it) {
+            t.row0 = ex.self_row0;
+            t.len = ex.self_len;
+            t.doc = -1;
+        } else {
+            t.row0 = (it - ex.first) * kTile;
+            t.len = min(kTile, ex.prefix_len - t.row0);
+            t.doc = -2;
+        }
     } else if (it < kMetaTiles) {
         const int2 m = s_meta[it];
         t.row0 = m.x;
@@ -107,7 +120,7 @@ template <int LAYOUT>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
-               float scale_log2, const __nv_bfloat16* __restrict__ q, int with_self) {
+               float scale_log2, const __nv_bfloat16* __restrict__ q, int with_self, int prefix_len) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -145,11 +158,14 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     const int n_pairs = n_parts >> 1;
     const int t_begin = (int)((long long)n_tiles * pair / n_pairs);
     const int t_end = (int)((long long)n_tiles * (pair + 1) / n_pairs);
-    // the CTA of the last pair of parts also takes the query-self block, as one more tile after its documents'
-    const bool has_self = with_self && pair == n_pairs - 1;
-    const int n_it = t_end - t_begin + (has_self ? 1 : 0);          // key tiles of this CTA
-    const int self_it = has_self ? n_it - 1 : -1;
-    const int self_row0 = b * lq;
+    // the CTA of the last pair of parts also takes the prefix cache and the query-self block, as more tiles after its
+    // documents'
+    const bool last_pair = pair == n_pairs - 1;
+    const bool has_self = with_self && last_pair;
+    const int n_doc_it = t_end - t_begin;
+    const int n_prefix_it = last_pair ? (prefix_len + kTile - 1) / kTile : 0;
+    const int n_it = n_doc_it + n_prefix_it + (has_self ? 1 : 0);   // key tiles of this CTA
+    const ExtraTiles ex = {n_doc_it, n_prefix_it, prefix_len, has_self ? n_it - 1 : -1, b * lq, lq};
     // first workspace row of this CTA in part 2*pair
     const size_t slot0 = ((size_t)lb * n_parts + 2 * pair) * rows_total + (size_t)kvh * rows + rg * rg_rows;
 
@@ -160,7 +176,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     }
     if (n_it <= 0) return;
     const int ti0 = tbase + t_begin;                                // first tile of this CTA in the plan's list
-    if (tid < min(n_it, kMetaTiles) && tid != self_it) {
+    if (tid < min(n_doc_it, kMetaTiles)) {
         const int len = pv.tile_len[ti0 + tid], doc = pv.tile_doc[ti0 + tid];
         s_meta[tid] = make_int2(pv.tile_row0[ti0 + tid], (len & 0xff) | (doc << 8));   // len 1..128 -> 0x80 at most
     }
@@ -206,11 +222,12 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
     int produced = 0;
     auto produce = [&](int u) {                                     // u-th ring use: K(u/2) if even, V(u/2) if odd
         const int st = ring_mod(u, alternate);
-        const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1, self_it, self_row0, lq);
+        const TileInfo tile = tile_info(s_meta, pv, ti0, u >> 1, ex);
         const int row0 = tile.row0;
         const int boxes = (tile.len + kBoxRows - 1) / kBoxRows;
-        const CUtensorMap* map = tile.doc < 0 ? ((u & 1) ? &maps.vs[boxes - 1] : &maps.ks[boxes - 1])
-                                              : ((u & 1) ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
+        const CUtensorMap* map = tile.doc == -1 ? ((u & 1) ? &maps.vs[boxes - 1] : &maps.ks[boxes - 1])
+                                 : tile.doc == -2 ? ((u & 1) ? &maps.vp[boxes - 1] : &maps.kp[boxes - 1])
+                                                  : ((u & 1) ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
         const uint32_t bar = smem_u32(&bars->kv_full[st][u & 1]);
         const uint32_t dst = ring_base + st * kTileBytes;
         mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
@@ -286,8 +303,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 ++c.tile;
             };
             auto keys_of = [&](int it) -> int {                     // MMA extent of a tile: its rows rounded up to 16
-                const int len = it == self_it ? lq : (it < kMetaTiles ? (s_meta[it].y & 0xff) : pv.tile_len[ti0 + it]);
-                return (len + 15) & ~15;
+                return (tile_info(s_meta, pv, ti0, it, ex).len + 15) & ~15;
             };
             Cursor ck = {0, 0, 0, 0}, cv = {1, 0, 0, 0};            // keys for the next QK^T, values for the next PV
             auto issue_s = [&](int n) -> bool {
@@ -342,7 +358,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
         const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
         const int chunk = t & 7, rsub = t >> 3;
         for (int it = 0; it < n_it; ++it) {
-            const TileInfo tile = tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq);
+            const TileInfo tile = tile_info(s_meta, pv, ti0, it, ex);
             const int len = tile.len;
             const float2* trig = pv.trig + (size_t)max(tile.doc, 0) * (kD / 2);
             const int st = ring_mod(2 * it, alternate);
@@ -413,16 +429,21 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             const bool row_valid = row_in_group < rows_here;
             const size_t tile_row = (size_t)kvh * rows + rg * rg_rows + row_in_group;
             float* tile_lse2 = ws.tile_lse2 + (size_t)layer * ws.max_tiles * rows_total;
-            float m_ref = -INFINITY, l_run = 0.f, l_docs = 0.f;
+            float m_ref = -INFINITY, l_run = 0.f, l_docs = 0.f;     // l_docs: the sum over the documents' keys alone
+            bool seen_extra = false;
             const int q_index = (rg * rg_rows + row_in_group) % lq;     // position of this row's token in the query
             bool ok = true;
             for (int j = 0; j < n_items; ++j) {
                 const int it = alternate ? 2 * j + w : j;
                 const int ti = ti0 + it;
-                const int len = tile_info(s_meta, pv, ti0, it, self_it, self_row0, lq).len;
+                const int len = tile_info(s_meta, pv, ti0, it, ex).len;
                 // keys this row may see: the whole tile of a document, the query tokens 0..q_index of the
                 // query-self block (causal mask, footnote to Eq. 1)
-                const int vis = it == self_it ? min(len, q_index + 1) : len;
+                const int vis = it == ex.self_it ? min(len, q_index + 1) : len;
+                if (it >= ex.first && !seen_extra) {                // from here on the keys are not the documents'
+                    l_docs = l_run;
+                    seen_extra = true;
+                }
                 ok = mbar_wait(smem_u32(&bars->s_full[w]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -468,6 +489,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                             tmem_st16(s_addr + cc * 16, pk);
                         }
                         l_run *= alpha;
+                        l_docs *= alpha;
                         tile_sum *= alpha;
                     }
                 };
@@ -494,11 +516,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars->p_ready[w]));
-                if (it == self_it) {
-                    l_docs = l_run;                                 // the documents' share of this part's sum (the block is the last tile)
-                } else if (row_valid) {
-                    tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
-                }
+                if (it < ex.first && row_valid) tile_lse2[(size_t)ti * rows_total + tile_row] = m_ref + log2f(tile_sum);
                 l_run += tile_sum;
             }
             if (ok) ok = mbar_wait(smem_u32(&bars->o_done[w]), (n_items - 1) & 1, abort_flag);
@@ -542,12 +560,8 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (row_valid) {
                     ws.part_m[slot] = m_ref;
                     ws.part_l[slot] = l_run;
-                    if (has_self && (alternate ? 2 * (n_items - 1) + w : n_items - 1) == self_it) {
-                        // which part of this row holds the block, and that part's sum over documents alone
-                        const size_t srow = (size_t)lb * rows_total + tile_row;
-                        ws.self_m[srow] = __int_as_float(2 * pair + (alternate ? w : 0));
-                        ws.self_l[srow] = l_docs;
-                    }
+                    // this part's sum over the documents alone: what the document scores are measured against
+                    if (ws.part_ld) ws.part_ld[slot] = seen_extra ? l_docs : l_run;
                 }
             }
         }
@@ -612,6 +626,16 @@ int make_self_map(CUtensorMap* map, const void* base, const cf_geom* g, const cf
     return make_rows_map(map, base, g->n_kv_heads, rows, row_bytes, span.n_layers, layer_bytes, box_rows);
 }
 
+// Keys or values of a shared prefix cache, [layers][prefix_len][kv heads][head_dim] dense, as a 4-D tensor
+// (head_dim, kv heads, prefix rows, layers).
+int make_prefix_map(CUtensorMap* map, const void* base, const cf_geom* g, const LayerSpan& span, int prefix_len,
+                    long long prefix_stride, int box_rows) {
+    const unsigned long long row_bytes = (unsigned long long)g->n_kv_heads * kD * 2;
+    const unsigned long long layer_bytes = span.n_layers > 1 ? (unsigned long long)prefix_stride * 2
+                                                             : (unsigned long long)prefix_len * row_bytes;
+    return make_rows_map(map, base, g->n_kv_heads, (unsigned long long)prefix_len, row_bytes, span.n_layers, layer_bytes, box_rows);
+}
+
 }  // namespace
 
 int launch_wait_probe(const PlanView& pv, long long limit_cycles, cudaStream_t stream) {
@@ -625,6 +649,7 @@ bool attn_tc_supported(const cf_geom* g, const cf_batch* b) {
 
 int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span, const void* q,
                    const void* k, const void* v, const void* k_self, const void* v_self, long long self_stride,
+                   const void* k_prefix, const void* v_prefix, long long prefix_stride, int prefix_len,
                    float scale_log2, const AttnWorkspace& ws, cudaStream_t stream) {
     const int rows = (g->n_q_heads / g->n_kv_heads) * b->q_len;
     const int row_groups = (rows + ws.rg_rows - 1) / ws.rg_rows;
@@ -646,6 +671,15 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
             maps.ks[i] = maps.k[i];
             maps.vs[i] = maps.v[i];
         }
+        if (prefix_len > 0) {
+            rc = make_prefix_map(&maps.kp[i], k_prefix, g, span, prefix_len, prefix_stride, (i + 1) * kBoxRows);
+            if (rc != CF_OK) return rc;
+            rc = make_prefix_map(&maps.vp[i], v_prefix, g, span, prefix_len, prefix_stride, (i + 1) * kBoxRows);
+            if (rc != CF_OK) return rc;
+        } else {
+            maps.kp[i] = maps.k[i];
+            maps.vp[i] = maps.v[i];
+        }
     }
     if (k_self && b->q_len > kTile) return CF_ERR_UNSUPPORTED;   // the query-self block is one key tile
     dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
@@ -656,7 +690,7 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
         if (configure_smem_once(configured[which], kernel, kSmemBytes) != CF_OK) return CF_ERR_CUDA;
         kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, bv, pv, ws, span.q_stride, g->n_q_heads,
                                                        g->n_kv_heads, scale_log2, static_cast<const __nv_bfloat16*>(q),
-                                                       k_self ? 1 : 0);
+                                                       k_self ? 1 : 0, prefix_len);
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
     if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);

@@ -96,13 +96,14 @@ struct AttnWorkspace {
     int n_layers;
     int max_tiles;     // tile slots per layer in tile_lse2
     int rg_rows;       // query rows per CTA of the tensor-core kernel: 256 (two row tiles) or 128
-    // The query-self block of a call that has one.  self_mode 1 (CUDA-core path): it is one more part,
-    // (self_m, self_l, self_o) like (part_m, part_l, part_o) in fp32.  self_mode 2 (tensor-core path):
-    // it is the last key tile of one of the parts; self_m holds that part's index (an int) and self_l
-    // the part's sum over the documents alone.  self_mode 0: none.
+    // Key blocks besides the documents (the query-self block, a shared prefix cache) of a call that has some.
+    // self_mode 1 (CUDA-core path): the query-self block is one more part, (self_m, self_l, self_o) like
+    // (part_m, part_l, part_o) in fp32.  self_mode 2 (tensor-core path): the blocks are further key tiles of
+    // the last parts, and part_ld holds every part's sum over the documents' keys alone.  self_mode 0: none.
     float* self_o;     // [L*B][Hq*Lq][D]
     float* self_m;     // [L*B][Hq*Lq]
     float* self_l;     // [L*B][Hq*Lq]
+    float* part_ld;    // [L*B][n_splits][Hq*Lq]    like part_l, the documents' keys only (self_mode 2)
     int self_mode;
 };
 size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers, bool with_self,
@@ -132,7 +133,8 @@ int launch_attn_simt(const cf_geom* g, const cf_batch* b, const PlanView& pv, co
                      const AttnWorkspace& ws, cudaStream_t stream);
 int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
                    const void* q, const void* k, const void* v, const void* k_self, const void* v_self,
-                   long long self_stride, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream);
+                   long long self_stride, const void* k_prefix, const void* v_prefix, long long prefix_stride,
+                   int prefix_len, float scale_log2, const AttnWorkspace& ws, cudaStream_t stream);
 bool attn_tc_supported(const cf_geom* g, const cf_batch* b);
 int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, const LayerSpan& span,
                    const AttnWorkspace& ws, void* out, float* lse, float* doc_scores,
@@ -145,7 +147,8 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     const void* q, const void* k_cache, const void* v_cache, const void* k_self,
                     const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
-                    size_t workspace_bytes, cudaStream_t stream);
+                    size_t workspace_bytes, cudaStream_t stream, const void* k_prefix = nullptr,
+                    const void* v_prefix = nullptr, long long prefix_stride = 0, int prefix_len = 0);
 
 // Arguments of the cache-construction attention kernels (cf_document_prefill_attn).
 struct DocAttnArgs {

@@ -88,6 +88,7 @@ int check_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* st) 
     if (st->strategy != CF_ALLOC_NONE && st->strategy != CF_ALLOC_ALIGN && st->strategy != CF_ALLOC_SORT)
         return CF_ERR_INVALID_ARG;
     if ((st->k_self == nullptr) != (st->v_self == nullptr)) return CF_ERR_INVALID_ARG;
+    if (st->prefix_len < 0 || (st->prefix_len > 0 && (!st->k_prefix || !st->v_prefix))) return CF_ERR_INVALID_ARG;
     return CF_OK;
 }
 
@@ -107,7 +108,7 @@ size_t cf_run_stack_workspace_bytes(const cf_geom* geom, const cf_batch* batch, 
     for (const Call& c : calls_of(stack)) {
         local.tiles_hint = live_tiles_hint(batch, stack, keep);
         const int m = c.last - c.first;
-        need = std::max(need, stack->k_self ? cf_attn_workspace_bytes_full(geom, &local, m)
+        need = std::max(need, (stack->k_self || stack->prefix_len > 0) ? cf_attn_workspace_bytes_full(geom, &local, m)
                                             : cf_attn_workspace_bytes_layers(geom, &local, m));
         if (c.prune_after >= 0) keep = std::min(keep, stack->prune_keep[c.prune_after]);
     }
@@ -121,7 +122,8 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
     if (!stack->q || !stack->k_cache || !stack->v_cache || !stack->out || !stack->score_accum || !plan || !workspace)
         return CF_ERR_INVALID_ARG;
     if (stack->n_layers > 1 && (stack->q_layer_stride <= 0 || stack->kv_layer_stride <= 0 || stack->out_layer_stride <= 0 ||
-                                (stack->k_self && stack->self_layer_stride <= 0)))
+                                (stack->k_self && stack->self_layer_stride <= 0) ||
+                                (stack->prefix_len > 0 && stack->prefix_layer_stride <= 0)))
         return CF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t esize = geom->dtype == CF_BF16 ? 2 : 4;
@@ -145,7 +147,16 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
         char* out = static_cast<char*>(stack->out) + (size_t)c.first * stack->out_layer_stride * esize;
         float* lse = stack->lse ? stack->lse + (size_t)c.first * lse_layer : nullptr;
         float* scores = stack->layer_scores ? stack->layer_scores + (size_t)c.first * nd : nullptr;
-        if (stack->k_self) {
+        if (stack->prefix_len > 0) {
+            const char* ks = stack->k_self ? static_cast<const char*>(stack->k_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
+            const char* vs = stack->v_self ? static_cast<const char*>(stack->v_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
+            const char* kp = static_cast<const char*>(stack->k_prefix) + (size_t)c.first * stack->prefix_layer_stride * esize;
+            const char* vp = static_cast<const char*>(stack->v_prefix) + (size_t)c.first * stack->prefix_layer_stride * esize;
+            rc = cf_query_prefill_attn_prefix(geom, &local, plan, m, q, stack->q_layer_stride, k, v, stack->kv_layer_stride,
+                                              kp, vp, stack->prefix_layer_stride, stack->prefix_len, ks, vs,
+                                              stack->self_layer_stride, stack->softmax_scale, out, stack->out_layer_stride,
+                                              lse, scores, stack->score_accum, workspace, workspace_bytes, stream);
+        } else if (stack->k_self) {
             const char* ks = static_cast<const char*>(stack->k_self) + (size_t)c.first * stack->self_layer_stride * esize;
             const char* vs = static_cast<const char*>(stack->v_self) + (size_t)c.first * stack->self_layer_stride * esize;
             rc = cf_query_prefill_attn_full(geom, &local, plan, m, q, stack->q_layer_stride, k, v, stack->kv_layer_stride,

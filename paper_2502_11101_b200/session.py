@@ -121,19 +121,21 @@ class Session:
                   k_final: Optional[torch.Tensor] = None, layer_scores: Optional[torch.Tensor] = None,
                   batch_layers: bool = False, k_self: Optional[torch.Tensor] = None,
                   v_self: Optional[torch.Tensor] = None, driver: str = "library",
-                  softmax_scale: float = 0.0) -> None:
+                  softmax_scale: float = 0.0, k_prefix: Optional[torch.Tensor] = None,
+                  v_prefix: Optional[torch.Tensor] = None) -> None:
         """Algorithm 2, Phases 1 and 2: q, out [L, B, Lq, Hq, D]; k, v [L, T, Hkv, D];
         lse [L, B, Hq, Lq]; `layer_scores` [L, n_docs_total] receives each layer's document scores.
 
         With `batch_layers` the layers between two pruning layers go to the attention kernels in one
         launch (possible here because every layer's query states are given up front).  With `k_self`,
         `v_self` [L, B, Lq, Hkv, D] every layer also attends the query tokens themselves (causal).
+        With `k_prefix`, `v_prefix` [L, P, Hkv, D] every layer also attends that shared prefix cache.
         `driver="library"`: one cf_run_stack call sequences the stack inside the library;
         `driver="calls"`: the same sequence issued from here, one library call per step."""
         if driver == "library":
             st, keepalive = B.make_stack(q, k, v, out, self.score_accum, schedule, strategy, batch_layers, lse,
                                          layer_scores, k_final, k_self, v_self, softmax_scale, self.doc_len,
-                                         self.req_doc_begin_h)
+                                         self.req_doc_begin_h, k_prefix, v_prefix)
             self.batch.tiles_hint = 0
             need = B.cf_run_stack_workspace_bytes(self.geom, self.batch, st)
             if need > self.workspace.numel():
@@ -141,7 +143,7 @@ class Session:
             B.cf_run_stack(self.geom, self.batch, st, self.plan, self.workspace)
             del keepalive
             return
-        assert driver == "calls"
+        assert driver == "calls" and k_prefix is None, "a prefix cache goes through the library's stack driver"
         sched = dict(schedule)
         n_layers = q.shape[0]
         self.set_live_docs(int(np.diff(self.req_doc_begin_h).max()))

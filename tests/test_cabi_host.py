@@ -97,9 +97,9 @@ def test_workspace_size_of_layer_batched_calls(lib):
         # per layer: the merged log-sum-exp of every row and one value per (tile slot, row)
         rows, tile_slots = 12 * 48, 50 + 8000 // 128 + 1
         assert need >= n_layers * 4 * (rows + tile_slots * rows)
-        # with a query-self block: one more part per row (reference, sum, fp32 row) at most
+        # with further key blocks: one more part per row (reference, sum, fp32 row) and one more sum per part and row
         full = cf.cf_attn_workspace_bytes_full(geom, batch, n_layers)
-        assert need < full <= need + n_layers * rows * 4 * (128 + 2) + 3 * 256
+        assert need < full <= need + n_layers * rows * 4 * (128 + 2 + cf.CF_MAX_SPLITS) + 4 * 256
     assert cf.cf_attn_workspace_bytes_full(geom, batch, 0) == 0
     assert cf.cf_attn_workspace_bytes_layers(geom, batch, 0) == 0
     assert cf.cf_attn_workspace_bytes_layers(geom, batch, cf.CF_MAX_LAYERS_PER_CALL + 1) == 0

@@ -655,3 +655,104 @@ def test_decoding_step_over_the_assembled_final_cache():
             got = out[l, b].float().cpu().numpy()
             assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref))
             assert np.all(np.abs(lse[l, b].cpu().numpy() - lse_ref) <= 1e-2)
+
+
+@pytest.mark.parametrize("prefix,q_len,heads,with_self", [
+    (40, 6, (8, 2), False),          # one prefix tile, one row tile, both warpgroups on alternate tiles
+    (200, 48, (12, 2), True),        # two prefix tiles, 288 rows per kv head, the query-self block behind them
+    (130, 64, (8, 2), True),         # 256 rows: two row tiles side by side
+    (128, 3, (4, 4), True),          # a full prefix tile, fewer document tiles than parts
+])
+def test_pinned_prefix_attended_inside_the_call(prefix, q_len, heads, with_self):
+    """cf_query_prefill_attn_prefix: the shared prefix cache rides along as further key tiles (delta 0, seen by
+    every query row), with or without the causal query-self block behind it; one softmax over prefix, kept
+    documents and query tokens in the oracle.  Document scores stay those of the documents alone, pruning
+    included; two layers in one call as well as one by one."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    hq, hkv = heads
+    d, pos_range, theta = 128, 4096, 1e4
+    lens = np.array([130, 64, 17, 96, 200, 128, 33], dtype=np.int32)
+    n = len(lens)
+    gen = torch.Generator().manual_seed(5)
+    rnd = lambda *shape: torch.randn(shape, generator=gen).bfloat16()
+    q, k, v = rnd(2, 1, q_len, hq, d), rnd(2, int(lens.sum()), hkv, d), rnd(2, int(lens.sum()), hkv, d)
+    kp, vp = rnd(2, prefix, hkv, d), rnd(2, prefix, hkv, d)
+    ks, vs = rnd(2, 1, q_len, hkv, d), rnd(2, 1, q_len, hkv, d)
+    sess = Session(hq, hkv, d, torch.bfloat16, pos_range, theta, q_len, lens, np.array([0, n], dtype=np.int32),
+                   np.full(n, prefix, dtype=np.int32), tail_reserve=q_len, prefix_len=prefix)
+    qg, kg, vg, kpg, vpg, ksg, vsg = [t.cuda() for t in (q, k, v, kp, vp, ks, vs)]
+    offsets = np.concatenate([[0], np.cumsum(lens)])
+
+    def reference(order):
+        """Per layer: (out, lse) over prefix + documents (+ query tokens), and the documents' scores."""
+        res = []
+        for layer in range(2):
+            dst, _, _, _ = oracle.allocate_positions(lens, order, pos_range, prefix, q_len)
+            assert np.all(dst[order] >= prefix)
+            k_rot = oracle.reposition_keys(k[layer].double().numpy(), offsets, np.full(n, prefix), dst, order, theta)
+            k_all = np.concatenate([kp[layer].double().numpy(), k_rot])
+            v_all = np.concatenate([vp[layer].double().numpy(), v[layer].double().numpy()])
+            qd = q[layer, 0].double().numpy()
+            o_ref, lse_ref, _, _ = oracle.query_prefill_attn(qd, k_all, v_all, np.concatenate([[0], prefix + offsets]),
+                                                             [0] + [1 + i for i in order], n + 1)
+            if with_self:
+                o_self, lse_self = oracle.query_self_block(qd, ks[layer, 0].double().numpy(), vs[layer, 0].double().numpy())
+                o_ref, lse_ref = oracle.merge_softmax_blocks(o_ref, lse_ref, o_self, lse_self)
+            _, _, _, s_docs = oracle.query_prefill_attn(qd, k_rot, v[layer].double().numpy(), offsets, order, n)
+            res.append((o_ref, lse_ref, s_docs))
+        return res
+
+    def check(out, lse, scores, ref):
+        for layer in range(2):
+            o_ref, lse_ref, s_docs = ref[layer]
+            got = out[layer, 0].float().cpu().numpy()
+            assert np.all(np.abs(got - o_ref) <= 1e-2 + 2e-2 * np.abs(o_ref)), layer
+            assert np.all(np.abs(lse[layer, 0].cpu().numpy() - lse_ref) <= 1e-2), layer
+            s_got = scores[layer].cpu().numpy()
+            assert np.all(np.abs(s_got - s_docs) <= 1e-2 / max(1, int((s_docs > 0).sum())) + 2e-2 * s_docs), layer
+            assert abs(float(s_got.sum()) - 1.0) < 1e-3
+
+    out = torch.full_like(qg, float("nan"))
+    lse = torch.full((2, 1, hq, q_len), float("nan"), device="cuda")
+    scores = torch.full((2, n), float("nan"), device="cuda")
+    sess.init()
+    sess.reserve_workspace(2, with_self=True)
+    self_kv = dict(k_self=ksg, v_self=vsg) if with_self else {}
+    # both layers in one call, every document kept
+    cf.cf_query_prefill_attn_prefix(sess.geom, sess.batch, sess.plan, qg, kg, vg, kpg, vpg, out, sess.workspace,
+                                    lse=lse, doc_scores=scores, score_accum=sess.score_accum, **self_kv)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    order = list(range(n))
+    ref = reference(order)
+    check(out, lse, scores, ref)
+    accum = ref[0][2] + ref[1][2]
+    assert np.all(np.abs(sess.score_accum.cpu().numpy() - accum) <= 1e-2 + 2e-2 * accum)
+    # a pruning step on those sums, then layer by layer over the survivors
+    sess.prune(3, oracle.ALLOC_ALIGN)
+    order = oracle.prune_topk(accum, order, 3, oracle.ALLOC_ALIGN)
+    assert sess.read_plan()["order"][0] == order
+    out.fill_(float("nan"))
+    for layer in range(2):
+        kw = {key: t[layer:layer + 1] for key, t in self_kv.items()}
+        cf.cf_query_prefill_attn_prefix(sess.geom, sess.batch, sess.plan, qg[layer:layer + 1], kg[layer:layer + 1],
+                                        vg[layer:layer + 1], kpg[layer:layer + 1], vpg[layer:layer + 1],
+                                        out[layer:layer + 1], sess.workspace, lse=lse[layer:layer + 1],
+                                        doc_scores=scores[layer:layer + 1], **kw)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    check(out, lse, scores, reference(order))
+    # the same through the library's stack driver: layer 1 over every document, pruning on its scores, layer 2
+    out2 = torch.full_like(qg, float("nan"))
+    lse2 = torch.full_like(lse, float("nan"))
+    scores2 = torch.full_like(scores, float("nan"))
+    sess.run_stack(qg, kg, vg, ((1, 3),), oracle.ALLOC_ALIGN, out2, lse2, None, scores2, batch_layers=False,
+                   k_prefix=kpg, v_prefix=vpg, **self_kv)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    first = reference(list(range(n)))
+    order2 = oracle.prune_topk(first[0][2], list(range(n)), 3, oracle.ALLOC_ALIGN)
+    assert sess.read_plan()["order"][0] == order2
+    check(out2, lse2, scores2, [first[0], reference(order2)[1]])
+
