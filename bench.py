@@ -35,7 +35,7 @@ METRIC = "cached KV tokens/s through reposition+query-prefill attn"
 # DRAM bytes (read + write) of one attention-kernel launch, averaged over the launches of a step, from the
 # ncu capture summarised under profiles/; quoted only while the kernel's sources still hash to `kernel_sha`.
 NCU_TRAFFIC = {("configs[2]", "layer-batched", "tcgen05"):
-               {"bytes_per_launch": 25.66e6, "kernel_sha": "a5fdc19e574e3b26", "summary": "profiles/attn_tc_kernel_workload3.md"}}
+               {"bytes_per_launch": 25.67e6, "kernel_sha": "61038b1f0faf1cea", "summary": "profiles/attn_tc_kernel_workload3.md"}}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 
@@ -615,6 +615,8 @@ def main():
     ap.add_argument("--q-len", type=int, default=0, help="variant: query rows per request (1 = the shape of a decoding step)")
     ap.add_argument("--self-block", action="store_true",
                     help="variant: every layer also attends the query tokens themselves (cf_query_prefill_attn_full)")
+    ap.add_argument("--only", default=None, choices=["reposition", "assemble", "decode", "document_prefill"],
+                    help="run one of the side measurements alone and print its JSON (profiling aid)")
     ap.add_argument("--prefix", type=int, default=0,
                     help="variant: every layer also attends a shared prefix cache of this many tokens "
                          "(cf_query_prefill_attn_prefix)")
@@ -662,6 +664,15 @@ def main():
     if args.force_simt:
         cf.cf_set_attn_path(1)
     peaks = load_peaks()
+    if args.only:
+        one = {"reposition": lambda: reposition_roofline(device, peaks),
+               "assemble": lambda: assemble_roofline(device, peaks),
+               "decode": lambda: decode_roofline(cf, device, peaks, "configs[3]-shaped final caches, one call per layer",
+                                                 28, 4, 4, 16000, 8, 1),
+               "document_prefill": lambda: docattn_roofline(cf, device, peaks)}[args.only]()
+        if rank == 0:
+            print(json.dumps(one), flush=True)
+        return
     n_reuse = {"eq6": 0, "k": cfg.n_docs, "1": 1, "k/5": max(1, cfg.n_docs // 5), "5": 5}[args.n_reuse]
 
     wl = GpuWorkload(cfg, args.seed + 7919 * rank, device, args.ring, batch_layers=not args.per_layer,
@@ -788,7 +799,7 @@ def main():
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
         t_total, tok_total, reps = 0.0, 0, 0
-        while t_total < 10.0 and reps < 8:
+        while t_total < 10.0 and reps < 24:
             dt, tk = oracle_sample(cfg, 50 + reps)
             t_total += dt
             tok_total += tk
