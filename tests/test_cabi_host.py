@@ -167,3 +167,48 @@ def test_stack_driver_checks_its_arguments_on_the_host(lib):
                             1 << 20, None) == cf.CF_ERR_INVALID_ARG
     assert lib.cf_debug_wait_timeout(ctypes.byref(geom), ctypes.byref(batch), fake, 0, None) == cf.CF_ERR_INVALID_ARG
     assert lib.cf_debug_wait_timeout(ctypes.byref(geom), ctypes.byref(batch), fake + 8, 1000, None) == cf.CF_ERR_WORKSPACE
+
+
+def test_decoding_calls_check_their_arguments_on_the_host(lib):
+    """Sizes are host arithmetic; every failing case returns before anything is launched."""
+    geom = cf.make_geom(28, 4, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256
+    need = cf.cf_decode_plan_bytes(geom, 4, 16064)
+    assert need > 0 and need % 256 == 0
+    assert cf.cf_decode_plan_bytes(geom, 8, 16064) > need                  # grows with the batch
+    assert cf.cf_decode_plan_bytes(geom, 0, 16064) == 0 and cf.cf_decode_plan_bytes(geom, 4, 0) == 0
+    one, eight = cf.cf_decode_workspace_bytes(geom, 4, 16064, 1), cf.cf_decode_workspace_bytes(geom, 4, 16064, 8)
+    assert 0 < one < eight and cf.cf_decode_workspace_bytes(geom, 4, 16064, 0) == 0
+    g = ctypes.byref(geom)
+    assert lib.cf_decode_plan(g, 4, 16064, None, 1, fake, need, None) == cf.CF_ERR_INVALID_ARG          # no row counts
+    assert lib.cf_decode_plan(g, 4, 16064, fake, 1, fake + 8, need, None) == cf.CF_ERR_WORKSPACE        # misaligned
+    assert lib.cf_decode_plan(g, 4, 16064, fake, 1, fake, need - 1, None) == cf.CF_ERR_WORKSPACE        # too small
+    assert lib.cf_decode_plan(g, 1 << 21, 16064, fake, 1, fake, need, None) == cf.CF_ERR_INVALID_ARG    # batch too large
+    assert lib.cf_decode_attn(g, 4, 16064, None, 1, fake, 0, fake, fake, 0, 0.0, fake, 0, None, fake, 1 << 20,
+                              None) == cf.CF_ERR_INVALID_ARG
+    assert lib.cf_decode_append(g, 4, 16064, 1, fake, fake, 0, fake, -1, fake, fake, 0, None, None) == cf.CF_ERR_INVALID_ARG
+    assert lib.cf_decode_append(g, 4, 16064, 1, fake + 2, fake, 0, fake, 0, fake, fake, 0, None, None) == cf.CF_ERR_INVALID_ARG
+    assert lib.cf_decode_append(g, 4, 16064, 2, fake, fake, 8, fake, 0, fake, fake, 8, None, None) == cf.CF_ERR_INVALID_ARG
+
+
+def test_prefix_call_checks_its_arguments_on_the_host(lib):
+    geom = cf.make_geom(12, 2, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256
+    batch = cf.cf_batch(1, 50, 48, 64, 48, 0, 0, 0, 8000, 2 * 128, fake, fake, fake)          # 64 positions reserved
+    g, b = ctypes.byref(geom), ctypes.byref(batch)
+    ws = cf.cf_attn_workspace_bytes_full(geom, batch, 1)
+
+    def call(prefix_len=64, k_prefix=fake, v_prefix=fake, k_self=None, v_self=None):
+        return lib.cf_query_prefill_attn_prefix(g, b, fake, 1, fake, 0, fake, fake, 0, k_prefix, v_prefix, 0, prefix_len,
+                                                k_self, v_self, 0, 0.0, fake, 0, None, None, None, fake, ws, None)
+
+    assert call(prefix_len=0) == cf.CF_ERR_INVALID_ARG
+    assert call(k_prefix=None) == cf.CF_ERR_INVALID_ARG
+    assert call(prefix_len=65) == cf.CF_ERR_INVALID_ARG                     # beyond the positions kept clear of documents
+    assert call(k_self=fake) == cf.CF_ERR_INVALID_ARG                       # keys of the query tokens without their values
+    f32 = cf.make_geom(4, 4, 64, cf.CF_F32, 4096, 1e4)                      # a geometry of the CUDA-core path
+    b32 = cf.cf_batch(1, 8, 16, 64, 16, 0, 0, 0, 256, 4 * 64, fake, fake, fake)
+    ws32 = cf.cf_attn_workspace_bytes_full(f32, b32, 1)
+    rc = lib.cf_query_prefill_attn_prefix(ctypes.byref(f32), ctypes.byref(b32), fake, 1, fake, 0, fake, fake, 0, fake, fake, 0,
+                                          64, None, None, 0, 0.0, fake, 0, None, None, None, fake, ws32, None)
+    assert rc == cf.CF_ERR_UNSUPPORTED
