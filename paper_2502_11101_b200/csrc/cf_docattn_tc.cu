@@ -79,29 +79,54 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
     q += (size_t)layer * a.q_layer_stride;
     out += (size_t)layer * a.out_layer_stride;
 
-    if (tid == 0) {
-        mbar_init(smem_u32(&bars->k_full), 1);
-        mbar_init(smem_u32(&bars->v_full), 1);
-        mbar_init(smem_u32(&bars->s_full), 1);
-        mbar_init(smem_u32(&bars->p_ready), 128);
-        mbar_init(smem_u32(&bars->o_done), 1);
-        bars->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // Keys or values of key tile i into their buffer (issued by the one thread of warp 4 that also issues the MMAs).
+    auto load = [&](int i, bool values) {
+        const KeyTile t = key_tile(i, n_prefix_tiles, a.prefix_len, row_first, n_doc_keys);
+        const int boxes = (t.len + kBoxRows - 1) / kBoxRows;
+        const CUtensorMap* map = t.doc_first < 0 ? (values ? &maps.vp[boxes - 1] : &maps.kp[boxes - 1])
+                                                 : (values ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
+        const uint32_t bar = smem_u32(values ? &bars->v_full : &bars->k_full);
+        const uint32_t dst = values ? v_base : k_base;
+        mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
+        tma_load_4d(dst, map, 0, kvh, t.row0, layer, bar);
+        tma_load_4d(dst + kHalfBytes, map, 64, kvh, t.row0, layer, bar);
+    };
+    // query rows of this CTA: every load is issued before the first is used (one round trip to memory, not thirteen)
+    constexpr int kQLoads = (kTile * 16 + kDocTcThreads - 1) / kDocTcThreads;
+    uint4 qv[kQLoads];
+#pragma unroll
+    for (int i = 0; i < kQLoads; ++i) {
+        const int idx = tid + i * kDocTcThreads;
+        const int chunk = idx & 15, r = idx >> 4;
+        qv[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < rows_here) {
+            const int row = r0 + r;
+            const int j = row / group, g = row - j * group;
+            qv[i] = __ldg(reinterpret_cast<const uint4*>(q + ((size_t)(row_first + j) * a.n_q_heads + kvh * group + g) * kD + chunk * 8));
+        }
     }
     if (warp == 4) {
+        if (lane == 0) {
+            mbar_init(smem_u32(&bars->k_full), 1);
+            mbar_init(smem_u32(&bars->v_full), 1);
+            mbar_init(smem_u32(&bars->s_full), 1);
+            mbar_init(smem_u32(&bars->p_ready), 128);
+            mbar_init(smem_u32(&bars->o_done), 1);
+            bars->abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            load(0, false);                                         // the first key and value tile travel during the set-up
+            load(0, true);
+        }
+        __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // query rows into swizzled shared memory (zero rows beyond the valid ones)
-    for (int idx = tid; idx < kTile * 16; idx += kDocTcThreads) {
+#pragma unroll
+    for (int i = 0; i < kQLoads; ++i) {
+        const int idx = tid + i * kDocTcThreads;
         const int chunk = idx & 15, r = idx >> 4;
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (r < rows_here) {
-            const int row = r0 + r;
-            const int j = row / group, g = row - j * group;
-            val = __ldg(reinterpret_cast<const uint4*>(q + ((size_t)(row_first + j) * a.n_q_heads + kvh * group + g) * kD + chunk * 8));
-        }
-        *reinterpret_cast<uint4*>(smem + (chunk >> 3) * kHalfBytes + swz(r, chunk & 7)) = val;
+        if (idx < kTile * 16) *reinterpret_cast<uint4*>(smem + (chunk >> 3) * kHalfBytes + swz(r, chunk & 7)) = qv[i];
     }
     fence_proxy_async();
     tc_fence_before();
@@ -112,17 +137,6 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
     if (warp == 4) {
         if (lane == 0) {
             // ---------------------------------------------------------- TMA loads and MMA issue
-            auto load = [&](int i, bool values) {
-                const KeyTile t = key_tile(i, n_prefix_tiles, a.prefix_len, row_first, n_doc_keys);
-                const int boxes = (t.len + kBoxRows - 1) / kBoxRows;
-                const CUtensorMap* map = t.doc_first < 0 ? (values ? &maps.vp[boxes - 1] : &maps.kp[boxes - 1])
-                                                         : (values ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
-                const uint32_t bar = smem_u32(values ? &bars->v_full : &bars->k_full);
-                const uint32_t dst = values ? v_base : k_base;
-                mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
-                tma_load_4d(dst, map, 0, kvh, t.row0, layer, bar);
-                tma_load_4d(dst + kHalfBytes, map, 64, kvh, t.row0, layer, bar);
-            };
             auto issue_s = [&](int i) -> bool {
                 const int n_keys = (key_tile(i, n_prefix_tiles, a.prefix_len, row_first, n_doc_keys).len + 15) & ~15;
                 if (!mbar_wait(smem_u32(&bars->k_full), i & 1, abort_flag)) return false;
@@ -137,8 +151,6 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
                 umma_commit(smem_u32(&bars->s_full));
                 return true;
             };
-            load(0, false);
-            load(0, true);
             bool ok = issue_s(0);
             for (int i = 0; i < n_tiles && ok; ++i) {
                 const bool more = i + 1 < n_tiles;
@@ -190,7 +202,11 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
                 tmem_ld32(s_addr + c * 32, sv);
                 tile_max = fmaxf(tile_max, chunk_max<true>(sv, vis - c * 32));
             }
-            const float m_new = fmaxf(m_run, tile_max * a.scale_log2);  // finite from the first tile on
+            // The reference maximum of a row only moves when a tile exceeds it by more than 2^8: any reference within
+            // the exponent range is exact enough, since P (bf16) and the sums (fp32) keep their relative precision,
+            // and the rescale of O below becomes rare after the first tile.
+            const float t_max = tile_max * a.scale_log2;
+            const float m_new = t_max > m_run + 8.0f ? t_max : m_run;   // finite from the first tile on
             const float alpha = fast_exp2(m_run - m_new);               // first tile: 0
             if (i > 0) {
                 ok = mbar_wait(smem_u32(&bars->o_done), (i - 1) & 1, abort_flag);   // PV(i-1) is complete
@@ -224,9 +240,7 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
             const float inv = 1.f / l_run;
             // rows leave through shared memory (the query tile: every QK^T has completed) for 256-byte stores
             unsigned char* stage = smem;
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tmem_ld32(o_addr + c * 32, o);
+            auto stage_chunk = [&](const uint32_t (&o)[32], int c) {       // 32 dims of the row: four 16-byte pieces
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
                     const int chunk = c * 4 + x;
@@ -236,10 +250,23 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, const __n
                                    pack_bf16(__uint_as_float(o[8 * x + 4]) * inv, __uint_as_float(o[8 * x + 5]) * inv),
                                    pack_bf16(__uint_as_float(o[8 * x + 6]) * inv, __uint_as_float(o[8 * x + 7]) * inv));
                 }
-            }
+            };
+            uint32_t oa[32], ob[32];                                        // the load of the next piece travels under the packing of this one
+            tmem_ld32_async(o_addr, oa);
+            tmem_ld_wait(oa);
+            tmem_ld32_async(o_addr + 32, ob);
+            stage_chunk(oa, 0);
+            tmem_ld_wait(ob);
+            tmem_ld32_async(o_addr + 64, oa);
+            stage_chunk(ob, 1);
+            tmem_ld_wait(oa);
+            tmem_ld32_async(o_addr + 96, ob);
+            stage_chunk(oa, 2);
+            tmem_ld_wait(ob);
+            stage_chunk(ob, 3);
             __syncwarp();
             const int warp_row0 = warp * 32;
-#pragma unroll 4
+#pragma unroll
             for (int x = 0; x < 16; ++x) {                              // two rows per step, 16 lanes each
                 const int rr = warp_row0 + 2 * x + (lane >> 4), chunk = lane & 15;
                 if (rr < rows_here) {
