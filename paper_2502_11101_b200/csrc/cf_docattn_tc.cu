@@ -46,22 +46,35 @@ struct DocBars {
     volatile int abort_flag;
 };
 
+// A key tile: up to 128 keys, first those of the prefix cache (rows p_row0 .. of the prefix tensors, visible to every
+// row), then those of the document (store rows d_row0 .., document tokens doc_first ..).  When the prefix length is a
+// multiple of the copy boxes' 32 rows the two parts share tiles (`joined`: the keys of an item are the sequence
+// [prefix; document tokens] cut every 128); otherwise the prefix has tiles of its own.
 struct KeyTile {
-    int row0, len, doc_first;      // doc_first: document token of the tile's first key, -1 for a prefix tile
+    int p_row0, p_len, d_row0, d_len, doc_first, len;
 };
 
-__device__ __forceinline__ KeyTile key_tile(int i, int n_prefix_tiles, int prefix_len, int row_first, int n_doc_keys) {
+__device__ __forceinline__ KeyTile key_tile(int i, bool joined, int n_prefix_tiles, int prefix_len, int row_first, int n_doc_keys) {
     KeyTile t;
-    if (i < n_prefix_tiles) {
-        t.row0 = i * kTile;
-        t.len = min(kTile, prefix_len - t.row0);
-        t.doc_first = -1;
+    if (joined) {
+        const int k0 = i * kTile;
+        t.p_row0 = k0;
+        t.p_len = max(0, min(kTile, prefix_len - k0));
+        t.doc_first = max(0, k0 - prefix_len);
+        t.d_len = max(0, min(kTile - t.p_len, n_doc_keys - t.doc_first));
+    } else if (i < n_prefix_tiles) {
+        t.p_row0 = i * kTile;
+        t.p_len = min(kTile, prefix_len - t.p_row0);
+        t.doc_first = 0;
+        t.d_len = 0;
     } else {
-        const int d0 = (i - n_prefix_tiles) * kTile;
-        t.row0 = row_first + d0;
-        t.len = min(kTile, n_doc_keys - d0);
-        t.doc_first = d0;
+        t.p_row0 = 0;
+        t.p_len = 0;
+        t.doc_first = (i - n_prefix_tiles) * kTile;
+        t.d_len = min(kTile, n_doc_keys - t.doc_first);
     }
+    t.d_row0 = row_first + t.doc_first;
+    t.len = t.p_len + t.d_len;
     return t;
 }
 
@@ -74,7 +87,7 @@ struct DocItem {
 // Shape of the item space.  An item holds whole tokens: rows_per_tile = (128 / G) * G rows, so that its query rows are one
 // box of the query tensor (G heads x 128 / G tokens) and arrive by bulk copy.
 struct DocGrid {
-    int row_tiles, total, group, n_prefix_tiles, rows_per_tile;
+    int row_tiles, total, group, n_prefix_tiles, rows_per_tile, joined, prefix_len;
 };
 
 __device__ __forceinline__ DocItem doc_item(const DocAttnArgs& a, const DocGrid& dg, int w) {
@@ -94,7 +107,8 @@ __device__ __forceinline__ DocItem doc_item(const DocAttnArgs& a, const DocGrid&
     if (it.r0 >= rows) return it;
     it.rows_here = min(dg.rows_per_tile, rows - it.r0);
     it.n_doc_keys = (it.r0 + it.rows_here - 1) / group + 1;       // document tokens 0 .. the last row's token
-    it.n_tiles = n_prefix_tiles + (it.n_doc_keys + kTile - 1) / kTile;
+    it.n_tiles = dg.joined ? (dg.prefix_len + it.n_doc_keys + kTile - 1) / kTile
+                           : n_prefix_tiles + (it.n_doc_keys + kTile - 1) / kTile;
     it.valid = true;
     return it;
 }
@@ -116,20 +130,28 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, DocGrid d
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = dg.group, n_prefix_tiles = dg.n_prefix_tiles;
+    const bool joined = dg.joined != 0;
     DocItem cur = next_item(a, dg, (int)blockIdx.x);
     if (!cur.valid) return;                                         // uniform over the CTA
 
     // Keys or values of key tile i of an item into their buffer (issued by the one thread of warp 4 that also issues the MMAs).
     auto load = [&](const DocItem& it, int i, bool values) {
-        const KeyTile t = key_tile(i, n_prefix_tiles, a.prefix_len, it.row_first, it.n_doc_keys);
-        const int boxes = (t.len + kBoxRows - 1) / kBoxRows;
-        const CUtensorMap* map = t.doc_first < 0 ? (values ? &maps.vp[boxes - 1] : &maps.kp[boxes - 1])
-                                                 : (values ? &maps.v[boxes - 1] : &maps.k[boxes - 1]);
+        const KeyTile t = key_tile(i, joined, n_prefix_tiles, a.prefix_len, it.row_first, it.n_doc_keys);
+        const int p_boxes = (t.p_len + kBoxRows - 1) / kBoxRows, d_boxes = (t.d_len + kBoxRows - 1) / kBoxRows;
         const uint32_t bar = smem_u32(values ? &bars->v_full : &bars->k_full);
         const uint32_t dst = values ? v_base : k_base;
-        mbar_expect_tx(bar, boxes * 2 * kBoxBytes);
-        tma_load_4d(dst, map, 0, it.kvh, t.row0, it.layer, bar);
-        tma_load_4d(dst + kHalfBytes, map, 64, it.kvh, t.row0, it.layer, bar);
+        mbar_expect_tx(bar, (p_boxes + d_boxes) * 2 * kBoxBytes);
+        if (p_boxes > 0) {
+            const CUtensorMap* map = values ? &maps.vp[p_boxes - 1] : &maps.kp[p_boxes - 1];
+            tma_load_4d(dst, map, 0, it.kvh, t.p_row0, it.layer, bar);
+            tma_load_4d(dst + kHalfBytes, map, 64, it.kvh, t.p_row0, it.layer, bar);
+        }
+        if (d_boxes > 0) {                                          // behind the prefix rows (a whole number of boxes)
+            const CUtensorMap* map = values ? &maps.v[d_boxes - 1] : &maps.k[d_boxes - 1];
+            const uint32_t d_dst = dst + t.p_len * 128;
+            tma_load_4d(d_dst, map, 0, it.kvh, t.d_row0, it.layer, bar);
+            tma_load_4d(d_dst + kHalfBytes, map, 64, it.kvh, t.d_row0, it.layer, bar);
+        }
     };
     // Query rows of an item (whole tokens, G heads each) into the query tile, one copy per 64-dim half.
     auto load_q = [&](const DocItem& it) {
@@ -177,7 +199,7 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, DocGrid d
             const uint32_t idesc_o = instr_desc(kD, true);
             int g = 0, n = 0;                                       // key tiles and items before the current one
             auto issue_s = [&](const DocItem& it, int i, int gi) -> bool {
-                const int n_keys = (key_tile(i, n_prefix_tiles, a.prefix_len, it.row_first, it.n_doc_keys).len + 15) & ~15;
+                const int n_keys = (key_tile(i, joined, n_prefix_tiles, a.prefix_len, it.row_first, it.n_doc_keys).len + 15) & ~15;
                 if (!mbar_wait(smem_u32(&bars->k_full), gi & 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint32_t idesc = instr_desc(n_keys, false);
@@ -204,7 +226,7 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, DocGrid d
                         load_q(nxt);
                         load(nxt, 0, false);
                     }
-                    const int n_keys = (key_tile(i, n_prefix_tiles, a.prefix_len, cur.row_first, cur.n_doc_keys).len + 15) & ~15;
+                    const int n_keys = (key_tile(i, joined, n_prefix_tiles, a.prefix_len, cur.row_first, cur.n_doc_keys).len + 15) & ~15;
                     ok = mbar_wait(smem_u32(&bars->v_full), (g + i) & 1, abort_flag) &&
                          mbar_wait(smem_u32(&bars->p_ready), (g + i) & 1, abort_flag);
                     if (!ok) break;
@@ -250,9 +272,9 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, DocGrid d
             const int token = row / group;
             float m_run = -INFINITY, l_run = 0.f;
             for (int i = 0; i < cur.n_tiles; ++i) {
-                const KeyTile t = key_tile(i, n_prefix_tiles, a.prefix_len, cur.row_first, cur.n_doc_keys);
-                // visible keys of this tile: all of a prefix tile; document tokens up to the row's own
-                const int vis = t.doc_first < 0 ? t.len : max(0, min(t.len, token - t.doc_first + 1));
+                const KeyTile t = key_tile(i, joined, n_prefix_tiles, a.prefix_len, cur.row_first, cur.n_doc_keys);
+                // visible keys of this tile: all of its prefix keys; document tokens up to the row's own
+                const int vis = t.p_len + max(0, min(t.d_len, token - t.doc_first + 1));
                 const int n_chunks = (t.len + 31) >> 5;
                 ok = mbar_wait(smem_u32(&bars->s_full), (g + i) & 1, abort_flag);
                 if (!ok) break;
@@ -392,7 +414,8 @@ docattn_tc_kernel(const __grid_constant__ DocMaps maps, DocAttnArgs a, DocGrid d
 }  // namespace
 
 bool docattn_tc_supported(const cf_geom* g, const cf_doc_batch* docs) {
-    return g->dtype == CF_BF16 && g->head_dim == 128 && docs->total_tokens > 0;
+    return g->dtype == CF_BF16 && g->head_dim == 128 && docs->total_tokens > 0 &&
+           g->n_q_heads / g->n_kv_heads <= kTile;                   // an item holds at least one whole token
 }
 
 int launch_docattn_tc(const cf_geom* g, const DocAttnArgs& a, const void* q, const void* k, const void* v,
@@ -454,7 +477,8 @@ int launch_docattn_tc(const cf_geom* g, const DocAttnArgs& a, const void* q, con
     if (configure_smem_once(configured, docattn_tc_kernel, kDocTcSmem) != CF_OK) return CF_ERR_CUDA;
     const int ctas = sm_count() > 0 ? 2 * sm_count() : 296;         // persistent: two CTAs per SM
     const unsigned grid = (unsigned)std::min<long long>(total, ctas);
-    const DocGrid dg = {(int)row_tiles, (int)total, group, (a.prefix_len + kTile - 1) / kTile, rows_per_tile};
+    const DocGrid dg = {(int)row_tiles, (int)total, group, (a.prefix_len + kTile - 1) / kTile, rows_per_tile,
+                        a.prefix_len % kBoxRows == 0 ? 1 : 0, a.prefix_len};
     docattn_tc_kernel<<<grid, kDocTcThreads, kDocTcSmem, stream>>>(maps, a, dg, static_cast<__nv_bfloat16*>(out), lse, status);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }

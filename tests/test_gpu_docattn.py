@@ -73,11 +73,12 @@ def _check(lens, n_layers, hq, hkv, d, dtype, prefix_len, scale=0.0, token_strid
 
 
 @pytest.mark.parametrize("force_simt", [False, True])
-@pytest.mark.parametrize("prefix_len", [0, 40, 130])
-@pytest.mark.parametrize("heads", [(12, 2), (4, 4)])
+@pytest.mark.parametrize("prefix_len", [0, 40, 64, 130, 160])
+@pytest.mark.parametrize("heads", [(12, 2), (4, 4), (28, 4)])
 def test_ragged_documents_bf16(heads, prefix_len, force_simt):
-    """Documents of 1, 63, 64, 65, 129 and 200 tokens behind a shared prefix of 0, 40 or 130 tokens;
-    grouped-query and multi-head geometry; both kernels of the library."""
+    """Documents of 1, 63, 64, 65, 129 and 200 tokens behind a shared prefix of 0, 40, 64, 130 or 160 tokens (a
+    prefix of a whole number of 32-row copy boxes shares key tiles with the document, any other has tiles of its own);
+    grouped-query (6 and 7 query heads per kv head: items of 126 rows) and multi-head geometry; both kernels of the library."""
     _check(RAGGED, 2, heads[0], heads[1], 128, torch.bfloat16, prefix_len, force_simt=force_simt)
 
 
