@@ -340,7 +340,8 @@ def decode_roofline(cf, device, peaks, label, n_q_heads, n_kv_heads, requests, r
 def docattn_roofline(cf, device, peaks, n_q_heads=12, n_kv_heads=2, n_docs=400, lo=128, hi=192, layers=4, prefix=64, iters=10):
     """cf_document_prefill_attn (offline cache construction, Sec. 2.2): documents shaped like the benchmark's attend a
     shared prefix and themselves under the causal mask.  Flops = 4 * head_dim * visible (row, key) pairs per query head
-    (QK^T and PV, the masked half of the square not counted)."""
+    (QK^T and PV, the masked half of the square not counted); bytes = every tensor once.  The roofline is the longer of
+    the two times: with six query heads per kv head and 64 + ~80 visible keys per row the pass is bound by memory."""
     rng = np.random.default_rng(0)
     lens = rng.integers(lo, hi + 1, size=n_docs)
     off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
@@ -371,10 +372,17 @@ def docattn_roofline(cf, device, peaks, n_q_heads=12, n_kv_heads=2, n_docs=400, 
     assert int(status.item()) == 0
     pairs = float(sum(int(n) * prefix + int(n) * (int(n) + 1) // 2 for n in lens))
     flops = 4.0 * 128 * pairs * n_q_heads * layers
-    tfs = flops / ms / 1e9
+    # algorithmic bytes: queries read and outputs written once, the documents' keys and values and the prefix cache read once
+    nbytes = float(2 * q.numel() * 2 + (k.numel() + v.numel() + kp.numel() + vp.numel()) * 2)
+    t_tensor, t_hbm = flops / (peaks["tflops"] * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)
+    tfs, gbs = flops / ms / 1e9, nbytes / ms / 1e6
+    hbm_bound = t_hbm >= t_tensor
     return {"kernel": "cf_document_prefill_attn", "workload": f"{n_docs} documents of {lo}-{hi} tokens behind a {prefix}-token "
-            f"prefix, {n_q_heads}/{n_kv_heads} heads, {layers} layers per call", "bound": "tensor", "flops_per_launch": flops,
-            "ms_per_launch": ms, "achieved": tfs, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": tfs / peaks["tflops"],
+            f"prefix, {n_q_heads}/{n_kv_heads} heads, {layers} layers per call", "bound": "hbm" if hbm_bound else "tensor",
+            "flops_per_launch": flops, "bytes_per_launch": nbytes, "ms_per_launch": ms,
+            "achieved": gbs if hbm_bound else tfs, "peak": peaks["hbm_gbs"] if hbm_bound else peaks["tflops"],
+            "unit": "GB/s" if hbm_bound else "TFLOP/s", "frac": max(t_tensor, t_hbm) / (ms * 1e-3),
+            "tflops": tfs, "tensor_frac": tfs / peaks["tflops"], "gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"],
             "tokens_per_s": total * layers / (ms * 1e-3), "peak_source": peaks["source"]}
 
 
