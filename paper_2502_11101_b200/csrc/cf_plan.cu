@@ -3,6 +3,7 @@
 // Sec. 2.5), and what the hot kernels consume: per-document rotation tables (Eq. 2 angles of
 // the delta of Eq. 5) and the list of key tiles.  One thread block per request; everything
 // runs in stream order so a layer stack needs no host round trip between layers.
+#include <algorithm>
 #include <cmath>
 
 #include "cf_common.cuh"
@@ -92,8 +93,8 @@ __device__ __forceinline__ int block_scan(int value, int* s_warp_sum, int* total
     }
     if (lane == 31) s_warp_sum[warp] = incl;
     __syncthreads();
-    if (warp == 0) {                                     // scan of the 32 warp sums
-        const int mine = s_warp_sum[lane];
+    if (warp == 0) {                                     // scan of the (at most 32) warp sums
+        const int mine = lane < (int)(blockDim.x >> 5) ? s_warp_sum[lane] : 0;
         int acc = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -136,6 +137,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
+    const int nthreads = (int)blockDim.x;               // at least the documents of any request, a multiple of 32
     const int doc0 = bv.req_doc_begin[b];
     const int n_docs = bv.req_doc_begin[b + 1] - doc0;
     if (n_docs > kMaxDocs || n_docs < 0) {
@@ -156,8 +158,8 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     const int keep_arg = (mode != 0 && keep_per_request) ? keep_per_request[b] : keep;
     const int kept_raw = (mode != 0 && tid < n_docs) ? pv.kept[doc0 + tid] : 0;    // rank tid, if there is one
     if (mode != 0 && tid < n_docs) s_all[tid] = score_accum[doc0 + tid];            // S of every document, by local id
-    for (int i = tid; i <= n_docs; i += kPlanThreads) s_row[i] = bv.doc_offsets[doc0 + i];
-    for (int i = tid; i < n_docs; i += kPlanThreads) {
+    for (int i = tid; i <= n_docs; i += nthreads) s_row[i] = bv.doc_offsets[doc0 + i];
+    for (int i = tid; i < n_docs; i += nthreads) {
         s_src[i] = bv.doc_src_start[doc0 + i];
         s_dst[i] = mode == 0 ? -1 : pv.dst_start[doc0 + i];
         s_group[i] = mode == 0 ? -1 : pv.group[doc0 + i];
@@ -168,9 +170,9 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     if (mode == 0) {
         n_kept = kept_count_in ? kept_count_in[b] : n_docs;
         n_kept = max(0, min(n_kept, n_docs));
-        for (int i = tid; i < n_docs; i += kPlanThreads) s_cnt[i] = 0;
+        for (int i = tid; i < n_docs; i += nthreads) s_cnt[i] = 0;
         __syncthreads();
-        for (int r = tid; r < n_kept; r += kPlanThreads) {
+        for (int r = tid; r < n_kept; r += nthreads) {
             int id = order ? order[doc0 + r] : r;
             if (id < 0 || id >= n_docs) {
                 raise_status(pv.status, CF_ERR_INVALID_ARG);
@@ -196,7 +198,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         __syncthreads();
         // rank by counting: how many kept documents beat this one (ties: lower id wins); eight
         // lanes share the count of one document
-        for (int r0 = 0; r0 < n_old; r0 += kPlanThreads / 8) {
+        for (int r0 = 0; r0 < n_old; r0 += nthreads / 8) {
             const int r = r0 + (tid >> 3);
             const float sc = r < n_old ? s_score[r] : 0.f;
             const int id = r < n_old ? s_ids[r] : 0;
@@ -225,21 +227,21 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         n_kept = keep_b;
         // (the clamp only matters for malformed input -- duplicate ids, NaN scores -- where two
         //  documents can claim one slot and leave another unwritten)
-        for (int r = tid; r < n_kept; r += kPlanThreads) s_ids[r] = max(0, min(s_tmp[r], n_docs - 1));
+        for (int r = tid; r < n_kept; r += nthreads) s_ids[r] = max(0, min(s_tmp[r], n_docs - 1));
         __syncthreads();
     }
 
     // ---- documents that are not kept ----------------------------------------------------------
     const bool reallocate = (mode == 0) || (strategy != CF_ALLOC_NONE);
-    for (int i = tid; i < n_docs; i += kPlanThreads) s_flag[i] = 0;
+    for (int i = tid; i < n_docs; i += nthreads) s_flag[i] = 0;
     __syncthreads();
-    for (int r = tid; r < n_kept; r += kPlanThreads) s_flag[s_ids[r]] = 1;
+    for (int r = tid; r < n_kept; r += nthreads) s_flag[s_ids[r]] = 1;
     __syncthreads();
 
     // ---- positional allocation ----------------------------------------------------------------
     if (reallocate && n_kept > 0) {
         int longest = 0;
-        for (int r = tid; r < n_kept; r += kPlanThreads) longest = max(longest, s_row[s_ids[r] + 1] - s_row[s_ids[r]]);
+        for (int r = tid; r < n_kept; r += nthreads) longest = max(longest, s_row[s_ids[r] + 1] - s_row[s_ids[r]]);
         atomicMax(&s_longest, longest);
         __syncthreads();
         longest = s_longest;
@@ -324,7 +326,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         s_cnt[id] = my_tiles;
     }
     __syncthreads();
-    for (int i = tid; i < n_docs; i += kPlanThreads) {
+    for (int i = tid; i < n_docs; i += nthreads) {
         const bool kept = s_flag[i] != 0;
         pv.dst_start[doc0 + i] = kept ? s_dst[i] : -1;
         pv.group[doc0 + i] = kept ? s_group[i] : -1;
@@ -332,7 +334,7 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
         pv.doc_tile_count[doc0 + i] = kept ? s_cnt[i] : 0;
     }
     if (tid < n_kept) pv.kept[doc0 + tid] = s_ids[tid];
-    for (int x = tid; x < total; x += kPlanThreads) {
+    for (int x = tid; x < total; x += nthreads) {
         int lo = 0, hi = n_kept;                             // last rank whose first tile is <= x
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -352,12 +354,12 @@ plan_kernel(GeomView gv, BatchView bv, PlanView pv, InvFreq inv_freq, int mode, 
     }
 
     // ---- rotation tables: cos, sin of (dst - src) * theta^(-2p/D) -------------------------------
-    // thread = (slice p, every (kPlanThreads / half)-th rank): the frequency is read once per thread
+    // thread = (slice p, every (nthreads / half)-th rank): the frequency is read once per thread
     {
         const int p = tid & (half - 1);
         const unsigned long long turns = inv_freq.turns[p];
         const double freq = inv_freq.f[p];
-        for (int r = tid >> half_log2; r < n_kept; r += kPlanThreads >> half_log2) {
+        for (int r = tid >> half_log2; r < n_kept; r += nthreads >> half_log2) {
             const int id = s_ids[r];
             const int delta = s_dst[id] - s_src[id];
             float2 entry;
@@ -394,7 +396,9 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
         const long double turn = (long double)inv_freq.f[p] / (2.0L * 3.14159265358979323846264338327950288L);
         inv_freq.turns[p] = (unsigned long long)ldexpl(turn, 64);          // < 2^62: theta > 1 keeps f <= 1
     }
-    plan_kernel<<<bv.n_requests, kPlanThreads, 0, stream>>>(gv, bv, pv, inv_freq, mode, order, kept_count,
+    // one thread per document of a request, a block no larger than that needs: its barriers and scans cost less
+    const int threads = std::min(kPlanThreads, std::max(128, (std::min(bv.n_docs_total, kMaxDocs) + 31) / 32 * 32));
+    plan_kernel<<<bv.n_requests, threads, 0, stream>>>(gv, bv, pv, inv_freq, mode, order, kept_count,
                                                            query_start, score_accum, keep,
                                                            keep_per_request, strategy);
     return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
