@@ -252,6 +252,30 @@ int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, con
                                  float* lse, float* doc_scores, float* score_accum,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* One layer at a time with the document scores deferred (Algorithm 2 uses S only where it prunes: S <- S + s^l of
+ * the layers since the last cut can be added together right before the next one).  For a running model, whose
+ * layers come one by one: cf_query_prefill_attn_slot is cf_query_prefill_attn for one layer without doc_scores and
+ * score_accum -- it leaves the layer's per-tile and per-row log-sum-exps in slot `slot` of the workspace --, and
+ * cf_accumulate_scores then does for slots 0 .. n_filled-1 what the attention calls would have done: doc_scores[i] =
+ * s of slot i (optional), S <- S + s in slot order (the per-layer calls' values up to the rounding of fp32 sums
+ * taken in another order; run-to-run identical).  Between the first slot
+ * call and cf_accumulate_scores the plan must not change (no cf_prune_topk), and every slot 0 .. n_filled-1 must
+ * have been filled; the slot calls of one workspace must not overlap on the device (they share its partial-result
+ * buffers).  One launch chain of two kernels per layer instead of three.
+ *   slot, n_slots   0 <= slot < n_slots <= CF_MAX_LAYERS_PER_CALL, n_slots * n_requests <= 65535; n_slots is the
+ *                   capacity the workspace is laid out for, the same in every call of the group
+ *   n_filled        1 .. n_slots: slots to score
+ *   workspace       at least cf_attn_workspace_bytes_slots(geom, batch, n_slots) bytes, the same buffer in every call
+ *   doc_scores      device float [n_filled][n_docs_total] or NULL;  score_accum  device float [n_docs_total] or NULL
+ * Errors as cf_query_prefill_attn. */
+size_t cf_attn_workspace_bytes_slots(const cf_geom* geom, const cf_batch* batch, int32_t n_slots);
+int cf_query_prefill_attn_slot(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t slot,
+                               int32_t n_slots, const void* q, const void* k_cache, const void* v_cache,
+                               float softmax_scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                               void* stream);
+int cf_accumulate_scores(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t n_filled, int32_t n_slots,
+                         float* doc_scores, float* score_accum, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The whole attention of the query tokens in layer_l (Algorithm 2): over the kept documents' caches
  * as in cf_query_prefill_attn_layers, and over the query tokens themselves under the causal mask
  * that the footnote to Eq. 1 refers to (query row j sees query tokens 0..j), merged into one softmax.
@@ -434,9 +458,11 @@ typedef struct cf_stack {
                                      happens after that layer's scores are accumulated                */
     const int32_t* prune_keep;    /* host [n_prune]: documents kept per request from then on          */
     int32_t strategy;             /* CF_ALLOC_NONE | CF_ALLOC_ALIGN | CF_ALLOC_SORT                   */
-    int32_t batch_layers;         /* 0: one attention launch chain per layer; 1: one per run of layers
-                                     between two pruning layers (same results up to the tolerance of
-                                     the split-KV merge)                                              */
+    int32_t batch_layers;         /* 0: one attention launch chain per layer (without k_self and prefix
+                                     the layers' scores wait in workspace slots and are added to S before
+                                     each pruning layer: cf_query_prefill_attn_slot, cf_accumulate_scores);
+                                     1: one chain per run of layers between two pruning layers (same
+                                     results up to the tolerance of the split-KV merge)               */
     float   softmax_scale;        /* 0 selects 1/sqrt(head_dim)                                       */
     int32_t reserved;
     const void* q;                /* [n_layers][n_requests][q_len][n_q_heads][head_dim]               */

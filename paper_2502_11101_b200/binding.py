@@ -25,11 +25,13 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcachefoc
 EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf_plan_layout_of",
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
+           "cf_attn_workspace_bytes_slots", "cf_query_prefill_attn_slot", "cf_accumulate_scores",
            "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_query_prefill_attn_prefix", "cf_assemble_final_cache", "cf_merge_attn",
            "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
            "cf_run_stack", "cf_document_prefill_attn", "cf_decode_plan_bytes", "cf_decode_plan", "cf_decode_status",
            "cf_decode_workspace_bytes", "cf_decode_attn", "cf_decode_append", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
 _SIZE_T_EXPORTS = ("cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers", "cf_attn_workspace_bytes_full",
+                   "cf_attn_workspace_bytes_slots",
                    "cf_run_stack_workspace_bytes", "cf_decode_plan_bytes", "cf_decode_workspace_bytes")
 
 
@@ -113,6 +115,11 @@ def load_library() -> ctypes.CDLL:
     lib.cf_attn_workspace_bytes_layers.argtypes = [gp, bp, i32]
     lib.cf_query_prefill_attn_layers.argtypes = [gp, bp, vp, i32, vp, i64, vp, vp, i64, ctypes.c_float, vp, i64,
                                                  vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.cf_attn_workspace_bytes_slots.restype = ctypes.c_size_t
+    lib.cf_attn_workspace_bytes_slots.argtypes = [gp, bp, i32]
+    lib.cf_query_prefill_attn_slot.argtypes = [gp, bp, vp, i32, i32, vp, vp, vp, ctypes.c_float, vp, vp, vp,
+                                               ctypes.c_size_t, vp]
+    lib.cf_accumulate_scores.argtypes = [gp, bp, vp, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_assemble_final_cache.argtypes = [gp, bp, vp, i32, i64, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cf_merge_attn.argtypes = [gp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.cf_attn_workspace_bytes_full.restype = ctypes.c_size_t
@@ -285,6 +292,33 @@ def cf_query_prefill_attn_layers(geom: cf_geom, batch: cf_batch, plan: torch.Ten
         _ptr(lse), _ptr(doc_scores), _ptr(score_accum), workspace.data_ptr(),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn_layers")
+
+
+def cf_attn_workspace_bytes_slots(geom: cf_geom, batch: cf_batch, n_slots: int) -> int:
+    return int(load_library().cf_attn_workspace_bytes_slots(ctypes.byref(geom), ctypes.byref(batch), n_slots))
+
+
+def cf_query_prefill_attn_slot(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, slot: int, n_slots: int,
+                               q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+                               workspace: torch.Tensor, lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                               stream=None) -> None:
+    """One layer (tensors as in cf_query_prefill_attn) whose document scores are left for cf_accumulate_scores."""
+    rc = load_library().cf_query_prefill_attn_slot(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), slot, n_slots, q.data_ptr(), k_cache.data_ptr(),
+        v_cache.data_ptr(), softmax_scale, out.data_ptr(), _ptr(lse), workspace.data_ptr(),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn_slot")
+
+
+def cf_accumulate_scores(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, n_filled: int, n_slots: int,
+                         workspace: torch.Tensor, doc_scores: Optional[torch.Tensor] = None,
+                         score_accum: Optional[torch.Tensor] = None, stream=None) -> None:
+    """`doc_scores` [n_filled, n_docs_total] (contiguous) and / or `score_accum` [n_docs_total]."""
+    assert doc_scores is None or (doc_scores.shape[0] == n_filled and doc_scores.is_contiguous())
+    rc = load_library().cf_accumulate_scores(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), n_filled, n_slots, _ptr(doc_scores), _ptr(score_accum),
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_accumulate_scores")
 
 
 def cf_assemble_final_cache(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, k_cache: torch.Tensor,

@@ -172,9 +172,10 @@ int choose_splits(const cf_geom* g, const cf_batch* b, int n_layers) {
 }
 
 size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, int n_layers, bool with_self,
-                             AttnWorkspace* ws, void* base_ptr) {
+                             AttnWorkspace* ws, void* base_ptr, int part_layers) {
     const size_t rows = (size_t)g->n_q_heads * b->q_len;
-    const size_t nlb = (size_t)b->n_requests * (size_t)n_layers;
+    const size_t nlb = (size_t)b->n_requests * (size_t)(part_layers > 0 ? part_layers : n_layers);   // layers of partial results
+    const size_t nlb_lse = (size_t)b->n_requests * (size_t)n_layers;
     const size_t max_tiles = (size_t)b->n_docs_total + (size_t)(b->total_tokens / kTile) + 1;
     char* base = static_cast<char*>(base_ptr);
     size_t off = 0;
@@ -187,7 +188,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
     size_t m = take(nlb * n_splits * rows);
     size_t l = take(nlb * n_splits * rows);
     size_t t = take((size_t)n_layers * max_tiles * rows);
-    size_t r = take(nlb * rows);
+    size_t r = take(nlb_lse * rows);
     size_t so = 0, sm = 0, sl = 0, ld = 0;
     if (with_self) {                                  // behind everything else: the rest of the layout does not move
         so = take(nlb * rows * g->head_dim);
@@ -247,9 +248,13 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t s, const void* k_prefix, const void* v_prefix,
-                    long long prefix_stride, int prefix_len) {
+                    long long prefix_stride, int prefix_len, int slot, int n_slots) {
     int rc = check_plan(geom, batch, plan);
     if (rc != CF_OK) return rc;
+    const bool slotted = slot >= 0;                   // one layer into slot `slot` of n_slots, scored later
+    if (slotted && (span.n_layers != 1 || n_slots <= 0 || n_slots > CF_MAX_LAYERS_PER_CALL || slot >= n_slots ||
+                    doc_scores || score_accum || (long long)n_slots * batch->n_requests > 65535))
+        return CF_ERR_INVALID_ARG;
     if (!q || !k_cache || !v_cache || !out || !workspace) return CF_ERR_INVALID_ARG;
     if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return CF_ERR_INVALID_ARG;
     if (span.n_layers <= 0 || span.n_layers > CF_MAX_LAYERS_PER_CALL ||
@@ -283,8 +288,15 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     }
     const int n_splits = choose_splits(geom, batch, span.n_layers);
     AttnWorkspace ws;
-    const size_t need = attn_workspace_layout(geom, batch, n_splits, span.n_layers, with_self || with_prefix, &ws, workspace);
+    const size_t need = slotted ? attn_workspace_layout(geom, batch, n_splits, n_slots, with_self || with_prefix, &ws, workspace, 1)
+                                : attn_workspace_layout(geom, batch, n_splits, span.n_layers, with_self || with_prefix, &ws, workspace);
     if (workspace_bytes < need) return CF_ERR_WORKSPACE;
+    if (slotted) {                                    // this call sees its slot as the one layer it has
+        const size_t rows_total = (size_t)geom->n_q_heads * batch->q_len;
+        ws.tile_lse2 += (size_t)slot * ws.max_tiles * rows_total;
+        ws.row_lse2 += (size_t)slot * batch->n_requests * rows_total;
+        ws.n_layers = 1;
+    }
     const float scale = softmax_scale == 0.0f ? 1.0f / std::sqrt((float)geom->head_dim) : softmax_scale;
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
     const bool tensor_core = g_attn_path.load() == 0 && attn_tc_supported(geom, batch);
@@ -553,6 +565,37 @@ int cf_query_prefill_attn_layers(const cf_geom* geom, const cf_batch* batch, con
     const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
     return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, nullptr, nullptr, 0, softmax_scale, out, lse,
                            doc_scores, score_accum, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t cf_attn_workspace_bytes_slots(const cf_geom* geom, const cf_batch* batch, int32_t n_slots) {
+    if (!batch || validate(geom, batch) != CF_OK || n_slots <= 0 || n_slots > CF_MAX_LAYERS_PER_CALL) return 0;
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), n_slots, false, nullptr, nullptr, 1);
+}
+
+int cf_query_prefill_attn_slot(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t slot,
+                               int32_t n_slots, const void* q, const void* k_cache, const void* v_cache,
+                               float softmax_scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+    if (slot < 0) return CF_ERR_INVALID_ARG;
+    const LayerSpan span = {1, 0, 0, 0};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, nullptr, nullptr, 0, softmax_scale, out, lse,
+                           nullptr, nullptr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), nullptr, nullptr,
+                           0, 0, slot, n_slots);
+}
+
+int cf_accumulate_scores(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t n_filled, int32_t n_slots,
+                         float* doc_scores, float* score_accum, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_plan(geom, batch, plan);
+    if (rc != CF_OK) return rc;
+    if (n_slots <= 0 || n_slots > CF_MAX_LAYERS_PER_CALL || n_filled <= 0 || n_filled > n_slots || !workspace)
+        return CF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return CF_ERR_WORKSPACE;
+    AttnWorkspace ws;
+    const size_t need = attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), n_slots, false, &ws, workspace, 1);
+    if (workspace_bytes < need) return CF_ERR_WORKSPACE;
+    ws.n_layers = n_filled;
+    return launch_scores(geom, batch, make_plan_view(geom, batch, const_cast<void*>(plan)), ws, doc_scores, score_accum,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const void* plan,

@@ -456,6 +456,11 @@ int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
         rc = g->head_dim == 128 ? launch_combine_typed<float, 128>(g, b, span, ws, out, lse, stream)
                                 : launch_combine_typed<float, 64>(g, b, span, ws, out, lse, stream);
     if (rc != CF_OK) return rc;
+    return launch_scores(g, b, pv, ws, doc_scores, score_accum, stream);
+}
+
+int launch_scores(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws, float* doc_scores,
+                  float* score_accum, cudaStream_t stream) {
     if (b->n_docs_total > 0 && (doc_scores || score_accum)) {
         score_kernel<<<(unsigned)b->n_docs_total, kScoreThreads, 0, stream>>>(make_batch_view(b), pv, ws,
                                                                    g->n_q_heads * b->q_len, doc_scores,

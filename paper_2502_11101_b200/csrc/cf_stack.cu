@@ -80,6 +80,13 @@ int max_docs_per_request(const cf_batch* b, const cf_stack* st) {
     return worst;
 }
 
+// With one attention call per layer and nothing but documents to attend, the layers' document scores are
+// left in slots of the workspace and added to S together: right before a pruning layer uses S, when the
+// slots are full, and after the last layer (cf_query_prefill_attn_slot, cf_accumulate_scores).
+constexpr int kScoreSlots = 8;
+bool deferred_scores(const cf_stack* st) { return !st->batch_layers && !st->k_self && st->prefix_len == 0; }
+int score_slots(const cf_stack* st) { return std::min(kScoreSlots, st->n_layers); }
+
 int check_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* st) {
     if (!batch || !st) return CF_ERR_INVALID_ARG;
     int rc = validate(geom, batch);
@@ -109,7 +116,8 @@ size_t cf_run_stack_workspace_bytes(const cf_geom* geom, const cf_batch* batch, 
         local.tiles_hint = live_tiles_hint(batch, stack, keep);
         const int m = c.last - c.first;
         need = std::max(need, (stack->k_self || stack->prefix_len > 0) ? cf_attn_workspace_bytes_full(geom, &local, m)
-                                            : cf_attn_workspace_bytes_layers(geom, &local, m));
+                              : deferred_scores(stack) ? cf_attn_workspace_bytes_slots(geom, &local, score_slots(stack))
+                                                       : cf_attn_workspace_bytes_layers(geom, &local, m));
         if (c.prune_after >= 0) keep = std::min(keep, stack->prune_keep[c.prune_after]);
     }
     return need;
@@ -139,6 +147,9 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
     if (rc != CF_OK) return rc;
 
     // Phase 1: layer_l (attention over the kept caches, S += s^l), pruning and re-allocation at the scheduled layers
+    const bool deferred = deferred_scores(stack);
+    const int n_slots = score_slots(stack);
+    int filled = 0;                                                 // layers whose scores wait in the workspace
     for (const Call& c : calls_of(stack)) {
         const int m = c.last - c.first;
         const char* q = static_cast<const char*>(stack->q) + (size_t)c.first * stack->q_layer_stride * esize;
@@ -163,6 +174,17 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
                                             ks, vs, stack->self_layer_stride, stack->softmax_scale, out,
                                             stack->out_layer_stride, lse, scores, stack->score_accum, workspace,
                                             workspace_bytes, stream);
+        } else if (deferred) {
+            rc = cf_query_prefill_attn_slot(geom, &local, plan, filled, n_slots, q, k, v, stack->softmax_scale, out, lse,
+                                            workspace, workspace_bytes, stream);
+            if (rc != CF_OK) return rc;
+            ++filled;
+            if (c.prune_after >= 0 || filled == n_slots || c.last == stack->n_layers) {
+                float* first = stack->layer_scores ? stack->layer_scores + (size_t)(c.last - filled) * nd : nullptr;
+                rc = cf_accumulate_scores(geom, &local, plan, filled, n_slots, first, stack->score_accum, workspace,
+                                          workspace_bytes, stream);
+                filled = 0;
+            }
         } else {
             rc = cf_query_prefill_attn_layers(geom, &local, plan, m, q, stack->q_layer_stride, k, v,
                                               stack->kv_layer_stride, stack->softmax_scale, out, stack->out_layer_stride,

@@ -162,12 +162,22 @@ class Session:
                     self.prune(sched[last], strategy)
                 first = last
         else:
+            n_slots, filled = min(8, n_layers), 0            # as cf_run_stack: the layers' scores wait in workspace slots
+            if k_self is None:
+                need = B.cf_attn_workspace_bytes_slots(self.geom, self.batch, n_slots)
+                if need > self.workspace.numel():
+                    self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
             for layer in range(1, n_layers + 1):
                 i = layer - 1
                 if k_self is None:
-                    self.attend(q[i], k[i], v[i], out[i], None if lse is None else lse[i], softmax_scale)
-                    if layer_scores is not None:
-                        layer_scores[i].copy_(self.doc_scores)
+                    B.cf_query_prefill_attn_slot(self.geom, self.batch, self.plan, filled, n_slots, q[i], k[i], v[i], out[i],
+                                                 self.workspace, None if lse is None else lse[i], softmax_scale)
+                    filled += 1
+                    if layer in sched or filled == n_slots or layer == n_layers:
+                        B.cf_accumulate_scores(self.geom, self.batch, self.plan, filled, n_slots, self.workspace,
+                                               None if layer_scores is None else layer_scores[layer - filled:layer],
+                                               self.score_accum)
+                        filled = 0
                 else:
                     self.attend_layers(q[i:i + 1], k[i:i + 1], v[i:i + 1], out[i:i + 1],
                                        None if lse is None else lse[i:i + 1],

@@ -150,7 +150,8 @@ def test_stack_driver_checks_its_arguments_on_the_host(lib):
     per_call = [cf.cf_attn_workspace_bytes_layers(geom, batch, m) for m in (4, 8)]
     assert cf.cf_run_stack_workspace_bytes(geom, batch, good) == max(per_call) > 0
     one_by_one, keep2 = stack([4, 12, 20], [25, 12, 6], batch_layers=0)
-    assert cf.cf_run_stack_workspace_bytes(geom, batch, one_by_one) == cf.cf_attn_workspace_bytes(geom, batch)
+    # one call per layer: partial results of one layer, the scores of up to eight layers waiting in slots
+    assert cf.cf_run_stack_workspace_bytes(geom, batch, one_by_one) == cf.cf_attn_workspace_bytes_slots(geom, batch, 8)
     # document lengths on the host let the call shrink its grids to the documents still kept
     lens = np.full(50, 160, np.int32)
     begin = np.array([0, 50], np.int32)
@@ -212,3 +213,20 @@ def test_prefix_call_checks_its_arguments_on_the_host(lib):
     rc = lib.cf_query_prefill_attn_prefix(ctypes.byref(f32), ctypes.byref(b32), fake, 1, fake, 0, fake, fake, 0, fake, fake, 0,
                                           64, None, None, 0, 0.0, fake, 0, None, None, None, fake, ws32, None)
     assert rc == cf.CF_ERR_UNSUPPORTED
+
+
+def test_deferred_score_calls_check_their_arguments_on_the_host(lib):
+    geom = cf.make_geom(12, 2, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256
+    batch = cf.cf_batch(1, 50, 48, 0, 48, 0, 0, 0, 8000, 2 * 128, fake, fake, fake)
+    g, b = ctypes.byref(geom), ctypes.byref(batch)
+    one, eight = cf.cf_attn_workspace_bytes_slots(geom, batch, 1), cf.cf_attn_workspace_bytes_slots(geom, batch, 8)
+    assert cf.cf_attn_workspace_bytes(geom, batch) == one < eight                  # partial results of one layer only
+    assert cf.cf_attn_workspace_bytes_slots(geom, batch, 0) == 0 and cf.cf_attn_workspace_bytes_slots(geom, batch, 65) == 0
+    slot = lambda s, n, bytes_=eight: lib.cf_query_prefill_attn_slot(g, b, fake, s, n, fake, fake, fake, 0.0, fake, None,
+                                                                      fake, bytes_, None)
+    assert slot(-1, 8) == cf.CF_ERR_INVALID_ARG and slot(8, 8) == cf.CF_ERR_INVALID_ARG and slot(0, 0) == cf.CF_ERR_INVALID_ARG
+    assert slot(0, 8, eight - 1) == cf.CF_ERR_WORKSPACE
+    acc = lambda f, n, bytes_=eight: lib.cf_accumulate_scores(g, b, fake, f, n, None, fake, fake, bytes_, None)
+    assert acc(0, 8) == cf.CF_ERR_INVALID_ARG and acc(9, 8) == cf.CF_ERR_INVALID_ARG and acc(1, 65) == cf.CF_ERR_INVALID_ARG
+    assert acc(8, 8, eight - 1) == cf.CF_ERR_WORKSPACE

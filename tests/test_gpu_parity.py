@@ -203,6 +203,59 @@ def test_layer_batched_call_is_reproducible_and_agrees_with_single_layer_calls()
     assert torch.allclose(acc_a, s_a.sum(0), rtol=1e-5) and torch.allclose(acc_a, acc_b, rtol=1e-3)
 
 
+@pytest.mark.parametrize("which", ["config3", "ragged-f32-d64"])
+def test_deferred_document_scores_equal_the_per_layer_calls(which):
+    """cf_query_prefill_attn_slot + cf_accumulate_scores against cf_query_prefill_attn layer by layer: the same outputs
+    bit for bit, the same per-layer scores and S up to the rounding of fp32 sums taken in another order (five layers in
+    four slots: two groups, the second partly filled);
+    the per-layer calls themselves are compared with the oracle by the stack tests."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    if which == "config3":
+        cfg = W.scaled_config(W.CONFIGS[3], n_layers=5, n_docs=20, schedule=())
+    else:
+        cfg = W.WorkloadConfig("ragged", 5, 8, 2, 64, "f32", 1e4, 4096, 7, 5, 70, 5, 1, 2, ())   # CUDA-core kernels
+    meta = W.make_meta(cfg, 1)
+    q = W.make_q(meta).cuda()
+    k, v = [t.cuda() for t in W.make_kv(meta)]
+    n_slots, nd = 4, meta.n_docs_total
+    runs = []
+    for mode in ("single", "slots"):
+        sess = Session(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.torch_dtype, cfg.pos_range, cfg.rope_theta,
+                       cfg.q_len, meta.doc_len, meta.req_doc_begin, meta.doc_src_start, tail_reserve=cfg.q_len)
+        sess.init()
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((5, cfg.batch, cfg.n_q_heads, cfg.q_len), float("nan"), device="cuda")
+        scores = torch.full((5, nd), float("nan"), device="cuda")
+        if mode == "single":
+            for i in range(5):
+                sess.attend(q[i], k[i], v[i], out[i], lse[i])
+                scores[i].copy_(sess.doc_scores)
+        else:
+            work = torch.empty(cf.cf_attn_workspace_bytes_slots(sess.geom, sess.batch, n_slots), dtype=torch.uint8, device="cuda")
+            work.fill_(0xFF)                                             # nothing in it needs zeroing
+            for first in (0, 4):
+                filled = min(n_slots, 5 - first)
+                for i in range(filled):
+                    cf.cf_query_prefill_attn_slot(sess.geom, sess.batch, sess.plan, i, n_slots, q[first + i], k[first + i],
+                                                  v[first + i], out[first + i], work, lse[first + i])
+                cf.cf_accumulate_scores(sess.geom, sess.batch, sess.plan, filled, n_slots, work,
+                                        scores[first:first + filled], sess.score_accum)
+        torch.cuda.synchronize()
+        assert sess.status() == 0
+        runs.append([t.float().cpu() for t in (out, lse, scores, sess.score_accum)])
+    for i, (a, b) in enumerate(zip(*runs)):
+        assert not torch.isnan(a).any() and not torch.isnan(b).any()
+        if i < 2:
+            assert torch.equal(a, b)                                     # outputs and log-sum-exps: the same kernels
+        else:                                                            # a layer's rows are summed by a quarter of the block
+            assert torch.allclose(a, b, rtol=1e-5, atol=1e-9)
+    with pytest.raises(cf.CacheFocusError):                              # a slot beyond the capacity
+        cf.cf_query_prefill_attn_slot(sess.geom, sess.batch, sess.plan, 4, n_slots, q[0], k[0], v[0], out[0], work)
+    with pytest.raises(cf.CacheFocusError):                              # more slots to score than there are
+        cf.cf_accumulate_scores(sess.geom, sess.batch, sess.plan, 5, n_slots, work, None, sess.score_accum)
+
+
 def test_interleaved_slice_layout():
     import paper_2502_11101_b200 as cf
     from paper_2502_11101_b200.session import Session
