@@ -35,7 +35,7 @@ METRIC = "cached KV tokens/s through reposition+query-prefill attn"
 # DRAM bytes (read + write) of one attention-kernel launch, averaged over the launches of a step, from the
 # ncu capture summarised under profiles/; quoted only while the kernel's sources still hash to `kernel_sha`.
 NCU_TRAFFIC = {("configs[2]", "layer-batched", "tcgen05"):
-               {"bytes_per_launch": 25.65e6, "kernel_sha": "a5ac1ee831f8b3ff", "summary": "profiles/attn_tc_kernel_workload3.md"}}
+               {"bytes_per_launch": 25.65e6, "kernel_sha": "5e8cbfebacd3ff26", "summary": "profiles/attn_tc_kernel_workload3.md"}}
 UNIT = "tokens/s"
 STRATEGY_ALIGN = 1
 

@@ -212,6 +212,7 @@ size_t attn_workspace_layout(const cf_geom* g, const cf_batch* b, int n_splits, 
         ws->self_l = with_self ? reinterpret_cast<float*>(base + sl) : nullptr;
         ws->part_ld = with_self ? reinterpret_cast<float*>(base + ld) : nullptr;
         ws->self_mode = 0;
+        ws->keys_in_place = 0;
     }
     return off;
 }
@@ -248,7 +249,7 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     const void* v_self, long long self_stride, float softmax_scale,
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t s, const void* k_prefix, const void* v_prefix,
-                    long long prefix_stride, int prefix_len, int slot, int n_slots) {
+                    long long prefix_stride, int prefix_len, int slot, int n_slots, bool keys_in_place) {
     int rc = check_plan(geom, batch, plan);
     if (rc != CF_OK) return rc;
     const bool slotted = slot >= 0;                   // one layer into slot `slot` of n_slots, scored later
@@ -311,6 +312,7 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     cudaEvent_t ev_start, ev_stop;
     const bool timed = prof_claim(&ev_start, &ev_stop) >= 0;
     if (timed) cudaEventRecord(ev_start, s);
+    ws.keys_in_place = keys_in_place ? 1 : 0;
     if (tensor_core) {
         ws.part_bf16 = 1;
         ws.self_mode = (with_self || with_prefix) ? 2 : 0;   // the blocks ride along as further key tiles

@@ -116,7 +116,9 @@ __device__ __forceinline__ int ring_div(int x, bool six) { return six ? x / 6 : 
 // Loads of one kind (keys or values) a stage has received before the one of tile `it`.
 __device__ __forceinline__ int ring_uses(int it, bool six) { return six ? it / 3 : it / 5; }
 
-template <int LAYOUT>
+// ROTATE = false: every document sits where it was cached (the final caches of a decoding step), so the keys go from
+// the copy straight to the tensor cores and the rotation warps stay idle.
+template <int LAYOUT, bool ROTATE>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                BatchView bv, PlanView pv, AttnWorkspace ws, long long q_layer_stride, int n_q_heads, int n_kv_heads,
@@ -309,7 +311,7 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
             auto issue_s = [&](int n) -> bool {
                 const int w = n & 1;
                 const int n_keys = keys_of(ck.tile);
-                if (!mbar_wait(bar_k_ready + ck.stage * 8, ck.parity, abort_flag)) return false;
+                if (!mbar_wait(ROTATE ? bar_k_ready + ck.stage * 8 : bar_kv_full + ck.stage * 16, ck.parity, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t a0 = w ? a_desc1 : a_desc0;
                 const uint64_t b0 = bk_desc + (uint64_t)(ck.stage * (kTileBytes >> 4));
@@ -353,6 +355,8 @@ attn_tc_kernel(const __grid_constant__ StoreMaps maps,
                 if (ok && n + 2 < n_seq) ok = issue_s(n + 2);
             }
         }
+    } else if (warp >= 8 && !ROTATE) {
+        // keys are used as cached: nothing to do
     } else if (warp >= 8) {
         // ------------------------------------------------------------------ key rotation (Eq. 5)
         const int t = warp < 12 ? tid - 256 : tid - 320;            // 0..191 (warps 8-11, 14, 15)
@@ -685,7 +689,7 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
     dim3 grid((unsigned)(ws.n_splits / 2), (unsigned)(g->n_kv_heads * row_groups),
               (unsigned)(b->n_requests * span.n_layers));
     BatchView bv = make_batch_view(b);
-    static PerDeviceOnce configured[2];
+    static PerDeviceOnce configured[3];
     auto run = [&](auto kernel, int which) {
         if (configure_smem_once(configured[which], kernel, kSmemBytes) != CF_OK) return CF_ERR_CUDA;
         kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, bv, pv, ws, span.q_stride, g->n_q_heads,
@@ -693,8 +697,9 @@ int launch_attn_tc(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                                                        k_self ? 1 : 0, prefix_len);
         return cudaGetLastError() == cudaSuccess ? CF_OK : CF_ERR_CUDA;
     };
-    if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF>, 0);
-    return run(attn_tc_kernel<CF_ROPE_INTERLEAVED>, 1);
+    if (ws.keys_in_place) return run(attn_tc_kernel<CF_ROPE_HALF, false>, 2);      // the slice layout plays no part
+    if (g->rope_layout == CF_ROPE_HALF) return run(attn_tc_kernel<CF_ROPE_HALF, true>, 0);
+    return run(attn_tc_kernel<CF_ROPE_INTERLEAVED, true>, 1);
 }
 
 }  // namespace cf

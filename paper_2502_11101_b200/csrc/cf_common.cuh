@@ -105,6 +105,7 @@ struct AttnWorkspace {
     float* self_l;     // [L*B][Hq*Lq]
     float* part_ld;    // [L*B][n_splits][Hq*Lq]    like part_l, the documents' keys only (self_mode 2)
     int self_mode;
+    int keys_in_place; // every document's destination equals its source (decoding over final caches): no rotation
 };
 // part_layers > 0: the partial results (and the further key blocks' buffers) are sized for that many layers only, the
 // per-tile and per-row log-sum-exps for n_layers (calls that fill one layer slot at a time and score the slots later).
@@ -151,7 +152,7 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
                     void* out, float* lse, float* doc_scores, float* score_accum, void* workspace,
                     size_t workspace_bytes, cudaStream_t stream, const void* k_prefix = nullptr,
                     const void* v_prefix = nullptr, long long prefix_stride = 0, int prefix_len = 0, int slot = -1,
-                    int n_slots = 0);
+                    int n_slots = 0, bool keys_in_place = false);
 // Document scores of the layers held in a workspace: doc_scores[l] = s^l (optional), S += s^l in layer order.
 int launch_scores(const cf_geom* g, const cf_batch* b, const PlanView& pv, const AttnWorkspace& ws, float* doc_scores,
                   float* score_accum, cudaStream_t stream);

@@ -192,7 +192,8 @@ int cf_decode_attn(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, 
     const LayerSpan span = {n_layers, q_layer_stride, kv_layer_stride, out_layer_stride};
     return run_attn_layers(&g, &b, static_cast<const char*>(decode_plan) + a.bytes, span, q, k_final, v_final, nullptr,
                            nullptr, 0, softmax_scale, out, lse, nullptr, nullptr, workspace, workspace_bytes,
-                           static_cast<cudaStream_t>(stream));
+                           static_cast<cudaStream_t>(stream), nullptr, nullptr, 0, 0, -1, 0,
+                           /*keys_in_place=*/true);           // the final caches are used where they lie
 }
 
 int cf_decode_append(const cf_geom* geom, int32_t n_requests, int32_t cache_rows, int32_t n_layers,
