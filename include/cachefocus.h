@@ -307,8 +307,8 @@ int cf_query_prefill_attn_full(const cf_geom* geom, const cf_batch* batch, const
  *                   (the positions the allocation keeps clear of documents)
  *   k_self, v_self  as in cf_query_prefill_attn_full, or both NULL: documents and prefix only
  *   workspace       at least cf_attn_workspace_bytes_full(geom, batch, n_layers) bytes
- * Built for bf16 storage with head_dim 128 (the tensor-core kernel); other geometries return
- * CF_ERR_UNSUPPORTED and join a prefix through a call of its own and cf_merge_attn. */
+ * With bf16 storage and head_dim 128 the prefix rides along as key tiles of the tensor-core kernel; other geometries
+ * compute it (and the query-self block) as one more part of the split-KV merge on the CUDA cores. */
 int cf_query_prefill_attn_prefix(const cf_geom* geom, const cf_batch* batch, const void* plan,
                                  int32_t n_layers, const void* q, int64_t q_layer_stride,
                                  const void* k_cache, const void* v_cache, int64_t kv_layer_stride,

@@ -302,11 +302,11 @@ int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan
     PlanView pv = make_plan_view(geom, batch, const_cast<void*>(plan));
     const bool tensor_core = g_attn_path.load() == 0 && attn_tc_supported(geom, batch);
     if (with_self && batch->q_len > CF_TILE_TOKENS) return CF_ERR_UNSUPPORTED;
-    if (with_prefix && !tensor_core) return CF_ERR_UNSUPPORTED;   // the CUDA-core path joins a prefix through cf_merge_attn
     if (!tensor_core) ws.part_ld = nullptr;           // only the tensor-core kernel reports per-part document sums
-    if (with_self && !tensor_core) {                  // the CUDA-core path computes the block as a part of its own
+    if ((with_self || with_prefix) && !tensor_core) { // the CUDA-core path computes these blocks as a part of their own
         ws.self_mode = 1;
-        rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, scale * kLog2e, ws, s);
+        rc = launch_self_block(geom, batch, span, self_stride, q, k_self, v_self, k_prefix, v_prefix, prefix_stride,
+                               prefix_len, scale * kLog2e, ws, s);
         if (rc != CF_OK) return rc;
     }
     cudaEvent_t ev_start, ev_stop;

@@ -143,8 +143,9 @@ int launch_combine(const cf_geom* g, const cf_batch* b, const PlanView& pv, cons
                    const AttnWorkspace& ws, void* out, float* lse, float* doc_scores,
                    float* score_accum, cudaStream_t stream);
 int launch_self_block(const cf_geom* g, const cf_batch* b, const LayerSpan& span, long long self_stride,
-                      const void* q, const void* k_self, const void* v_self, float scale_log2,
-                      const AttnWorkspace& ws, cudaStream_t stream);
+                      const void* q, const void* k_self, const void* v_self, const void* k_prefix, const void* v_prefix,
+                      long long prefix_stride, int prefix_len, float scale_log2, const AttnWorkspace& ws,
+                      cudaStream_t stream);
 // Shared body of the attention entry points (k_self = v_self = null: cached documents only).
 int run_attn_layers(const cf_geom* geom, const cf_batch* batch, const void* plan, const LayerSpan& span,
                     const void* q, const void* k_cache, const void* v_cache, const void* k_self,

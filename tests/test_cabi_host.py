@@ -207,12 +207,6 @@ def test_prefix_call_checks_its_arguments_on_the_host(lib):
     assert call(k_prefix=None) == cf.CF_ERR_INVALID_ARG
     assert call(prefix_len=65) == cf.CF_ERR_INVALID_ARG                     # beyond the positions kept clear of documents
     assert call(k_self=fake) == cf.CF_ERR_INVALID_ARG                       # keys of the query tokens without their values
-    f32 = cf.make_geom(4, 4, 64, cf.CF_F32, 4096, 1e4)                      # a geometry of the CUDA-core path
-    b32 = cf.cf_batch(1, 8, 16, 64, 16, 0, 0, 0, 256, 4 * 64, fake, fake, fake)
-    ws32 = cf.cf_attn_workspace_bytes_full(f32, b32, 1)
-    rc = lib.cf_query_prefill_attn_prefix(ctypes.byref(f32), ctypes.byref(b32), fake, 1, fake, 0, fake, fake, 0, fake, fake, 0,
-                                          64, None, None, 0, 0.0, fake, 0, None, None, None, fake, ws32, None)
-    assert rc == cf.CF_ERR_UNSUPPORTED
 
 
 def test_deferred_score_calls_check_their_arguments_on_the_host(lib):

@@ -717,6 +717,25 @@ def test_decoding_step_over_the_assembled_final_cache():
     (128, 3, (4, 4), True),          # a full prefix tile, fewer document tiles than parts
 ])
 def test_pinned_prefix_attended_inside_the_call(prefix, q_len, heads, with_self):
+    _pinned_prefix_case(prefix, q_len, heads, with_self)
+
+
+@pytest.mark.parametrize("prefix,q_len,heads,with_self", [
+    (40, 6, (8, 2), False),          # a prefix alone: one chunk of keys
+    (200, 48, (12, 2), True),        # two chunks of prefix keys, then the causal chunk of the query tokens
+    (128, 3, (4, 4), True),          # a full chunk
+])
+def test_pinned_prefix_on_the_cuda_core_path(prefix, q_len, heads, with_self):
+    """The same cases through the CUDA-core kernels: prefix and query-self block are one more part of the merge."""
+    import paper_2502_11101_b200 as cf
+    cf.cf_set_attn_path(1)
+    try:
+        _pinned_prefix_case(prefix, q_len, heads, with_self)
+    finally:
+        cf.cf_set_attn_path(0)
+
+
+def _pinned_prefix_case(prefix, q_len, heads, with_self):
     """cf_query_prefill_attn_prefix: the shared prefix cache rides along as further key tiles (delta 0, seen by
     every query row), with or without the causal query-self block behind it; one softmax over prefix, kept
     documents and query tokens in the oracle.  Document scores stay those of the documents alone, pruning
