@@ -195,15 +195,15 @@ class GpuWorkload:
         # (on the tensor-core path the block is a key tile of the attention kernel, not a launch)
         per_call = 4 if self.self_kernel else 3
         prunes = sum(1 for l, _ in cfg.schedule if l <= cfg.n_layers)
-        if not self.batch_layers and self.self_kv[0][0] is None and self.prefix_kv is None:
-            # one call per layer, documents only: the stack driver leaves the layers' scores in up to eight workspace
+        if not self.batch_layers:
+            # one call per layer: the stack driver leaves the layers' scores in up to eight workspace
             # slots and adds them to S with one launch before each pruning layer, when the slots are full and at the end
             cuts, slots, groups, filled = {l for l, _ in cfg.schedule}, min(8, cfg.n_layers), 0, 0
             for layer in range(1, cfg.n_layers + 1):
                 filled += 1
                 if layer in cuts or filled == slots or layer == cfg.n_layers:
                     groups, filled = groups + 1, 0
-            return 2 + 2 * cfg.n_layers + groups + prunes + 1
+            return 2 + (per_call - 1) * cfg.n_layers + groups + prunes + 1
         return 2 + per_call * len(self.calls()) + prunes + 1
 
 

@@ -275,6 +275,17 @@ int cf_query_prefill_attn_slot(const cf_geom* geom, const cf_batch* batch, const
                                void* stream);
 int cf_accumulate_scores(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t n_filled, int32_t n_slots,
                          float* doc_scores, float* score_accum, void* workspace, size_t workspace_bytes, void* stream);
+/* The slot call with the key blocks besides the documents (one layer of cf_query_prefill_attn_prefix without the
+ * scores): a shared prefix cache (prefix_len > 0; k_prefix, v_prefix [prefix_len][n_kv_heads][head_dim]) and / or the
+ * query tokens' own keys and values (k_self, v_self [n_requests][q_len][n_kv_heads][head_dim]; both NULL: none); at
+ * least one of the two.  Its workspace is larger (cf_attn_workspace_bytes_slots_full); cf_accumulate_scores reads
+ * either kind. */
+size_t cf_attn_workspace_bytes_slots_full(const cf_geom* geom, const cf_batch* batch, int32_t n_slots);
+int cf_query_prefill_attn_slot_full(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t slot,
+                                    int32_t n_slots, const void* q, const void* k_cache, const void* v_cache,
+                                    const void* k_prefix, const void* v_prefix, int32_t prefix_len, const void* k_self,
+                                    const void* v_self, float softmax_scale, void* out, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream);
 
 /* The whole attention of the query tokens in layer_l (Algorithm 2): over the kept documents' caches
  * as in cf_query_prefill_attn_layers, and over the query tokens themselves under the causal mask
@@ -458,9 +469,9 @@ typedef struct cf_stack {
                                      happens after that layer's scores are accumulated                */
     const int32_t* prune_keep;    /* host [n_prune]: documents kept per request from then on          */
     int32_t strategy;             /* CF_ALLOC_NONE | CF_ALLOC_ALIGN | CF_ALLOC_SORT                   */
-    int32_t batch_layers;         /* 0: one attention launch chain per layer (without k_self and prefix
-                                     the layers' scores wait in workspace slots and are added to S before
-                                     each pruning layer: cf_query_prefill_attn_slot, cf_accumulate_scores);
+    int32_t batch_layers;         /* 0: one attention launch chain per layer (the layers' scores wait in
+                                     workspace slots and are added to S before each pruning layer:
+                                     cf_query_prefill_attn_slot[_full], cf_accumulate_scores);
                                      1: one chain per run of layers between two pruning layers (same
                                      results up to the tolerance of the split-KV merge)               */
     float   softmax_scale;        /* 0 selects 1/sqrt(head_dim)                                       */

@@ -26,12 +26,13 @@ EXPORTS = ["cf_error_string", "cf_allocate_positions", "cf_schedule_linear", "cf
            "cf_plan_init", "cf_plan_status", "cf_reposition_keys", "cf_attn_workspace_bytes",
            "cf_attn_workspace_bytes_layers", "cf_query_prefill_attn", "cf_query_prefill_attn_layers",
            "cf_attn_workspace_bytes_slots", "cf_query_prefill_attn_slot", "cf_accumulate_scores",
+           "cf_attn_workspace_bytes_slots_full", "cf_query_prefill_attn_slot_full",
            "cf_attn_workspace_bytes_full", "cf_query_prefill_attn_full", "cf_query_prefill_attn_prefix", "cf_assemble_final_cache", "cf_merge_attn",
            "cf_query_prefill_attn_static", "cf_prune_topk", "cf_prune_topk_host", "cf_run_stack_workspace_bytes",
            "cf_run_stack", "cf_document_prefill_attn", "cf_decode_plan_bytes", "cf_decode_plan", "cf_decode_status",
            "cf_decode_workspace_bytes", "cf_decode_attn", "cf_decode_append", "cf_set_attn_path", "cf_profile_begin", "cf_profile_end", "cf_debug_wait_timeout"]
 _SIZE_T_EXPORTS = ("cf_attn_workspace_bytes", "cf_attn_workspace_bytes_layers", "cf_attn_workspace_bytes_full",
-                   "cf_attn_workspace_bytes_slots",
+                   "cf_attn_workspace_bytes_slots", "cf_attn_workspace_bytes_slots_full",
                    "cf_run_stack_workspace_bytes", "cf_decode_plan_bytes", "cf_decode_workspace_bytes")
 
 
@@ -120,6 +121,10 @@ def load_library() -> ctypes.CDLL:
     lib.cf_query_prefill_attn_slot.argtypes = [gp, bp, vp, i32, i32, vp, vp, vp, ctypes.c_float, vp, vp, vp,
                                                ctypes.c_size_t, vp]
     lib.cf_accumulate_scores.argtypes = [gp, bp, vp, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.cf_attn_workspace_bytes_slots_full.restype = ctypes.c_size_t
+    lib.cf_attn_workspace_bytes_slots_full.argtypes = [gp, bp, i32]
+    lib.cf_query_prefill_attn_slot_full.argtypes = [gp, bp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp, ctypes.c_float,
+                                                    vp, vp, vp, ctypes.c_size_t, vp]
     lib.cf_assemble_final_cache.argtypes = [gp, bp, vp, i32, i64, vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cf_merge_attn.argtypes = [gp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.cf_attn_workspace_bytes_full.restype = ctypes.c_size_t
@@ -308,6 +313,26 @@ def cf_query_prefill_attn_slot(geom: cf_geom, batch: cf_batch, plan: torch.Tenso
         v_cache.data_ptr(), softmax_scale, out.data_ptr(), _ptr(lse), workspace.data_ptr(),
         workspace.numel() * workspace.element_size(), _stream(stream))
     _check(rc, "cf_query_prefill_attn_slot")
+
+
+def cf_attn_workspace_bytes_slots_full(geom: cf_geom, batch: cf_batch, n_slots: int) -> int:
+    return int(load_library().cf_attn_workspace_bytes_slots_full(ctypes.byref(geom), ctypes.byref(batch), n_slots))
+
+
+def cf_query_prefill_attn_slot_full(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, slot: int, n_slots: int,
+                                    q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+                                    workspace: torch.Tensor, k_prefix: Optional[torch.Tensor] = None,
+                                    v_prefix: Optional[torch.Tensor] = None, k_self: Optional[torch.Tensor] = None,
+                                    v_self: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                                    softmax_scale: float = 0.0, stream=None) -> None:
+    """One layer with a prefix cache `k_prefix`, `v_prefix` [P, Hkv, D] and / or the query tokens' own `k_self`,
+    `v_self` [B, Lq, Hkv, D]; document scores left for cf_accumulate_scores."""
+    rc = load_library().cf_query_prefill_attn_slot_full(
+        ctypes.byref(geom), ctypes.byref(batch), plan.data_ptr(), slot, n_slots, q.data_ptr(), k_cache.data_ptr(),
+        v_cache.data_ptr(), _ptr(k_prefix), _ptr(v_prefix), 0 if k_prefix is None else k_prefix.shape[0], _ptr(k_self),
+        _ptr(v_self), softmax_scale, out.data_ptr(), _ptr(lse), workspace.data_ptr(),
+        workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "cf_query_prefill_attn_slot_full")
 
 
 def cf_accumulate_scores(geom: cf_geom, batch: cf_batch, plan: torch.Tensor, n_filled: int, n_slots: int,

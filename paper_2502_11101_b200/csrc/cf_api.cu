@@ -585,6 +585,25 @@ int cf_query_prefill_attn_slot(const cf_geom* geom, const cf_batch* batch, const
                            0, 0, slot, n_slots);
 }
 
+size_t cf_attn_workspace_bytes_slots_full(const cf_geom* geom, const cf_batch* batch, int32_t n_slots) {
+    if (!batch || validate(geom, batch) != CF_OK || n_slots <= 0 || n_slots > CF_MAX_LAYERS_PER_CALL) return 0;
+    return attn_workspace_layout(geom, batch, choose_splits(geom, batch, 1), n_slots, true, nullptr, nullptr, 1);
+}
+
+int cf_query_prefill_attn_slot_full(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t slot,
+                                    int32_t n_slots, const void* q, const void* k_cache, const void* v_cache,
+                                    const void* k_prefix, const void* v_prefix, int32_t prefix_len, const void* k_self,
+                                    const void* v_self, float softmax_scale, void* out, float* lse, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+    if (slot < 0 || prefix_len < 0 || (prefix_len == 0 && !k_self) || (k_self == nullptr) != (v_self == nullptr))
+        return CF_ERR_INVALID_ARG;
+    const LayerSpan span = {1, 0, 0, 0};
+    return run_attn_layers(geom, batch, plan, span, q, k_cache, v_cache, k_self, v_self, 0, softmax_scale, out, lse,
+                           nullptr, nullptr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                           prefix_len > 0 ? k_prefix : nullptr, prefix_len > 0 ? v_prefix : nullptr, 0, prefix_len, slot,
+                           n_slots);
+}
+
 int cf_accumulate_scores(const cf_geom* geom, const cf_batch* batch, const void* plan, int32_t n_filled, int32_t n_slots,
                          float* doc_scores, float* score_accum, void* workspace, size_t workspace_bytes, void* stream) {
     int rc = check_plan(geom, batch, plan);

@@ -80,11 +80,11 @@ int max_docs_per_request(const cf_batch* b, const cf_stack* st) {
     return worst;
 }
 
-// With one attention call per layer and nothing but documents to attend, the layers' document scores are
+// With one attention call per layer the layers' document scores are
 // left in slots of the workspace and added to S together: right before a pruning layer uses S, when the
 // slots are full, and after the last layer (cf_query_prefill_attn_slot, cf_accumulate_scores).
 constexpr int kScoreSlots = 8;
-bool deferred_scores(const cf_stack* st) { return !st->batch_layers && !st->k_self && st->prefix_len == 0; }
+bool deferred_scores(const cf_stack* st) { return !st->batch_layers; }
 int score_slots(const cf_stack* st) { return std::min(kScoreSlots, st->n_layers); }
 
 int check_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* st) {
@@ -115,9 +115,12 @@ size_t cf_run_stack_workspace_bytes(const cf_geom* geom, const cf_batch* batch, 
     for (const Call& c : calls_of(stack)) {
         local.tiles_hint = live_tiles_hint(batch, stack, keep);
         const int m = c.last - c.first;
-        need = std::max(need, (stack->k_self || stack->prefix_len > 0) ? cf_attn_workspace_bytes_full(geom, &local, m)
-                              : deferred_scores(stack) ? cf_attn_workspace_bytes_slots(geom, &local, score_slots(stack))
-                                                       : cf_attn_workspace_bytes_layers(geom, &local, m));
+        const bool blocks = stack->k_self || stack->prefix_len > 0;
+        need = std::max(need, deferred_scores(stack)
+                                  ? (blocks ? cf_attn_workspace_bytes_slots_full(geom, &local, score_slots(stack))
+                                            : cf_attn_workspace_bytes_slots(geom, &local, score_slots(stack)))
+                                  : (blocks ? cf_attn_workspace_bytes_full(geom, &local, m)
+                                            : cf_attn_workspace_bytes_layers(geom, &local, m)));
         if (c.prune_after >= 0) keep = std::min(keep, stack->prune_keep[c.prune_after]);
     }
     return need;
@@ -158,7 +161,25 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
         char* out = static_cast<char*>(stack->out) + (size_t)c.first * stack->out_layer_stride * esize;
         float* lse = stack->lse ? stack->lse + (size_t)c.first * lse_layer : nullptr;
         float* scores = stack->layer_scores ? stack->layer_scores + (size_t)c.first * nd : nullptr;
-        if (stack->prefix_len > 0) {
+        if (deferred) {
+            const char* ks = stack->k_self ? static_cast<const char*>(stack->k_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
+            const char* vs = stack->v_self ? static_cast<const char*>(stack->v_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
+            const char* kp = stack->prefix_len > 0 ? static_cast<const char*>(stack->k_prefix) + (size_t)c.first * stack->prefix_layer_stride * esize : nullptr;
+            const char* vp = stack->prefix_len > 0 ? static_cast<const char*>(stack->v_prefix) + (size_t)c.first * stack->prefix_layer_stride * esize : nullptr;
+            rc = (ks || kp) ? cf_query_prefill_attn_slot_full(geom, &local, plan, filled, n_slots, q, k, v, kp, vp,
+                                                              stack->prefix_len, ks, vs, stack->softmax_scale, out, lse,
+                                                              workspace, workspace_bytes, stream)
+                            : cf_query_prefill_attn_slot(geom, &local, plan, filled, n_slots, q, k, v, stack->softmax_scale,
+                                                         out, lse, workspace, workspace_bytes, stream);
+            if (rc != CF_OK) return rc;
+            ++filled;
+            if (c.prune_after >= 0 || filled == n_slots || c.last == stack->n_layers) {
+                float* first = stack->layer_scores ? stack->layer_scores + (size_t)(c.last - filled) * nd : nullptr;
+                rc = cf_accumulate_scores(geom, &local, plan, filled, n_slots, first, stack->score_accum, workspace,
+                                          workspace_bytes, stream);
+                filled = 0;
+            }
+        } else if (stack->prefix_len > 0) {
             const char* ks = stack->k_self ? static_cast<const char*>(stack->k_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
             const char* vs = stack->v_self ? static_cast<const char*>(stack->v_self) + (size_t)c.first * stack->self_layer_stride * esize : nullptr;
             const char* kp = static_cast<const char*>(stack->k_prefix) + (size_t)c.first * stack->prefix_layer_stride * esize;
@@ -174,17 +195,6 @@ int cf_run_stack(const cf_geom* geom, const cf_batch* batch, const cf_stack* sta
                                             ks, vs, stack->self_layer_stride, stack->softmax_scale, out,
                                             stack->out_layer_stride, lse, scores, stack->score_accum, workspace,
                                             workspace_bytes, stream);
-        } else if (deferred) {
-            rc = cf_query_prefill_attn_slot(geom, &local, plan, filled, n_slots, q, k, v, stack->softmax_scale, out, lse,
-                                            workspace, workspace_bytes, stream);
-            if (rc != CF_OK) return rc;
-            ++filled;
-            if (c.prune_after >= 0 || filled == n_slots || c.last == stack->n_layers) {
-                float* first = stack->layer_scores ? stack->layer_scores + (size_t)(c.last - filled) * nd : nullptr;
-                rc = cf_accumulate_scores(geom, &local, plan, filled, n_slots, first, stack->score_accum, workspace,
-                                          workspace_bytes, stream);
-                filled = 0;
-            }
         } else {
             rc = cf_query_prefill_attn_layers(geom, &local, plan, m, q, stack->q_layer_stride, k, v,
                                               stack->kv_layer_stride, stack->softmax_scale, out, stack->out_layer_stride,

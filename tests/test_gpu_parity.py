@@ -256,6 +256,57 @@ def test_deferred_document_scores_equal_the_per_layer_calls(which):
         cf.cf_accumulate_scores(sess.geom, sess.batch, sess.plan, 5, n_slots, work, None, sess.score_accum)
 
 
+@pytest.mark.parametrize("simt", [False, True])
+def test_deferred_scores_with_prefix_and_query_self_block(simt):
+    """cf_query_prefill_attn_slot_full + cf_accumulate_scores against cf_query_prefill_attn_prefix layer by layer
+    (three layers in two slots; a 40-token prefix and the causal block of the query tokens): the same outputs bit for
+    bit, scores and S up to fp32 rounding.  Both kernel families."""
+    import paper_2502_11101_b200 as cf
+    from paper_2502_11101_b200.session import Session
+    hq, hkv, d, q_len, prefix, n_layers = 8, 2, 128, 20, 40, 3
+    lens = np.array([130, 64, 17, 96, 200], dtype=np.int32)
+    n = len(lens)
+    gen = torch.Generator().manual_seed(9)
+    rnd = lambda *shape: torch.randn(shape, generator=gen).bfloat16().cuda()
+    q, k, v = rnd(n_layers, 1, q_len, hq, d), rnd(n_layers, int(lens.sum()), hkv, d), rnd(n_layers, int(lens.sum()), hkv, d)
+    kp, vp = rnd(n_layers, prefix, hkv, d), rnd(n_layers, prefix, hkv, d)
+    ks, vs = rnd(n_layers, 1, q_len, hkv, d), rnd(n_layers, 1, q_len, hkv, d)
+    cf.cf_set_attn_path(1 if simt else 0)
+    try:
+        runs = []
+        for mode in ("calls", "slots"):
+            sess = Session(hq, hkv, d, torch.bfloat16, 4096, 1e4, q_len, lens, np.array([0, n], dtype=np.int32),
+                           np.full(n, prefix, dtype=np.int32), tail_reserve=q_len, prefix_len=prefix)
+            sess.init()
+            out = torch.full_like(q, float("nan"))
+            lse = torch.full((n_layers, 1, hq, q_len), float("nan"), device="cuda")
+            scores = torch.full((n_layers, n), float("nan"), device="cuda")
+            if mode == "calls":
+                sess.reserve_workspace(1, with_self=True)
+                for i in range(n_layers):
+                    cf.cf_query_prefill_attn_prefix(sess.geom, sess.batch, sess.plan, q[i:i + 1], k[i:i + 1], v[i:i + 1],
+                                                    kp[i:i + 1], vp[i:i + 1], out[i:i + 1], sess.workspace, lse=lse[i:i + 1],
+                                                    doc_scores=scores[i:i + 1], score_accum=sess.score_accum,
+                                                    k_self=ks[i:i + 1], v_self=vs[i:i + 1])
+            else:
+                work = torch.empty(cf.cf_attn_workspace_bytes_slots_full(sess.geom, sess.batch, 2), dtype=torch.uint8, device="cuda")
+                for first, filled in ((0, 2), (2, 1)):
+                    for i in range(filled):
+                        l = first + i
+                        cf.cf_query_prefill_attn_slot_full(sess.geom, sess.batch, sess.plan, i, 2, q[l], k[l], v[l], out[l], work,
+                                                           k_prefix=kp[l], v_prefix=vp[l], k_self=ks[l], v_self=vs[l], lse=lse[l])
+                    cf.cf_accumulate_scores(sess.geom, sess.batch, sess.plan, filled, 2, work, scores[first:first + filled],
+                                            sess.score_accum)
+            torch.cuda.synchronize()
+            assert sess.status() == 0
+            runs.append([t.float().cpu() for t in (out, lse, scores, sess.score_accum)])
+    finally:
+        cf.cf_set_attn_path(0)
+    for i, (a, b) in enumerate(zip(*runs)):
+        assert not torch.isnan(a).any() and not torch.isnan(b).any()
+        assert torch.equal(a, b) if i < 2 else torch.allclose(a, b, rtol=1e-5, atol=1e-9)
+
+
 def test_interleaved_slice_layout():
     import paper_2502_11101_b200 as cf
     from paper_2502_11101_b200.session import Session
