@@ -224,3 +224,23 @@ def test_deferred_score_calls_check_their_arguments_on_the_host(lib):
     acc = lambda f, n, bytes_=eight: lib.cf_accumulate_scores(g, b, fake, f, n, None, fake, fake, bytes_, None)
     assert acc(0, 8) == cf.CF_ERR_INVALID_ARG and acc(9, 8) == cf.CF_ERR_INVALID_ARG and acc(1, 65) == cf.CF_ERR_INVALID_ARG
     assert acc(8, 8, eight - 1) == cf.CF_ERR_WORKSPACE
+
+
+def test_slot_call_with_further_key_blocks_checks_its_arguments_on_the_host(lib):
+    geom = cf.make_geom(12, 2, 128, cf.CF_BF16, 32768, 1e6)
+    fake = 256
+    batch = cf.cf_batch(1, 50, 48, 64, 48, 0, 0, 0, 8000, 2 * 128, fake, fake, fake)          # 64 positions kept for a prefix
+    g, b = ctypes.byref(geom), ctypes.byref(batch)
+    plain, full = cf.cf_attn_workspace_bytes_slots(geom, batch, 4), cf.cf_attn_workspace_bytes_slots_full(geom, batch, 4)
+    assert 0 < plain < full and cf.cf_attn_workspace_bytes_slots_full(geom, batch, 0) == 0
+
+    def call(slot=0, n_slots=4, k_prefix=fake, prefix_len=64, k_self=fake, v_self=fake, nbytes=full):
+        return lib.cf_query_prefill_attn_slot_full(g, b, fake, slot, n_slots, fake, fake, fake, k_prefix, fake, prefix_len,
+                                                   k_self, v_self, 0.0, fake, None, fake, nbytes, None)
+
+    assert call(prefix_len=0, k_self=None, v_self=None) == cf.CF_ERR_INVALID_ARG      # neither block: the plain slot call
+    assert call(v_self=None) == cf.CF_ERR_INVALID_ARG                                 # keys of the query tokens without values
+    assert call(prefix_len=65) == cf.CF_ERR_INVALID_ARG                               # beyond the positions kept clear
+    assert call(k_prefix=None) == cf.CF_ERR_INVALID_ARG
+    assert call(slot=4) == cf.CF_ERR_INVALID_ARG and call(prefix_len=-1) == cf.CF_ERR_INVALID_ARG
+    assert call(nbytes=full - 1) == cf.CF_ERR_WORKSPACE
