@@ -33,7 +33,8 @@ def _inputs(seed, lens, n_layers, hq, hkv, d, dtype, prefix_len):
     return q, k, v, kp, vp
 
 
-def _check(lens, n_layers, hq, hkv, d, dtype, prefix_len, scale=0.0, token_stride=None, seed=0, force_simt=False):
+def _check(lens, n_layers, hq, hkv, d, dtype, prefix_len, scale=0.0, token_stride=None, seed=0, force_simt=False,
+           sample=None):
     q, k, v, kp, vp = _inputs(seed, lens, n_layers, hq, hkv, d, dtype, prefix_len)
     off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
     total = int(off[-1])
@@ -58,8 +59,11 @@ def _check(lens, n_layers, hq, hkv, d, dtype, prefix_len, scale=0.0, token_strid
     assert int(status[0]) == 0
     o_got, l_got = out.float().cpu().numpy(), lse.cpu().numpy()
     tight = dtype == torch.float32
+    assert not np.isnan(o_got).any() and not np.isnan(l_got).any()      # every row of every document was written
     for l in range(n_layers):
         for i, n_tok in enumerate(lens):
+            if sample is not None and (l, i) not in sample:
+                continue
             a, b = int(off[i]), int(off[i + 1])
             o_ref, lse_ref = oracle.document_prefill_attn(
                 q[l, a:b].double().numpy(), k[l, a:b].double().numpy(), v[l, a:b].double().numpy(),
@@ -124,3 +128,14 @@ def test_empty_batch_and_argument_errors():
         raise cf.CacheFocusError(rc, "cf_document_prefill_attn")
     assert e.value.code == cf.CF_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+def test_bench_sized_batch_sampled():
+    """The batch bench.py times (400 passages of 128-192 tokens behind a 64-token prefix, 12/2 heads, four layers: each
+    persistent CTA walks some ninety work items), a dozen (layer, document) pairs compared with the oracle, every
+    output checked to have been written."""
+    rng = np.random.default_rng(0)
+    lens = [int(x) for x in rng.integers(128, 193, size=400)]
+    picks = {(int(l), int(i)) for l, i in zip(rng.integers(0, 4, size=12), rng.integers(0, 400, size=12))}
+    picks |= {(0, 0), (3, 399), (1, int(np.argmax(lens))), (2, int(np.argmin(lens)))}
+    _check(lens, 4, 12, 2, 128, torch.bfloat16, 64, seed=4, sample=picks)
