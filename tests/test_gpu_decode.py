@@ -115,3 +115,42 @@ def test_decode_calls_report_a_full_slot():
     assert bool(torch.all(k_fin[0, 0, 10] == 1)) and float(k_fin[0, 1].abs().sum()) == 0.0   # the full slot was skipped
     with pytest.raises(cf.CacheFocusError):
         cf.cf_decode_plan(geom, B, cache_rows, rows, 1, plan[: plan.numel() // 2])
+
+
+@pytest.mark.parametrize("layers_per_call", [1, 2])
+def test_bench_sized_caches_one_step(layers_per_call):
+    """Caches of the size bench.py times for decoding (28 query / 4 kv heads, four requests with up to 16 000 rows in
+    use: every CTA walks tens of full key tiles), ragged fill levels, one appended token; every (layer, request) against
+    the oracle."""
+    L, B, hq, hkv, d, cache_rows = 2, 4, 28, 4, 128, 16064
+    geom = cf.make_geom(hq, hkv, d, cf.CF_BF16, 32768, 1e6)
+    used = np.array([16000, 15001, 9000, 127], dtype=np.int32)
+    gen = torch.Generator().manual_seed(11)
+    k_fin = torch.randn((L, B, cache_rows, hkv, d), generator=gen).bfloat16()
+    v_fin = torch.randn((L, B, cache_rows, hkv, d), generator=gen).bfloat16()
+    q_new = torch.randn((L, B, hq, d), generator=gen).bfloat16()
+    k_new = torch.randn((L, B, hkv, d), generator=gen).bfloat16()
+    v_new = torch.randn((L, B, hkv, d), generator=gen).bfloat16()
+    kg, vg, rows = k_fin.cuda(), v_fin.cuda(), torch.from_numpy(used).cuda()
+    plan = torch.zeros(cf.cf_decode_plan_bytes(geom, B, cache_rows), dtype=torch.uint8, device="cuda")
+    work = torch.empty(cf.cf_decode_workspace_bytes(geom, B, cache_rows, layers_per_call), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((L, B, hq, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((L, B, hq), float("nan"), device="cuda")
+    cf.cf_decode_append(geom, B, cache_rows, kg, vg, rows, 0, k_new.cuda(), v_new.cuda(), status)
+    cf.cf_decode_plan(geom, B, cache_rows, rows, 1, plan)
+    qg = q_new.cuda()
+    for l0 in range(0, L, layers_per_call):
+        l1 = l0 + layers_per_call
+        cf.cf_decode_attn(geom, B, cache_rows, plan, qg[l0:l1], kg[l0:l1], vg[l0:l1], out[l0:l1], work, lse[l0:l1])
+    torch.cuda.synchronize()
+    assert cf.cf_decode_status(geom, B, cache_rows, plan) == 0 and int(status.item()) == 0
+    for l in range(L):
+        for b in range(B):
+            n = int(used[b])
+            o_ref, lse_ref = oracle.decode_steps(k_fin[l, b, :n].double().numpy(), v_fin[l, b, :n].double().numpy(),
+                                                 q_new[l, b][None].double().numpy(), k_new[l, b][None].double().numpy(),
+                                                 v_new[l, b][None].double().numpy())
+            got = out[l, b].float().cpu().numpy()
+            assert np.all(np.abs(got - o_ref[0]) <= 1e-2 + 2e-2 * np.abs(o_ref[0])), (l, b)
+            assert np.all(np.abs(lse[l, b].cpu().numpy() - lse_ref[0]) <= 1e-2), (l, b)
