@@ -396,8 +396,9 @@ int launch_plan(const GeomView& gv, const BatchView& bv, const PlanView& pv, int
         const long double turn = (long double)inv_freq.f[p] / (2.0L * 3.14159265358979323846264338327950288L);
         inv_freq.turns[p] = (unsigned long long)ldexpl(turn, 64);          // < 2^62: theta > 1 keeps f <= 1
     }
-    // one thread per document of a request, a block no larger than that needs: its barriers and scans cost less
-    const int threads = std::min(kPlanThreads, std::max(128, (std::min(bv.n_docs_total, kMaxDocs) + 31) / 32 * 32));
+    // one thread per document of a request; barriers and scans cost less in a small block, the rotation tables (64 slices
+    // per kept document) want many threads: 256 is the measured optimum for batches of up to 256 documents
+    const int threads = std::min(kPlanThreads, std::max(256, (std::min(bv.n_docs_total, kMaxDocs) + 31) / 32 * 32));
     plan_kernel<<<bv.n_requests, threads, 0, stream>>>(gv, bv, pv, inv_freq, mode, order, kept_count,
                                                            query_start, score_accum, keep,
                                                            keep_per_request, strategy);
